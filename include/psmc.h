@@ -1,0 +1,194 @@
+/*
+ * psmc -- the per-token Power-SMC step on one NVIDIA B200 (sm_100a), C-ABI.
+ *
+ * Everything here runs in hand-written CUDA kernels; there is no CPU fallback.
+ * The calls follow Algorithm 1 of the paper: N particles per prompt ("group"),
+ * G independent groups, R = G*N rows.  One decoded token is one psmc_step()
+ * (rows 5-11 of Algorithm 1: proposal, draw, weight update of Eq. 7, EOS
+ * handling, normalisation and ESS of Eq. 5, ESS-triggered systematic
+ * resampling) followed by psmc_reindex_kv() (row 14, Appendix C) and, after the
+ * last token, psmc_select() (row 18).
+ *
+ * Conventions
+ *   - Every call returns a psmc_status; nothing throws or aborts.
+ *   - "DEVICE" pointers are CUDA global-memory addresses on the context's
+ *     device; "HOST" pointers are ordinary process memory.  The caller owns
+ *     every buffer it passes; the context owns its own state.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All work is stream-ordered and asynchronous unless a call says it syncs.
+ *     Calls on one context must be issued on one stream (or be ordered by the
+ *     caller): they share the context's scratch memory.
+ *   - Errors the host can see (null pointer, size out of range, step beyond
+ *     T_max) return at once and enqueue nothing.  Errors only the device can
+ *     see (a NaN or +inf logit, a row without finite logits, a hazardous gather
+ *     vector, a bounded wait that ran out) set a sticky device status word that
+ *     psmc_sync_status() returns; the kernels never trap.
+ *   - Randomness is a counter hash, so a run is a pure function of (seed,
+ *     inputs): sm64(x) is the splitmix64 finaliser of x + 0x9E3779B97F4A7C15;
+ *     H(a,b,c,d,e) = sm64(sm64(sm64(sm64(sm64(a)^b)^c)^d)^e); a uniform is
+ *     ((H >> 12) + 0.5) * 2^-52.  Streams: H(seed,1,group,t,slot) token draw,
+ *     H(seed,2,group,t,0) resampling offset, H(seed,3,group,0,0) final draw.
+ */
+#ifndef PSMC_H
+#define PSMC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct psmc_ctx psmc_ctx; /* opaque, owned by the library */
+
+typedef enum {
+    PSMC_OK = 0,
+    PSMC_E_INVAL = 1,   /* bad argument                                            */
+    PSMC_E_NOMEM = 2,   /* device or host allocation failed                        */
+    PSMC_E_CUDA = 3,    /* a CUDA runtime call failed                              */
+    PSMC_E_STATE = 4,   /* call out of order (e.g. step beyond T_max)              */
+    PSMC_E_NUMERIC = 5, /* NaN / +inf logit, or a row with no finite logit         */
+    PSMC_E_TIMEOUT = 6, /* a bounded device-side wait gave up                      */
+    PSMC_E_HAZARD = 7   /* in-place gather vector reads a row that is also written */
+} psmc_status;
+
+typedef enum { PSMC_F32 = 0, PSMC_BF16 = 1 } psmc_dtype;
+
+/* ------------------------------------------------------------------------- */
+/* Context (inputs of Algorithm 1: alpha, N, kappa, T_max, proposal)          */
+/* ------------------------------------------------------------------------- */
+
+/* One group.  N particles (1..1024), V vocabulary size (>= 2), alpha >= 1 the
+ * power exponent of Eq. 1, tau > 0 the proposal temperature at full alpha
+ * (Corollary 1: tau = 1/alpha is the variance-optimal choice), ess_thresh =
+ * kappa in (0,1] (resample when ESS < kappa*N, row 12), ramp = T_ramp tokens of
+ * linear exponent bridging (Section 4.3; 0 = off), eos_id in [0,V).  History
+ * capacity T_max = 4096, initial KV length 0.  Allocates device state on the
+ * current CUDA device. */
+psmc_status psmc_init(psmc_ctx** out, int N, int V, float alpha, float tau, float ess_thresh,
+                      int ramp, uint64_t seed, int eos_id);
+
+/* G independent groups with per-group initial KV length (HOST array [G], may
+ * be NULL = 0) and history capacity T_max steps. */
+psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, float alpha, float tau,
+                              float ess_thresh, int ramp, uint64_t seed, int eos_id, int T_max,
+                              const int32_t* prompt_len_host);
+
+psmc_status psmc_destroy(psmc_ctx*);                 /* syncs the device, frees everything   */
+psmc_status psmc_reset(psmc_ctx*, uint64_t seed);    /* t=0, weights 1, S=0, done=0; syncs    */
+
+/* ------------------------------------------------------------------------- */
+/* One token (Algorithm 1 rows 4-17 without the cache move)                   */
+/* ------------------------------------------------------------------------- */
+
+/* logits: DEVICE [R, V] row-major, row stride `ld` elements (>= V), dtype dt.
+ * Rows whose start is 16-byte aligned take the 128-bit load path (base pointer
+ * 16-byte aligned and ld*sizeof(elem) a multiple of 16); otherwise a scalar
+ * path is used.  Finished rows are not read.  On return (stream-ordered) the
+ * views below hold this step's results. */
+psmc_status psmc_step(psmc_ctx*, const void* logits, psmc_dtype dt, int64_t ld, void* stream);
+
+/* The same step fed from HOST memory: copies [R,V] logits (row stride ld) to a
+ * staging buffer owned by the context, runs the step, copies the R drawn
+ * tokens (as seen by each slot after resampling, i.e. the next LM input) back
+ * to tokens_out_host, and synchronises the stream.  Pinned host memory makes
+ * the copies asynchronous with respect to the host until that final sync. */
+psmc_status psmc_step_host(psmc_ctx*, const void* logits_host, psmc_dtype dt, int64_t ld,
+                           int32_t* tokens_out_host, void* stream);
+
+/* Stateless form of the logit pass alone (Eq. 7 with the proposal of
+ * Corollary 1): for each row r with done[r]==0 computes L1 = logsumexp(l),
+ * Lb = logsumexp(beta*l), draws y = min{v : sum_{u<=v} exp(beta*l_u) >= U_r *
+ * sum_all} and writes tok[r] = y, logp[r] = l_y - L1, loginc[r] = alpha_t *
+ * logp[r] - (beta*l_y - Lb).  All pointers DEVICE.  u: [R] uniforms in (0,1).
+ * done may be NULL (all live); rows with done[r]!=0 are left untouched.
+ * scratch: at least psmc_logits_pass_scratch_bytes(R, V) bytes, 256-byte
+ * aligned, zero-filled before the FIRST use (the pass leaves it zeroed again);
+ * status_word: one int32, sticky PSMC_E_* code (0 = fine). */
+size_t psmc_logits_pass_scratch_bytes(int R, int V);
+psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R, int V, int64_t ld,
+                             double beta, double alpha_t, const double* u, const uint8_t* done,
+                             void* scratch, size_t scratch_bytes, int32_t* tok, double* logp,
+                             double* loginc, int32_t* status_word, void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* KV-cache reindex (Algorithm 1 row 14, Appendix C)                          */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+    int n_layers;
+    void* const* k;        /* HOST array [n_layers] of DEVICE pointers, each [R, H, max_len, D] */
+    void* const* v;        /* same for values                                                   */
+    int n_kv_heads;        /* H */
+    int head_dim;          /* D */
+    int max_len;
+    psmc_dtype dt;
+    int64_t stride_row;    /* elements between rows (particles)                    */
+    int64_t stride_head;   /* elements between heads; (position, dim) is contiguous */
+} psmc_kv_desc;
+
+/* Applies the slot map of the most recent step to caller-owned caches: for
+ * every layer, K and V, head h and slot k with map[k] != k, positions
+ * [0, len) of row map[k] are copied onto row k, where len is the live length
+ * of the source row; the tail of row k is not touched.  Groups that did not
+ * resample move nothing, and a step without any resampling returns after
+ * reading one device counter (no host sync either way).
+ *   dst == NULL: in place on src.  The step's own slot map never reads a row it
+ *     writes.  idx_override (DEVICE [R], may be NULL) replaces the map by an
+ *     arbitrary gather vector with ROW indices in [0,R) and full-length copies
+ *     (max_len positions); in place it must be hazard-free, else
+ *     PSMC_E_HAZARD is raised in the status word and nothing is written.
+ *   dst != NULL: out-of-place gather dst[k] = src[idx[k]] for every k (also
+ *     idx[k]==k), i.e. index_select on the particle dimension.
+ * The bulk-copy (TMA) path needs 16-byte aligned row/head starts and
+ * head_dim*sizeof(elem) a multiple of 16; otherwise a plain-load path runs. */
+psmc_status psmc_reindex_kv(psmc_ctx*, const psmc_kv_desc* src, const psmc_kv_desc* dst,
+                            const int32_t* idx_override, void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Output (Algorithm 1 row 18)                                                */
+/* ------------------------------------------------------------------------- */
+
+/* Per group draws I ~ Categorical(W) from the current weights and writes the
+ * token string of particle I.  DEVICE outputs: out_tokens [G, T_max] (the
+ * first t entries are tokens, EOS repeated after termination, the rest -1),
+ * out_len [G] (tokens up to and including the first EOS, else t), out_index
+ * [G] (the slot I).  Any of them may be NULL. */
+psmc_status psmc_select(psmc_ctx*, int32_t* out_tokens, int32_t* out_len, int32_t* out_index,
+                        void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Views of the context state: DEVICE pointers, valid until psmc_destroy;      */
+/* contents are those of the most recent step once the stream has reached it.  */
+/* ------------------------------------------------------------------------- */
+const int32_t* psmc_tokens(psmc_ctx*);       /* [R] token drawn by each slot in the last step            */
+const int32_t* psmc_last_tokens(psmc_ctx*);  /* [R] last token of the particle now in each slot          */
+const double*  psmc_log_weights(psmc_ctx*);  /* [R] unnormalised log W after the step (0 after resample) */
+const double*  psmc_log_inc(psmc_ctx*);      /* [R] log omega of the last step (Eq. 7)                   */
+const double*  psmc_logp_tok(psmc_ctx*);     /* [R] log p(y_t) of the last step                          */
+const double*  psmc_cum_logp(psmc_ctx*);     /* [R] S = log p(y_{1:t})                                   */
+const int32_t* psmc_ancestors(psmc_ctx*);    /* [R] systematic-resampling ancestors A (identity if none) */
+const int32_t* psmc_slot_map(psmc_ctx*);     /* [R] hazard-free map applied to state and KV              */
+const int32_t* psmc_resampled(psmc_ctx*);    /* [G] 0/1                                                  */
+const double*  psmc_ess(psmc_ctx*);          /* [G] ESS of Eq. 5 before resampling                       */
+const double*  psmc_log_z(psmc_ctx*);        /* [G] running log of the normaliser estimate               */
+const int32_t* psmc_lens(psmc_ctx*);         /* [R] live KV length                                       */
+const uint8_t* psmc_done(psmc_ctx*);         /* [R]                                                      */
+const int32_t* psmc_move_count(psmc_ctx*);   /* [1] slots rewritten by the last step's maps              */
+
+int psmc_step_index(const psmc_ctx*);        /* t: tokens decoded so far                                 */
+int psmc_rows(const psmc_ctx*);              /* R                                                        */
+
+/* Overwrite particle state from HOST arrays [R] (any may be NULL = keep);
+ * synchronises.  For unit tests and for resuming a saved run. */
+psmc_status psmc_set_state(psmc_ctx*, const double* log_w, const double* cum_logp,
+                           const uint8_t* done, const int32_t* lens);
+
+/* Synchronises `stream` and returns the sticky device status word (PSMC_OK if
+ * nothing went wrong since the last reset). */
+psmc_status psmc_sync_status(psmc_ctx*, void* stream);
+const char* psmc_strerror(psmc_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSMC_H */

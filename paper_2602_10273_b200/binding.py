@@ -1,0 +1,281 @@
+"""Thin ctypes binding of libpsmc.so: same names as include/psmc.h, argument marshalling only.
+
+Every step of the path runs in the CUDA kernels of the library; nothing here computes.  The
+library must have been built (``python -m paper_2602_10273_b200.build``); a missing or unloadable
+library is an error, never a reason to fall back to anything else.  torch supplies device memory
+and the stream: tensors are passed as ``data_ptr()``, the stream as ``cuda_stream``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK, E_INVAL, E_NOMEM, E_CUDA, E_STATE, E_NUMERIC, E_TIMEOUT, E_HAZARD = range(8)
+F32, BF16 = 0, 1
+
+_lib = None
+
+
+class PsmcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().psmc_strerror(code).decode() if _lib is not None else str(code)
+        super().__init__("%s: %s (status %d)" % (where, msg, code))
+
+
+class KvDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("k", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)),
+                ("n_kv_heads", C.c_int), ("head_dim", C.c_int), ("max_len", C.c_int), ("dt", C.c_int),
+                ("stride_row", C.c_int64), ("stride_head", C.c_int64)]
+
+
+def lib():
+    """Load libpsmc.so (once).  Raises if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_build.LIB):
+            raise ImportError("libpsmc.so is missing at %s: run `python -m paper_2602_10273_b200.build` "
+                              "(nvcc, sm_100a); this package has no CPU or eager fallback" % _build.LIB)
+        L = C.CDLL(_build.LIB)
+        vp, i32p, f64p, u8p = C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p
+        L.psmc_init.restype = C.c_int
+        L.psmc_init.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_float, C.c_float, C.c_float, C.c_int,
+                                C.c_uint64, C.c_int]
+        L.psmc_init_batched.restype = C.c_int
+        L.psmc_init_batched.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float,
+                                        C.c_int, C.c_uint64, C.c_int, C.c_int, C.POINTER(C.c_int32)]
+        L.psmc_destroy.restype = C.c_int
+        L.psmc_destroy.argtypes = [vp]
+        L.psmc_reset.restype = C.c_int
+        L.psmc_reset.argtypes = [vp, C.c_uint64]
+        L.psmc_step.restype = C.c_int
+        L.psmc_step.argtypes = [vp, vp, C.c_int, C.c_int64, vp]
+        L.psmc_step_host.restype = C.c_int
+        L.psmc_step_host.argtypes = [vp, vp, C.c_int, C.c_int64, vp, vp]
+        L.psmc_logits_pass_scratch_bytes.restype = C.c_size_t
+        L.psmc_logits_pass_scratch_bytes.argtypes = [C.c_int, C.c_int]
+        L.psmc_logits_pass.restype = C.c_int
+        L.psmc_logits_pass.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_double, C.c_double, f64p, u8p,
+                                       vp, C.c_size_t, i32p, f64p, f64p, i32p, vp]
+        L.psmc_reindex_kv.restype = C.c_int
+        L.psmc_reindex_kv.argtypes = [vp, C.POINTER(KvDesc), C.POINTER(KvDesc), i32p, vp]
+        L.psmc_select.restype = C.c_int
+        L.psmc_select.argtypes = [vp, i32p, i32p, i32p, vp]
+        for name in ("psmc_tokens", "psmc_last_tokens", "psmc_log_weights", "psmc_log_inc", "psmc_logp_tok",
+                     "psmc_cum_logp", "psmc_ancestors", "psmc_slot_map", "psmc_resampled", "psmc_ess",
+                     "psmc_log_z", "psmc_lens", "psmc_done", "psmc_move_count"):
+            f = getattr(L, name)
+            f.restype = C.c_void_p
+            f.argtypes = [vp]
+        L.psmc_step_index.restype = C.c_int
+        L.psmc_step_index.argtypes = [vp]
+        L.psmc_rows.restype = C.c_int
+        L.psmc_rows.argtypes = [vp]
+        L.psmc_set_state.restype = C.c_int
+        L.psmc_set_state.argtypes = [vp, vp, vp, vp, vp]
+        L.psmc_sync_status.restype = C.c_int
+        L.psmc_sync_status.argtypes = [vp, vp]
+        L.psmc_strerror.restype = C.c_char_p
+        L.psmc_strerror.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise PsmcError(code, where)
+
+
+def _ptr(t) -> int:
+    """Device or host address of a tensor / numpy array / raw int (None -> NULL)."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("logits / KV must be float32 or bfloat16, got %s" % t.dtype)
+
+
+_VIEW_DTYPES = {"psmc_tokens": torch.int32, "psmc_last_tokens": torch.int32, "psmc_log_weights": torch.float64,
+                "psmc_log_inc": torch.float64, "psmc_logp_tok": torch.float64, "psmc_cum_logp": torch.float64,
+                "psmc_ancestors": torch.int32, "psmc_slot_map": torch.int32, "psmc_resampled": torch.int32,
+                "psmc_ess": torch.float64, "psmc_log_z": torch.float64, "psmc_lens": torch.int32,
+                "psmc_done": torch.uint8, "psmc_move_count": torch.int32}
+
+
+_TYPESTR = {torch.int32: "<i4", torch.float64: "<f8", torch.uint8: "|u1"}
+
+
+class _DevArray:
+    """Minimal __cuda_array_interface__ carrier so torch can wrap a raw device pointer."""
+
+    def __init__(self, addr: int, n: int, dtype: torch.dtype):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": _TYPESTR[dtype], "data": (addr, False),
+                                         "version": 2, "strides": None}
+
+
+class Psmc:
+    """Handle on a psmc_ctx.  Methods carry the C names without the prefix."""
+
+    def __init__(self, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, G=1, T_max=4096, prompt_len=None):
+        self._h = C.c_void_p()
+        self.G, self.N, self.V, self.R, self.T_max = G, N, V, G * N, T_max
+        pl = None
+        if prompt_len is not None:
+            pl = np.ascontiguousarray(prompt_len, dtype=np.int32)
+            assert pl.size == G
+        code = lib().psmc_init_batched(C.byref(self._h), G, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, T_max,
+                                       None if pl is None else pl.ctypes.data_as(C.POINTER(C.c_int32)))
+        _check(code, "psmc_init_batched")
+        self._kv_keepalive = None
+
+    def destroy(self):
+        if self._h:
+            lib().psmc_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def reset(self, seed):
+        _check(lib().psmc_reset(self._h, seed), "psmc_reset")
+
+    def step(self, logits: torch.Tensor, stream=None):
+        """logits: CUDA tensor [R, V] (float32 / bfloat16), unit stride along V."""
+        assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1 and logits.shape == (self.R, self.V)
+        _check(lib().psmc_step(self._h, logits.data_ptr(), _dtype_code(logits), logits.stride(0), _stream(stream)),
+               "psmc_step")
+
+    def step_host(self, logits: torch.Tensor, tokens_out: torch.Tensor, stream=None):
+        """logits: HOST tensor [R, V] (ideally pinned); tokens_out: HOST int32 [R]."""
+        assert not logits.is_cuda and not tokens_out.is_cuda and tokens_out.dtype == torch.int32
+        assert logits.dim() == 2 and logits.stride(1) == 1 and logits.shape == (self.R, self.V)
+        _check(lib().psmc_step_host(self._h, logits.data_ptr(), _dtype_code(logits), logits.stride(0),
+                                    tokens_out.data_ptr(), _stream(stream)), "psmc_step_host")
+
+    def make_kv_desc(self, k_layers, v_layers):
+        """k_layers / v_layers: lists of CUDA tensors [R, H, max_len, D] with (max_len, D) contiguous."""
+        k0 = k_layers[0]
+        R, H, L, D = k0.shape
+        assert R == self.R and k0.stride(3) == 1 and k0.stride(2) == D
+        n = len(k_layers)
+        ka = (C.c_void_p * n)(*[t.data_ptr() for t in k_layers])
+        va = (C.c_void_p * n)(*[t.data_ptr() for t in v_layers])
+        for t in list(k_layers) + list(v_layers):
+            assert t.shape == k0.shape and t.stride() == k0.stride() and t.dtype == k0.dtype and t.is_cuda
+        d = KvDesc(n, C.cast(ka, C.POINTER(C.c_void_p)), C.cast(va, C.POINTER(C.c_void_p)), H, D, L,
+                   _dtype_code(k0), k0.stride(0), k0.stride(1))
+        d._keep = (ka, va, list(k_layers), list(v_layers))
+        return d
+
+    def reindex_kv(self, src: KvDesc, dst: KvDesc = None, idx_override: torch.Tensor = None, stream=None):
+        if idx_override is not None:
+            assert idx_override.is_cuda and idx_override.dtype == torch.int32 and idx_override.numel() == self.R
+        _check(lib().psmc_reindex_kv(self._h, C.byref(src), None if dst is None else C.byref(dst),
+                                     _ptr(idx_override), _stream(stream)), "psmc_reindex_kv")
+
+    def select(self, out_tokens=None, out_len=None, out_index=None, stream=None):
+        dev = torch.device("cuda", torch.cuda.current_device())
+        if out_tokens is None:
+            out_tokens = torch.empty((self.G, self.T_max), dtype=torch.int32, device=dev)
+        if out_len is None:
+            out_len = torch.empty(self.G, dtype=torch.int32, device=dev)
+        if out_index is None:
+            out_index = torch.empty(self.G, dtype=torch.int32, device=dev)
+        _check(lib().psmc_select(self._h, out_tokens.data_ptr(), out_len.data_ptr(), out_index.data_ptr(),
+                                 _stream(stream)), "psmc_select")
+        return out_tokens, out_len, out_index
+
+    def set_state(self, log_w=None, cum_logp=None, done=None, lens=None):
+        a = None if log_w is None else np.ascontiguousarray(log_w, dtype=np.float64)
+        b = None if cum_logp is None else np.ascontiguousarray(cum_logp, dtype=np.float64)
+        c = None if done is None else np.ascontiguousarray(done, dtype=np.uint8)
+        d = None if lens is None else np.ascontiguousarray(lens, dtype=np.int32)
+        _check(lib().psmc_set_state(self._h, _ptr(a), _ptr(b), _ptr(c), _ptr(d)), "psmc_set_state")
+
+    def sync_status(self, stream=None) -> int:
+        return lib().psmc_sync_status(self._h, _stream(stream))
+
+    @property
+    def step_index(self) -> int:
+        return lib().psmc_step_index(self._h)
+
+    def device_view(self, name: str, n: int) -> torch.Tensor:
+        """The library-owned device array behind a view accessor, wrapped (not copied) as a CUDA tensor."""
+        addr = getattr(lib(), name)(self._h)
+        return torch.as_tensor(_DevArray(addr, n, _VIEW_DTYPES[name]), device="cuda")
+
+    def _view(self, name: str, n: int) -> torch.Tensor:
+        """Copy of a device view as a CPU tensor (synchronises the current stream)."""
+        return self.device_view(name, n).cpu()
+
+    def view_ptr(self, name: str) -> int:
+        """Raw device address of a state view (e.g. 'psmc_last_tokens')."""
+        return getattr(lib(), name)(self._h)
+
+    tokens = property(lambda s: s._view("psmc_tokens", s.R))
+    last_tokens = property(lambda s: s._view("psmc_last_tokens", s.R))
+    log_weights = property(lambda s: s._view("psmc_log_weights", s.R))
+    log_inc = property(lambda s: s._view("psmc_log_inc", s.R))
+    logp_tok = property(lambda s: s._view("psmc_logp_tok", s.R))
+    cum_logp = property(lambda s: s._view("psmc_cum_logp", s.R))
+    ancestors = property(lambda s: s._view("psmc_ancestors", s.R))
+    slot_map = property(lambda s: s._view("psmc_slot_map", s.R))
+    resampled = property(lambda s: s._view("psmc_resampled", s.G))
+    ess = property(lambda s: s._view("psmc_ess", s.G))
+    log_z = property(lambda s: s._view("psmc_log_z", s.G))
+    lens = property(lambda s: s._view("psmc_lens", s.R))
+    done = property(lambda s: s._view("psmc_done", s.R))
+    move_count = property(lambda s: int(s._view("psmc_move_count", 1)[0]))
+
+
+def init(N, V, alpha, tau, ess_thresh, ramp, seed, eos_id) -> Psmc:
+    """psmc_init: one group."""
+    return Psmc(N, V, alpha, tau, ess_thresh, ramp, seed, eos_id)
+
+
+def init_batched(G, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, T_max, prompt_len=None) -> Psmc:
+    """psmc_init_batched: G independent groups."""
+    return Psmc(N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, G=G, T_max=T_max, prompt_len=prompt_len)
+
+
+def logits_pass_scratch_bytes(R: int, V: int) -> int:
+    return lib().psmc_logits_pass_scratch_bytes(R, V)
+
+
+def logits_pass(logits: torch.Tensor, beta: float, alpha_t: float, u: torch.Tensor, done, scratch: torch.Tensor,
+                tok: torch.Tensor, logp: torch.Tensor, loginc: torch.Tensor, status_word: torch.Tensor, stream=None):
+    """psmc_logits_pass: the stateless logit pass.  All tensors on the GPU; scratch zero-filled uint8."""
+    R, V = logits.shape
+    assert logits.stride(1) == 1 and u.dtype == torch.float64 and tok.dtype == torch.int32
+    _check(lib().psmc_logits_pass(logits.data_ptr(), _dtype_code(logits), R, V, logits.stride(0), beta, alpha_t,
+                                  u.data_ptr(), _ptr(done), scratch.data_ptr(), scratch.numel() * scratch.element_size(),
+                                  tok.data_ptr(), logp.data_ptr(), loginc.data_ptr(), status_word.data_ptr(),
+                                  _stream(stream)), "psmc_logits_pass")

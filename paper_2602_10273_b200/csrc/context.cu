@@ -1,0 +1,335 @@
+// Context, argument checks and the extern "C" face of libpsmc.so.  The arithmetic of the step
+// lives in the kernels; this file owns device state, computes the exponent schedule of
+// Section 4.3 for the token at hand and enqueues the kernels on the caller's stream.
+#include <new>
+#include <string.h>
+
+#include "internal.h"
+
+using namespace psmc;
+
+struct psmc_ctx {
+    int device;
+    int G, N, V, R, ramp, eos, T_max, t;
+    double alpha, tau, kappa;
+    uint64_t seed;
+    int32_t* prompt_len_host;  // [G]
+    // particle state
+    double *logW, *S;
+    uint8_t* done;
+    int32_t* len;
+    // results of the last step
+    int32_t *tok_draw, *tok, *last_tok, *anc, *map, *resampled;
+    double *logp, *loginc, *ess, *logZ;
+    // ancestry log for psmc_select
+    int32_t *hist_tok, *hist_map;  // [T_max][R]
+    // move records: [0] from the step, [1] from an idx_override
+    MoveSource* sources[2];
+    int32_t* dst_rows[2];
+    int32_t* counts[2];  // {n_sources, n_moves}
+    int32_t* status;
+    void* scratch;       // logit-pass tickets and span triples
+    void* staging;       // psmc_step_host: device copy of the host logits
+    size_t staging_bytes;
+};
+
+namespace {
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t count) {
+    return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(T));
+}
+
+// Section 4.3 with one stage per token: alpha_t = 1 + (alpha - 1) * min(t, T_ramp) / T_ramp
+double alpha_at(const psmc_ctx* c, int t) {
+    if (c->ramp <= 0) return c->alpha;
+    const int s = t < c->ramp ? t : c->ramp;
+    return 1.0 + (c->alpha - 1.0) * (double)s / (double)c->ramp;
+}
+
+psmc_status reset_device_state(psmc_ctx* c) {
+    const size_t R = (size_t)c->R, G = (size_t)c->G;
+    cudaError_t e = cudaSuccess;
+    auto z = [&](void* p, size_t bytes) { if (e == cudaSuccess) e = cudaMemset(p, 0, bytes); };
+    z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
+    z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
+    z(c->counts[0], 8); z(c->counts[1], 8); z(c->status, 4);
+    z(c->scratch, logits_pass_scratch_bytes(c->R, c->V));
+    if (e != cudaSuccess) return PSMC_E_CUDA;
+    // lens = prompt length of the group; identity maps; tokens -1; ESS = N
+    int32_t* h = new (std::nothrow) int32_t[R];
+    double* hd = new (std::nothrow) double[G];
+    if (!h || !hd) { delete[] h; delete[] hd; return PSMC_E_NOMEM; }
+    for (size_t r = 0; r < R; ++r) h[r] = c->prompt_len_host[r / c->N];
+    e = cudaMemcpy(c->len, h, 4 * R, cudaMemcpyHostToDevice);
+    for (size_t r = 0; r < R; ++r) h[r] = (int32_t)(r % c->N);
+    if (e == cudaSuccess) e = cudaMemcpy(c->anc, h, 4 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(c->map, h, 4 * R, cudaMemcpyHostToDevice);
+    for (size_t r = 0; r < R; ++r) h[r] = -1;
+    if (e == cudaSuccess) e = cudaMemcpy(c->tok, h, 4 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(c->tok_draw, h, 4 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(c->last_tok, h, 4 * R, cudaMemcpyHostToDevice);
+    for (size_t g = 0; g < G; ++g) hd[g] = (double)c->N;
+    if (e == cudaSuccess) e = cudaMemcpy(c->ess, hd, 8 * G, cudaMemcpyHostToDevice);
+    delete[] h;
+    delete[] hd;
+    c->t = 0;
+    return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+void free_ctx(psmc_ctx* c) {
+    if (!c) return;
+    void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok_draw, c->tok, c->last_tok, c->anc, c->map, c->resampled,
+                    c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
+                    c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->scratch, c->staging};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    delete[] c->prompt_len_host;
+    delete c;
+}
+
+}  // namespace
+
+extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, float alpha, float tau, float ess_thresh,
+                                         int ramp, uint64_t seed, int eos_id, int T_max,
+                                         const int32_t* prompt_len_host) {
+    if (!out) return PSMC_E_INVAL;
+    *out = nullptr;
+    if (G < 1 || N < 1 || N > kMaxParticles || V < 2 || !(alpha >= 1.f) || !(tau > 0.f) || !(ess_thresh > 0.f) ||
+        !(ess_thresh <= 1.f) || ramp < 0 || eos_id < 0 || eos_id >= V || T_max < 1)
+        return PSMC_E_INVAL;
+    if ((int64_t)G * N > (1 << 24)) return PSMC_E_INVAL;
+    psmc_ctx* c = new (std::nothrow) psmc_ctx();
+    if (!c) return PSMC_E_NOMEM;
+    memset(c, 0, sizeof(*c));
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return PSMC_E_CUDA; }
+    c->G = G; c->N = N; c->V = V; c->R = G * N; c->ramp = ramp; c->eos = eos_id; c->T_max = T_max;
+    c->alpha = (double)alpha; c->tau = (double)tau; c->kappa = (double)ess_thresh; c->seed = seed;
+    c->prompt_len_host = new (std::nothrow) int32_t[G];
+    if (!c->prompt_len_host) { free_ctx(c); return PSMC_E_NOMEM; }
+    for (int g = 0; g < G; ++g) {
+        c->prompt_len_host[g] = prompt_len_host ? prompt_len_host[g] : 0;
+        if (c->prompt_len_host[g] < 0) { free_ctx(c); return PSMC_E_INVAL; }
+    }
+    const size_t R = (size_t)c->R;
+    cudaError_t e = cudaSuccess;
+    auto ok = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
+    ok(dev_alloc(&c->logW, R)); ok(dev_alloc(&c->S, R)); ok(dev_alloc(&c->done, R)); ok(dev_alloc(&c->len, R));
+    ok(dev_alloc(&c->tok_draw, R)); ok(dev_alloc(&c->tok, R)); ok(dev_alloc(&c->last_tok, R));
+    ok(dev_alloc(&c->anc, R)); ok(dev_alloc(&c->map, R)); ok(dev_alloc(&c->resampled, (size_t)G));
+    ok(dev_alloc(&c->logp, R)); ok(dev_alloc(&c->loginc, R)); ok(dev_alloc(&c->ess, (size_t)G));
+    ok(dev_alloc(&c->logZ, (size_t)G));
+    ok(dev_alloc(&c->hist_tok, R * (size_t)T_max)); ok(dev_alloc(&c->hist_map, R * (size_t)T_max));
+    for (int s = 0; s < 2; ++s) {
+        ok(dev_alloc(&c->sources[s], R)); ok(dev_alloc(&c->dst_rows[s], R)); ok(dev_alloc(&c->counts[s], 2));
+    }
+    ok(dev_alloc(&c->status, 1));
+    ok(cudaMalloc(&c->scratch, logits_pass_scratch_bytes(c->R, c->V)));
+    if (e != cudaSuccess) { free_ctx(c); return e == cudaErrorMemoryAllocation ? PSMC_E_NOMEM : PSMC_E_CUDA; }
+    psmc_status st = reset_device_state(c);
+    if (st != PSMC_OK) { free_ctx(c); return st; }
+    if (cudaDeviceSynchronize() != cudaSuccess) { free_ctx(c); return PSMC_E_CUDA; }
+    *out = c;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_init(psmc_ctx** out, int N, int V, float alpha, float tau, float ess_thresh, int ramp,
+                                 uint64_t seed, int eos_id) {
+    return psmc_init_batched(out, 1, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, 4096, nullptr);
+}
+
+extern "C" psmc_status psmc_destroy(psmc_ctx* c) {
+    if (!c) return PSMC_E_INVAL;
+    cudaDeviceSynchronize();
+    free_ctx(c);
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_reset(psmc_ctx* c, uint64_t seed) {
+    if (!c) return PSMC_E_INVAL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    c->seed = seed;
+    psmc_status st = reset_device_state(c);
+    if (st != PSMC_OK) return st;
+    return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt, int64_t ld, void* stream) {
+    if (!c || !logits || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
+    if (c->t >= c->T_max) return PSMC_E_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int t = c->t + 1;
+    const double alpha_t = alpha_at(c, t), alpha_prev = alpha_at(c, t - 1);
+    const double beta_t = alpha_t / (c->alpha * c->tau);  // tau = 1/alpha gives beta_t = alpha_t (Corollary 1)
+
+    LogitsPassArgs la{};
+    la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld;
+    la.beta = beta_t; la.alpha_t = alpha_t; la.u = nullptr; la.seed = c->seed; la.t = t; la.N = c->N;
+    la.done = c->done; la.scratch = c->scratch; la.tok = c->tok_draw; la.logp = c->logp; la.loginc = c->loginc;
+    la.status = c->status;
+    la.zero_words = c->counts[0];  // the step's two move counters are cleared by the first kernel of the step
+    if (launch_logits_pass(la, s) != cudaSuccess) return PSMC_E_CUDA;
+
+    WeightsArgs wa{};
+    wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos;
+    wa.alpha_t = alpha_t; wa.delta = alpha_t - alpha_prev; wa.kappa = c->kappa; wa.seed = c->seed;
+    wa.tok_draw = c->tok_draw; wa.logp = c->logp; wa.loginc = c->loginc;
+    wa.logW = c->logW; wa.S = c->S; wa.done = c->done; wa.len = c->len;
+    wa.tok = c->tok; wa.last_tok = c->last_tok; wa.anc = c->anc; wa.map = c->map;
+    wa.resampled = c->resampled; wa.ess = c->ess; wa.logZ = c->logZ;
+    wa.hist_tok = c->hist_tok + (size_t)(t - 1) * c->R;
+    wa.hist_map = c->hist_map + (size_t)(t - 1) * c->R;
+    wa.sources = c->sources[0]; wa.dst_rows = c->dst_rows[0];
+    wa.n_sources = c->counts[0]; wa.n_moves = c->counts[0] + 1;
+    wa.status = c->status;
+    if (launch_weights_resample(wa, s) != cudaSuccess) return PSMC_E_CUDA;
+    c->t = t;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_step_host(psmc_ctx* c, const void* logits_host, psmc_dtype dt, int64_t ld,
+                                      int32_t* tokens_out_host, void* stream) {
+    if (!c || !logits_host || !tokens_out_host || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16))
+        return PSMC_E_INVAL;
+    if (c->t >= c->T_max) return PSMC_E_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esize = dt == PSMC_F32 ? 4 : 2;
+    // staging rows are padded to 16 bytes so that the 128-bit load path applies
+    const int64_t ld_dev = ((int64_t)c->V * esize + 15) / 16 * 16 / esize;
+    const size_t need = (size_t)c->R * ld_dev * esize;
+    if (c->staging_bytes < need) {
+        if (c->staging) { cudaStreamSynchronize(s); cudaFree(c->staging); c->staging = nullptr; c->staging_bytes = 0; }
+        if (cudaMalloc(&c->staging, need) != cudaSuccess) return PSMC_E_NOMEM;
+        c->staging_bytes = need;
+    }
+    if (cudaMemcpy2DAsync(c->staging, ld_dev * esize, logits_host, ld * esize, (size_t)c->V * esize, c->R,
+                          cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PSMC_E_CUDA;
+    psmc_status st = psmc_step(c, c->staging, dt, ld_dev, stream);
+    if (st != PSMC_OK) return st;
+    if (cudaMemcpyAsync(tokens_out_host, c->last_tok, 4 * (size_t)c->R, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return PSMC_E_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, const psmc_kv_desc* dst,
+                                       const int32_t* idx_override, void* stream) {
+    if (!c || !src || !src->k || !src->v) return PSMC_E_INVAL;
+    if (src->n_layers < 1 || src->n_kv_heads < 1 || src->head_dim < 1 || src->max_len < 1) return PSMC_E_INVAL;
+    if (src->dt != PSMC_F32 && src->dt != PSMC_BF16) return PSMC_E_INVAL;
+    const int64_t min_head = (int64_t)src->max_len * src->head_dim;
+    if (src->stride_head < min_head || src->stride_row < (int64_t)src->n_kv_heads * src->stride_head)
+        return PSMC_E_INVAL;
+    if (dst) {
+        if (!dst->k || !dst->v || !idx_override) return PSMC_E_INVAL;  // out of place needs an explicit gather vector
+        if (dst->n_layers != src->n_layers || dst->n_kv_heads != src->n_kv_heads || dst->head_dim != src->head_dim ||
+            dst->max_len != src->max_len || dst->dt != src->dt)
+            return PSMC_E_INVAL;
+        if (dst->stride_head < min_head || dst->stride_row < (int64_t)dst->n_kv_heads * dst->stride_head)
+            return PSMC_E_INVAL;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int set = idx_override ? 1 : 0;
+    if (idx_override) {
+        if (launch_build_moves(idx_override, c->R, src->max_len, dst ? 0 : 1, c->sources[1], c->dst_rows[1],
+                               c->counts[1], c->counts[1] + 1, c->status, s) != cudaSuccess)
+            return PSMC_E_CUDA;
+    }
+    const psmc_kv_desc* d = dst ? dst : src;
+    const int64_t esize = src->dt == PSMC_F32 ? 4 : 2;
+    KvLaunch k;
+    k.H = src->n_kv_heads;
+    k.row_bytes_stride = src->stride_row * esize;
+    k.head_bytes_stride = src->stride_head * esize;
+    k.dst_row_bytes_stride = d->stride_row * esize;
+    k.dst_head_bytes_stride = d->stride_head * esize;
+    k.pos_bytes = (int)(src->head_dim * esize);
+    k.max_len = src->max_len;
+    k.sources = c->sources[set];
+    k.dst_rows = c->dst_rows[set];
+    k.n_sources = c->counts[set];
+    k.status = c->status;
+    uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |
+                    (uint64_t)k.dst_head_bytes_stride | (uint64_t)k.pos_bytes;
+    for (int l = 0; l < src->n_layers; ++l) {
+        if (!src->k[l] || !src->v[l] || !d->k[l] || !d->v[l]) return PSMC_E_INVAL;
+        bits |= (uint64_t)(uintptr_t)src->k[l] | (uint64_t)(uintptr_t)src->v[l] | (uint64_t)(uintptr_t)d->k[l] |
+                (uint64_t)(uintptr_t)d->v[l];
+    }
+    k.bulk_ok = (bits % 16 == 0) ? 1 : 0;
+    for (int l0 = 0; l0 < src->n_layers; l0 += kMaxKvPtrs / 2) {
+        const int nl = src->n_layers - l0 < kMaxKvPtrs / 2 ? src->n_layers - l0 : kMaxKvPtrs / 2;
+        for (int l = 0; l < nl; ++l) {
+            k.src[2 * l] = static_cast<char*>(src->k[l0 + l]);
+            k.src[2 * l + 1] = static_cast<char*>(src->v[l0 + l]);
+            k.dst[2 * l] = static_cast<char*>(d->k[l0 + l]);
+            k.dst[2 * l + 1] = static_cast<char*>(d->v[l0 + l]);
+        }
+        k.n_ptrs = 2 * nl;
+        if (launch_reindex_kv(k, s) != cudaSuccess) return PSMC_E_CUDA;
+    }
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_select(psmc_ctx* c, int32_t* out_tokens, int32_t* out_len, int32_t* out_index,
+                                   void* stream) {
+    if (!c) return PSMC_E_INVAL;
+    SelectArgs a{};
+    a.G = c->G; a.N = c->N; a.R = c->R; a.t = c->t; a.T_max = c->T_max; a.eos = c->eos; a.seed = c->seed;
+    a.logW = c->logW; a.hist_tok = c->hist_tok; a.hist_map = c->hist_map;
+    a.out_tokens = out_tokens; a.out_len = out_len; a.out_index = out_index;
+    return launch_select(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_set_state(psmc_ctx* c, const double* log_w, const double* cum_logp, const uint8_t* done,
+                                      const int32_t* lens) {
+    if (!c) return PSMC_E_INVAL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    const size_t R = (size_t)c->R;
+    cudaError_t e = cudaSuccess;
+    if (log_w) e = cudaMemcpy(c->logW, log_w, 8 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && cum_logp) e = cudaMemcpy(c->S, cum_logp, 8 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && done) e = cudaMemcpy(c->done, done, R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && lens) e = cudaMemcpy(c->len, lens, 4 * R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_sync_status(psmc_ctx* c, void* stream) {
+    if (!c) return PSMC_E_INVAL;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PSMC_E_CUDA;
+    int32_t w = 0;
+    if (cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PSMC_E_CUDA;
+    return (psmc_status)w;
+}
+
+extern "C" const char* psmc_strerror(psmc_status s) {
+    switch (s) {
+        case PSMC_OK: return "ok";
+        case PSMC_E_INVAL: return "invalid argument";
+        case PSMC_E_NOMEM: return "out of memory";
+        case PSMC_E_CUDA: return "CUDA runtime error";
+        case PSMC_E_STATE: return "call out of order";
+        case PSMC_E_NUMERIC: return "NaN/+inf logit or a row without finite logits";
+        case PSMC_E_TIMEOUT: return "bounded device wait ran out";
+        case PSMC_E_HAZARD: return "in-place gather vector reads a row that is also written";
+    }
+    return "unknown status";
+}
+
+extern "C" const int32_t* psmc_tokens(psmc_ctx* c) { return c ? c->tok : nullptr; }
+extern "C" const int32_t* psmc_last_tokens(psmc_ctx* c) { return c ? c->last_tok : nullptr; }
+extern "C" const double* psmc_log_weights(psmc_ctx* c) { return c ? c->logW : nullptr; }
+extern "C" const double* psmc_log_inc(psmc_ctx* c) { return c ? c->loginc : nullptr; }
+extern "C" const double* psmc_logp_tok(psmc_ctx* c) { return c ? c->logp : nullptr; }
+extern "C" const double* psmc_cum_logp(psmc_ctx* c) { return c ? c->S : nullptr; }
+extern "C" const int32_t* psmc_ancestors(psmc_ctx* c) { return c ? c->anc : nullptr; }
+extern "C" const int32_t* psmc_slot_map(psmc_ctx* c) { return c ? c->map : nullptr; }
+extern "C" const int32_t* psmc_resampled(psmc_ctx* c) { return c ? c->resampled : nullptr; }
+extern "C" const double* psmc_ess(psmc_ctx* c) { return c ? c->ess : nullptr; }
+extern "C" const double* psmc_log_z(psmc_ctx* c) { return c ? c->logZ : nullptr; }
+extern "C" const int32_t* psmc_lens(psmc_ctx* c) { return c ? c->len : nullptr; }
+extern "C" const uint8_t* psmc_done(psmc_ctx* c) { return c ? c->done : nullptr; }
+extern "C" const int32_t* psmc_move_count(psmc_ctx* c) { return c ? c->counts[0] + 1 : nullptr; }
+extern "C" int psmc_step_index(const psmc_ctx* c) { return c ? c->t : -1; }
+extern "C" int psmc_rows(const psmc_ctx* c) { return c ? c->R : -1; }

@@ -1,0 +1,112 @@
+// Host-side declarations shared by the translation units of libpsmc.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/psmc.h"
+
+namespace psmc {
+
+constexpr int kMaxParticles = 1024;  // one CTA per group in the weight/resample kernel
+constexpr int kSMs = 148;            // B200
+
+// ---------------------------------------------------------------- logit pass (Eq. 7, Corollary 1)
+struct LogitsPassArgs {
+    const void* logits;
+    int dt;          // psmc_dtype
+    int R, V;
+    int64_t ld;
+    double beta, alpha_t;
+    const double* u;       // [R] uniforms, or NULL to hash (seed, token stream, row / N, t, row % N)
+    uint64_t seed;
+    int t, N;
+    const uint8_t* done;   // may be NULL
+    void* scratch;         // counters + partials
+    int32_t* tok;
+    double* logp;
+    double* loginc;
+    int32_t* status;
+    int32_t* zero_words;   // optional: two consecutive words the pass clears before anything else (may be NULL)
+};
+int logits_pass_span(int R, int V);               // elements per warp task
+size_t logits_pass_scratch_bytes(int R, int V);
+cudaError_t launch_logits_pass(const LogitsPassArgs& a, cudaStream_t stream);
+
+// ---------------------------------------------------------------- weights, ESS, resampling
+struct MoveSource {      // one surviving particle with surplus offspring
+    int32_t src_row;     // row to read
+    int32_t len;         // positions [0, len) to copy
+    int32_t dst_begin;   // first entry of its destinations in the destination list
+    int32_t n_dst;       // how many rows receive it
+};
+struct WeightsArgs {
+    int G, N, R, t, eos;
+    double alpha_t, delta, kappa;
+    uint64_t seed;
+    // from the logit pass
+    const int32_t* tok_draw;
+    double* logp;      // zeroed here for finished rows
+    double* loginc;
+    // particle state, updated in place
+    double* logW;
+    double* S;
+    uint8_t* done;
+    int32_t* len;
+    // per-step results
+    int32_t* tok;       // [R] token of each slot this step (EOS for finished rows)
+    int32_t* last_tok;  // [R] after the map
+    int32_t* anc;
+    int32_t* map;
+    int32_t* resampled; // [G]
+    double* ess;        // [G]
+    double* logZ;       // [G]
+    int32_t* hist_tok;  // row t-1 of [T_max][R]
+    int32_t* hist_map;
+    // move records for the cache reindex
+    MoveSource* sources;
+    int32_t* dst_rows;
+    int32_t* n_sources;  // [1]
+    int32_t* n_moves;    // [1]
+    int32_t* status;
+};
+cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream);
+
+// ---------------------------------------------------------------- KV reindex (Appendix C)
+constexpr int kMaxKvPtrs = 128;  // K and V pointers per launch (64 layers); more layers take more launches
+struct KvLaunch {
+    char* src[kMaxKvPtrs];
+    char* dst[kMaxKvPtrs];
+    int n_ptrs;
+    int H;
+    int64_t row_bytes_stride, head_bytes_stride;  // bytes
+    int64_t dst_row_bytes_stride, dst_head_bytes_stride;
+    int pos_bytes;   // head_dim * sizeof(elem)
+    int max_len;
+    const MoveSource* sources;
+    const int32_t* dst_rows;
+    const int32_t* n_sources;
+    int32_t* status;
+    int bulk_ok;     // 16-byte alignment holds everywhere
+};
+cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream);
+// turn an arbitrary gather vector into move records (and check in-place hazards)
+cudaError_t launch_build_moves(const int32_t* idx, int R, int max_len, int in_place, MoveSource* sources,
+                               int32_t* dst_rows, int32_t* n_sources, int32_t* n_moves, int32_t* status,
+                               cudaStream_t stream);
+
+// ---------------------------------------------------------------- final draw and back-trace
+struct SelectArgs {
+    int G, N, R, t, T_max, eos;
+    uint64_t seed;
+    const double* logW;
+    const int32_t* hist_tok;
+    const int32_t* hist_map;
+    int32_t* out_tokens;
+    int32_t* out_len;
+    int32_t* out_index;
+};
+cudaError_t launch_select(const SelectArgs& a, cudaStream_t stream);
+
+}  // namespace psmc

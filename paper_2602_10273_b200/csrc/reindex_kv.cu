@@ -1,0 +1,264 @@
+// KV-cache reindex (Algorithm 1 row 14, Appendix C): copy the live prefix of surviving rows
+// onto the rows of discarded particles, for every layer, K and V, and head.
+//
+// The move list comes from the resampling kernel as "sources": one record per surviving row
+// with surplus offspring, naming the rows that receive it.  A source chunk is read ONCE and
+// written to each of its destinations, so bytes moved = unique reads + writes.
+//
+// Bulk path (sm_100a): one warp per CTA; lane 0 drives a ring of shared-memory stages with the
+// TMA engine: cp.async.bulk global->shared (completion on an mbarrier), then cp.async.bulk
+// shared->global per destination (bulk async-groups).  No thread touches the payload, so the copy
+// is bit-exact by construction and the SM's load/store units stay idle.  No multicast anywhere.
+// Every mbarrier wait is bounded; on expiry the kernel raises PSMC_E_TIMEOUT, drains its own
+// copies and returns.  Plain path: 256 threads copy with ordinary loads/stores of the widest unit
+// the alignment allows; used when the 16-byte rules of bulk copies do not hold.
+#include "common.cuh"
+#include "internal.h"
+
+namespace psmc {
+namespace {
+
+constexpr int kChunk = 16384;   // bytes per stage
+constexpr int kStages = 4;
+constexpr int kBulkCtasPerSm = 3;
+constexpr uint32_t kWaitTries = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait: false when the tries ran out
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t k = 0; k < kWaitTries; ++k)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Work item w -> (source record, pointer/head segment, chunk) and its byte range.
+struct Item {
+    const char* src;
+    int64_t dst_off;  // byte offset inside a destination row-head segment = chunk * kChunk
+    int seg_ptr, seg_head;
+    int dst_begin, n_dst;
+    uint32_t bytes;
+};
+__device__ __forceinline__ bool decode(const KvLaunch& k, int64_t w, int n_seg, int n_chunk, int chunk_bytes, Item& it) {
+    const int chunk = (int)(w % n_chunk);
+    const int64_t q = w / n_chunk;
+    const int seg = (int)(q % n_seg);
+    const int s = (int)(q / n_seg);
+    const MoveSource ms = k.sources[s];
+    int len = ms.len < k.max_len ? ms.len : k.max_len;
+    const int64_t seg_bytes = (int64_t)len * k.pos_bytes;
+    const int64_t off = (int64_t)chunk * chunk_bytes;
+    if (off >= seg_bytes) return false;
+    it.seg_ptr = seg / k.H;
+    it.seg_head = seg - it.seg_ptr * k.H;
+    it.src = k.src[it.seg_ptr] + (int64_t)ms.src_row * k.row_bytes_stride + (int64_t)it.seg_head * k.head_bytes_stride + off;
+    it.dst_off = off;
+    it.dst_begin = ms.dst_begin;
+    it.n_dst = ms.n_dst;
+    const int64_t left = seg_bytes - off;
+    it.bytes = (uint32_t)(left < chunk_bytes ? left : chunk_bytes);
+    return true;
+}
+__device__ __forceinline__ char* dst_addr(const KvLaunch& k, const Item& it, int d) {
+    const int row = k.dst_rows[it.dst_begin + d];
+    return k.dst[it.seg_ptr] + (int64_t)row * k.dst_row_bytes_stride + (int64_t)it.seg_head * k.dst_head_bytes_stride +
+           it.dst_off;
+}
+
+__global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant__ KvLaunch k) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bars[kStages];
+    __shared__ Item ring[kStages];
+
+    const int n_src = *reinterpret_cast<const volatile int32_t*>(k.n_sources);
+    if (n_src <= 0) return;  // nothing resampled this step
+    if (threadIdx.x != 0) return;
+
+    for (int s = 0; s < kStages; ++s) mbar_init(&bars[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+
+    const int n_seg = k.n_ptrs * k.H;
+    const int n_chunk = (int)(((int64_t)k.max_len * k.pos_bytes + kChunk - 1) / kChunk);
+    const int64_t total = (int64_t)n_src * n_seg * n_chunk;
+
+    int64_t pw = blockIdx.x;
+    Item cand;
+    while (pw < total && !decode(k, pw, n_seg, n_chunk, kChunk, cand)) pw += gridDim.x;
+
+    int issued = 0, consumed = 0;
+    bool failed = false;
+    for (int i = 0;; ++i) {
+        // consume item i-(kStages-1): its load has had kStages-1 iterations to land
+        const int j = i - (kStages - 1);
+        if (j >= 0 && j < issued) {
+            const int slot = j % kStages;
+            if (!mbar_wait(&bars[slot], (uint32_t)((j / kStages) & 1))) {
+                failed = true;
+                break;
+            }
+            fence_async_smem();
+            const Item it = ring[slot];
+            for (int d = 0; d < it.n_dst; ++d) bulk_store(dst_addr(k, it, d), smem + (size_t)slot * kChunk, it.bytes);
+            bulk_commit();
+            ++consumed;
+        }
+        // produce item i into slot i % kStages, last used by item i-kStages
+        if (pw < total) {
+            const int slot = i % kStages;
+            if (i >= kStages) bulk_wait_read<1>();  // all store groups but the newest have read their stage
+            ring[slot] = cand;
+            mbar_expect_tx(&bars[slot], cand.bytes);
+            bulk_load(smem + (size_t)slot * kChunk, cand.src, cand.bytes, &bars[slot]);
+            ++issued;
+            pw += gridDim.x;
+            while (pw < total && !decode(k, pw, n_seg, n_chunk, kChunk, cand)) pw += gridDim.x;
+        } else if (consumed == issued) {
+            break;
+        }
+    }
+    if (failed) {
+        raise_status(k.status, PSMC_E_TIMEOUT);
+        // do not leave with loads still landing in this CTA's shared memory: bounded second wait
+        for (int j = consumed; j < issued; ++j) mbar_wait(&bars[j % kStages], (uint32_t)((j / kStages) & 1));
+    }
+    bulk_wait_all();
+}
+
+// ---- plain path: ordinary loads and stores of unit type U ----
+template <typename U>
+__global__ void __launch_bounds__(256) reindex_plain_kernel(const __grid_constant__ KvLaunch k) {
+    const int n_src = *reinterpret_cast<const volatile int32_t*>(k.n_sources);
+    if (n_src <= 0) return;
+    const int n_seg = k.n_ptrs * k.H;
+    const int n_chunk = (int)(((int64_t)k.max_len * k.pos_bytes + kChunk - 1) / kChunk);
+    const int64_t total = (int64_t)n_src * n_seg * n_chunk;
+    for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
+        Item it;
+        if (!decode(k, w, n_seg, n_chunk, kChunk, it)) continue;
+        const int n_units = it.bytes / (int)sizeof(U);
+        const U* s = reinterpret_cast<const U*>(it.src);
+        for (int e = threadIdx.x; e < n_units; e += blockDim.x) {
+            const U v = s[e];
+            for (int d = 0; d < it.n_dst; ++d) reinterpret_cast<U*>(dst_addr(k, it, d))[e] = v;
+        }
+    }
+}
+
+// ---- arbitrary gather vector -> move records, with the in-place hazard check ----
+__global__ void __launch_bounds__(1024) build_moves_kernel(const int32_t* idx, int R, int max_len, int in_place,
+                                                           MoveSource* sources, int32_t* dst_rows, int32_t* n_sources,
+                                                           int32_t* n_moves, int32_t* status) {
+    __shared__ int bad, count;
+    if (threadIdx.x == 0) {
+        bad = 0;
+        count = 0;
+    }
+    __syncthreads();
+    for (int kk = threadIdx.x; kk < R; kk += blockDim.x) {
+        const int s = idx[kk];
+        if (s < 0 || s >= R) {
+            atomicMax(&bad, PSMC_E_INVAL);
+        } else if (in_place && s != kk && idx[s] != s) {
+            atomicMax(&bad, PSMC_E_HAZARD);  // row s is read here and rewritten elsewhere
+        }
+    }
+    __syncthreads();
+    if (bad) {
+        if (threadIdx.x == 0) {
+            *n_sources = 0;
+            *n_moves = 0;
+            raise_status(status, bad);
+        }
+        return;
+    }
+    for (int kk = threadIdx.x; kk < R; kk += blockDim.x) {
+        const int s = idx[kk];
+        if (in_place && s == kk) continue;
+        const int pos = atomicAdd(&count, 1);
+        dst_rows[pos] = kk;
+        MoveSource ms;
+        ms.src_row = s;
+        ms.len = max_len;
+        ms.dst_begin = pos;
+        ms.n_dst = 1;
+        sources[pos] = ms;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        *n_sources = count;
+        *n_moves = count;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream) {
+    if (k.bulk_ok) {
+        static bool configured = false;
+        const int smem = kStages * kChunk;
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(reindex_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        reindex_bulk_kernel<<<kSMs * kBulkCtasPerSm, 32, smem, stream>>>(k);
+        return cudaGetLastError();
+    }
+    // widest unit that divides every address, stride and row size
+    uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |
+                    (uint64_t)k.dst_head_bytes_stride | (uint64_t)k.pos_bytes;
+    for (int i = 0; i < k.n_ptrs; ++i) bits |= (uint64_t)(uintptr_t)k.src[i] | (uint64_t)(uintptr_t)k.dst[i];
+    const int grid = kSMs * 8;
+    if (bits % 16 == 0) reindex_plain_kernel<uint4><<<grid, 256, 0, stream>>>(k);
+    else if (bits % 8 == 0) reindex_plain_kernel<uint2><<<grid, 256, 0, stream>>>(k);
+    else if (bits % 4 == 0) reindex_plain_kernel<uint32_t><<<grid, 256, 0, stream>>>(k);
+    else if (bits % 2 == 0) reindex_plain_kernel<uint16_t><<<grid, 256, 0, stream>>>(k);
+    else reindex_plain_kernel<uint8_t><<<grid, 256, 0, stream>>>(k);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_moves(const int32_t* idx, int R, int max_len, int in_place, MoveSource* sources,
+                               int32_t* dst_rows, int32_t* n_sources, int32_t* n_moves, int32_t* status,
+                               cudaStream_t stream) {
+    build_moves_kernel<<<1, 1024, 0, stream>>>(idx, R, max_len, in_place, sources, dst_rows, n_sources, n_moves, status);
+    return cudaGetLastError();
+}
+
+}  // namespace psmc

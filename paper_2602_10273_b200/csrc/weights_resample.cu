@@ -1,0 +1,168 @@
+// Weights, ESS and ESS-triggered systematic resampling for one token (Algorithm 1 rows 6-16,
+// Eq. 5, and the stage-boundary update of Section 4.3 / Appendix B).  One CTA per group, one
+// thread per particle (N <= 1024); reductions and prefix sums run on warp shuffles plus a
+// 33-entry shared array, in an order fixed by the thread index.
+//
+// Per particle i of group g (row r = g*N + i):
+//   log W_r += (alpha_t - alpha_{t-1}) * S_r                     stage boundary (all rows)
+//   live:  log W_r += log omega_r;  S_r += log p(y);  len_r += 1;  done_r |= (y == EOS)
+//   done:  y = EOS, factor 1
+// Per group:  w_i = exp(log W_i - max), C = inclusive prefix of w, ESS = (sum w)^2 / sum w^2.
+// If ESS < kappa*N:  u0 = hash uniform, A_i = min{j : C_j * N >= (u0 + i) * C_{N-1}} (N-1 if none),
+// offspring counts -> hazard-free slot map (survivors stay; dead slots, in increasing order, take
+// the surplus offspring, sources in increasing order), state gathered by the map, log W <- 0,
+// log Z-hat += max + log(sum w / N).  Move records for the KV reindex are appended to global lists.
+#include "common.cuh"
+#include "internal.h"
+
+namespace psmc {
+namespace {
+
+__global__ void weights_resample_kernel(const WeightsArgs a) {
+    __shared__ double sh_red[33];
+    __shared__ int sh_redi[33];
+    __shared__ double sh_C[kMaxParticles];
+    __shared__ double sh_S[kMaxParticles];
+    __shared__ int sh_off[kMaxParticles];
+    __shared__ int sh_Einc[kMaxParticles];
+    __shared__ int sh_len[kMaxParticles];
+    __shared__ int sh_tok[kMaxParticles];
+    __shared__ unsigned char sh_done[kMaxParticles];
+    __shared__ int sh_base[2];
+
+    const int g = blockIdx.x, i = threadIdx.x, N = a.N;
+    const bool on = i < N;
+    const int r = g * N + (on ? i : 0);
+
+    // ---- per-particle update ----
+    double lw = -INFINITY, S = 0.0;
+    int tk = a.eos, ln = 0;
+    unsigned char dn = 1;
+    if (on) {
+        dn = a.done[r];
+        S = a.S[r];
+        ln = a.len[r];
+        lw = a.logW[r] + a.delta * S;
+        if (dn) {
+            a.logp[r] = 0.0;
+            a.loginc[r] = 0.0;
+        } else {
+            tk = a.tok_draw[r];
+            if (tk < 0) tk = a.eos;  // the logit pass flagged the row; keep indices valid
+            lw += a.loginc[r];
+            S += a.logp[r];
+            ln += 1;
+            if (tk == a.eos) dn = 1;
+        }
+        a.tok[r] = tk;
+        a.hist_tok[r] = tk;
+    }
+
+    // ---- normalise, ESS (Eq. 5) ----
+    const double M = block_max(lw, sh_red);
+    const double w = on ? exp(lw - M) : 0.0;
+    double s1;
+    const double C = block_scan_incl(w, sh_red, &s1);
+    const double s2 = block_sum(w * w, sh_red);
+    const double ess = s1 * s1 / s2;
+    const bool fire = ess < a.kappa * (double)N;
+    if (i == 0) {
+        a.ess[g] = ess;
+        a.resampled[g] = fire ? 1 : 0;
+    }
+
+    if (!fire) {
+        if (on) {
+            a.logW[r] = lw;
+            a.S[r] = S;
+            a.done[r] = dn;
+            a.len[r] = ln;
+            a.anc[r] = i;
+            a.map[r] = i;
+            a.hist_map[r] = i;
+            a.last_tok[r] = tk;
+        }
+        return;
+    }
+
+    // ---- systematic resampling ----
+    if (on) {
+        sh_C[i] = C;
+        sh_S[i] = S;
+        sh_len[i] = ln;
+        sh_tok[i] = tk;
+        sh_done[i] = dn;
+        sh_off[i] = 0;
+    }
+    __syncthreads();
+    int anc = N - 1;
+    if (on) {
+        const double u0 = hash_uniform(hash5(a.seed, kStreamResample, (uint64_t)g, (uint64_t)a.t, 0));
+        const double pos = (u0 + (double)i) * s1;
+        int lo = 0, hi = N;  // first j in [0,N) with C_j * N >= pos; C is non-decreasing
+        while (lo < hi) {
+            int mid = (lo + hi) >> 1;
+            if (sh_C[mid] * (double)N >= pos) hi = mid; else lo = mid + 1;
+        }
+        anc = lo < N ? lo : N - 1;
+        atomicAdd(&sh_off[anc], 1);
+    }
+    __syncthreads();
+
+    // ---- slot map ----
+    const int off = on ? sh_off[i] : 1;
+    const int dead = (on && off == 0) ? 1 : 0;
+    const int surplus = (on && off > 1) ? off - 1 : 0;
+    int n_dead, n_src;
+    const int dead_incl = block_scan_incl(dead, sh_redi, &n_dead);
+    const int sur_incl = block_scan_incl(surplus, sh_redi, (int*)nullptr);
+    const int src_incl = block_scan_incl(surplus > 0 ? 1 : 0, sh_redi, &n_src);
+    if (on) sh_Einc[i] = sur_incl;
+    if (i == 0) {
+        sh_base[0] = atomicAdd(a.n_moves, n_dead);
+        sh_base[1] = atomicAdd(a.n_sources, n_src);
+    }
+    __syncthreads();
+    int mp = i;
+    if (dead) {
+        const int rank = dead_incl - 1;  // this dead slot takes surplus offspring number `rank`
+        int lo = 0, hi = N;              // first j with Einc[j] > rank
+        while (lo < hi) {
+            int mid = (lo + hi) >> 1;
+            if (sh_Einc[mid] > rank) hi = mid; else lo = mid + 1;
+        }
+        mp = lo < N ? lo : N - 1;
+        a.dst_rows[sh_base[0] + rank] = r;
+    }
+    if (surplus > 0) {
+        MoveSource ms;
+        ms.src_row = r;
+        ms.len = ln;
+        ms.dst_begin = sh_base[0] + (sur_incl - surplus);
+        ms.n_dst = surplus;
+        a.sources[sh_base[1] + src_incl - 1] = ms;
+    }
+
+    // ---- copy particle state by the map, uniform weights ----
+    if (on) {
+        a.logW[r] = 0.0;
+        a.S[r] = sh_S[mp];
+        a.done[r] = sh_done[mp];
+        a.len[r] = sh_len[mp];
+        a.anc[r] = anc;
+        a.map[r] = mp;
+        a.hist_map[r] = mp;
+        a.last_tok[r] = sh_tok[mp];
+    }
+    if (i == 0) a.logZ[g] += M + log(s1 / (double)N);
+}
+
+}  // namespace
+
+cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream) {
+    int threads = ((a.N + 31) / 32) * 32;
+    weights_resample_kernel<<<a.G, threads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace psmc

@@ -1,0 +1,388 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle.  Needs a B200."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2602_10273_b200 import binding as B
+from paper_2602_10273_b200.workload import cuda as WC
+from paper_2602_10273_b200.workload import gen as W
+
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _to_double(t):
+    if t.dtype == torch.bfloat16:
+        return W.bf16_bits_to_f32(_bf16_bits(t)).astype(np.float64)
+    return t.cpu().numpy().astype(np.float64)
+
+
+def run_logits_pass(logits, beta, alpha_t, u, done=None):
+    R, V = logits.shape
+    dev = logits.device
+    scratch = torch.zeros(B.logits_pass_scratch_bytes(R, V) + 256, dtype=torch.uint8, device=dev)
+    off = (-scratch.data_ptr()) % 256
+    scratch = scratch[off:off + B.logits_pass_scratch_bytes(R, V)]
+    tok = torch.full((R,), -7, dtype=torch.int32, device=dev)
+    logp = torch.zeros(R, dtype=torch.float64, device=dev)
+    loginc = torch.zeros(R, dtype=torch.float64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ud = torch.from_numpy(np.asarray(u, dtype=np.float64)).to(dev)
+    dd = None if done is None else torch.from_numpy(np.asarray(done, dtype=np.uint8)).to(dev)
+    for _ in range(2):  # twice: the pass must leave its scratch ready for the next call
+        B.logits_pass(logits, beta, alpha_t, ud, dd, scratch, tok, logp, loginc, status)
+    torch.cuda.synchronize()
+    assert int(scratch[: 4 * R].view(torch.int32).abs().sum()) == 0
+    return tok.cpu().numpy(), logp.cpu().numpy(), loginc.cpu().numpy(), int(status.item())
+
+
+def check_rows_against_oracle(logits, beta, alpha_t, u, tok, logp, loginc, rows=None):
+    lg = _to_double(logits)
+    flagged = 0
+    for r in (range(lg.shape[0]) if rows is None else rows):
+        o = O.row(lg[r], beta, alpha_t, float(u[r]))
+        if o["y"] != tok[r]:
+            assert o["margin"] <= P.TOK_MARGIN, "row %d: %d vs %d margin %.3e" % (r, tok[r], o["y"], o["margin"])
+            flagged += 1
+            o = O.row(lg[r], beta, alpha_t, float(u[r]), force=int(tok[r]))
+        assert abs(o["log_omega"] - loginc[r]) <= P.TOL_LOGINC, (r, o["log_omega"], loginc[r])
+        assert abs(o["logp_y"] - logp[r]) <= P.TOL_LOGINC
+    return flagged
+
+
+# ------------------------------------------------------------------ the logit pass alone
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("beta", [1.0, 2.0, 4.0, 8.0, 2.71875])
+@pytest.mark.parametrize("V", [1000, 1024, 5003, 40000])
+def test_logits_pass_matches_oracle(dtype, beta, V):
+    torch.manual_seed(V + int(beta * 8))
+    R = 9
+    logits = (torch.randn(R, V, device="cuda") * 3.0).to(dtype)
+    logits[3, : V // 2] = -math.inf                       # zero-mass stretch
+    logits[4] = 1.5                                       # flat row
+    logits[5] = -math.inf
+    logits[5, V - 3] = 0.25                               # one-hot row
+    u = np.array([O.uniform(O.hash5(9, 1, 0, V, r)) for r in range(R)])
+    u[6], u[7] = 2.0**-53, 1.0 - 2.0**-53                  # the two ends of (0,1)
+    tok, logp, loginc, status = run_logits_pass(logits, beta, beta, u)
+    assert status == B.OK
+    check_rows_against_oracle(logits, beta, beta, u, tok, logp, loginc)
+    assert tok[5] == V - 3 and abs(loginc[5]) < 1e-12
+    assert abs(loginc[4] - (1.0 - beta) * math.log(V)) < 1e-5
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_logits_pass_unaligned_rows_and_non_optimal_proposal(dtype):
+    torch.manual_seed(3)
+    R, V = 5, 3001
+    u = np.array([O.uniform(O.hash5(3, 1, 0, 1, r)) for r in range(R)])
+    # ld 3007: rows are not 16-byte aligned (scalar loads); ld 3008: aligned rows with a ragged tail of one logit
+    for ld in (3007, 3008):
+        base = (torch.randn(R, ld, device="cuda") * 2.0).to(dtype)
+        logits = base[:, :V]
+        for beta, alpha_t in ((4.0, 4.0), (1.5, 4.0), (3.0, 2.0)):
+            tok, logp, loginc, status = run_logits_pass(logits, beta, alpha_t, u)
+            assert status == B.OK
+            check_rows_against_oracle(logits, beta, alpha_t, u, tok, logp, loginc)
+
+
+def test_logits_pass_skips_done_rows_and_flags_bad_rows():
+    R, V = 6, 4096
+    logits = torch.randn(R, V, device="cuda").to(torch.bfloat16)
+    u = np.full(R, 0.37)
+    done = np.array([0, 1, 0, 0, 1, 0], dtype=np.uint8)
+    tok, logp, loginc, status = run_logits_pass(logits, 4.0, 4.0, u, done)
+    assert status == B.OK and tok[1] == -7 and tok[4] == -7 and (tok[[0, 2, 3, 5]] >= 0).all()
+    for bad in (float("nan"), float("inf")):
+        l2 = logits.clone()
+        l2[2, 100] = bad
+        tok, _, _, status = run_logits_pass(l2, 4.0, 4.0, u)
+        assert status == B.E_NUMERIC and tok[2] == -1 and tok[0] >= 0
+    l2 = logits.clone()
+    l2[3] = -math.inf
+    tok, _, _, status = run_logits_pass(l2, 4.0, 4.0, u)
+    assert status == B.E_NUMERIC and tok[3] == -1
+
+
+def test_logits_pass_token_independence_on_device():
+    """Theorem 1 on the CUDA path: at beta = alpha the increment does not depend on the uniform."""
+    V = 20000
+    logits = (torch.randn(1, V, device="cuda") * 3).to(torch.bfloat16).repeat(16, 1).contiguous()
+    u = (np.arange(16) + 0.5) / 16
+    tok, logp, loginc, status = run_logits_pass(logits, 4.0, 4.0, u)
+    assert status == B.OK and len(set(tok.tolist())) > 3
+    assert np.ptp(loginc) == 0.0
+    assert np.all(np.diff(tok) >= 0)                      # the inverse CDF is monotone in U
+
+
+# ------------------------------------------------------------------ weights / ESS / resampling on identical state
+@pytest.mark.parametrize("N", [1, 2, 4, 8, 32, 33, 100, 1024])
+def test_resampling_kernel_bit_exact_on_identical_log_weights(N):
+    rng = np.random.default_rng(N)
+    V, G = 64, 3
+    for trial in range(4):
+        ps = B.Psmc(N, V, 2.0, 0.5, 1.0, 0, 11 + trial, V - 1, G=G, T_max=4, prompt_len=[5, 6, 7])
+        orc = O.Oracle(N, V, 2.0, 0.5, 1.0, 0, 11 + trial, V - 1, G=G, T_max=4, prompt_len=[5, 6, 7])
+        lw = rng.normal(0, 2.0 + trial, size=G * N)
+        lw[N:2 * N] = -1.25                                # group 1: uniform weights, must not resample
+        S = rng.normal(-3, 1, size=G * N)
+        lens = np.repeat([5, 6, 7], N).astype(np.int32) + rng.integers(0, 3, size=G * N).astype(np.int32)
+        ps.set_state(log_w=lw, cum_logp=S, lens=lens)
+        orc.set_state(logW=lw, S=S, lens=lens)
+        logits = torch.zeros(G * N, V, device="cuda")      # flat logits: log omega = (1-2) ln 64 for every row
+        ps.step(logits)
+        orc.step(logits.cpu().numpy(), force_tok=ps.tokens.numpy())
+        assert ps.sync_status() == B.OK
+        assert np.array_equal(ps.resampled.numpy(), orc.resampled) and orc.resampled[1] == 0
+        assert np.array_equal(ps.ancestors.numpy(), orc.ancestors)
+        assert np.array_equal(ps.slot_map.numpy(), orc.slot_map)
+        assert np.array_equal(ps.lens.numpy(), orc.lens)
+        assert np.allclose(ps.ess.numpy(), orc.ess, rtol=1e-12)
+        assert np.allclose(ps.log_weights.numpy(), orc.log_weights, atol=1e-9)
+        assert np.allclose(ps.cum_logp.numpy(), orc.cum_logp, atol=1e-9)
+        assert np.allclose(ps.log_z.numpy(), orc.log_z, atol=1e-9)
+        ps.destroy()
+
+
+# ------------------------------------------------------------------ closed loops on the named configurations
+def test_closed_loop_tiny_full():
+    c = W.CONFIGS["tiny"]
+    st = P.closed_loop(c, seed=1, T=c.T, kv_shape=(c.n_layers, c.n_kv_heads, c.max_len, c.head_dim))
+    assert st.steps == 64 and st.resample_events > 0 and st.slots_moved > 0
+    print("tiny:", st)
+
+
+@pytest.mark.parametrize("seed", [2, 3])
+def test_closed_loop_tiny_other_seeds(seed):
+    c = W.CONFIGS["tiny"]
+    P.closed_loop(c, seed=seed, T=c.T, kv_shape=(c.n_layers, c.n_kv_heads, c.max_len, c.head_dim))
+
+
+def test_closed_loop_llama_shape():
+    c = W.CONFIGS["llama2_7b"]
+    st = P.closed_loop(c, seed=1, T=96, kv_shape=(2, 4, 512 + 96 + 8, c.head_dim))
+    assert st.resample_events > 0
+    print("llama2_7b:", st)
+
+
+def test_closed_loop_qwen_shape_with_ramp():
+    c = W.CONFIGS["qwen25_7b"]
+    st = P.closed_loop(c, seed=1, T=48, kv_shape=(2, c.n_kv_heads, 256 + 48 + 8, c.head_dim))
+    print("qwen25_7b (ramp steps):", st)
+    st = P.closed_loop(c, seed=2, T=40, ramp=16)          # leaves the ramp after 16 tokens: beta = 4 exactly
+    assert st.resample_events > 0
+    print("qwen25_7b (ramp 16):", st)
+
+
+def test_closed_loop_resampling_stress():
+    c = W.CONFIGS["resample_stress"]
+    st = P.closed_loop(c, seed=1, T=40, ramp=8, kv_shape=(1, c.n_kv_heads, 128 + 40 + 8, c.head_dim))
+    assert st.resample_events >= 10
+    print("resample_stress (ramp 8):", st)
+    st = P.closed_loop(c, seed=2, T=24)                   # inside the 256-token ramp: fractional exponents
+    print("resample_stress (in ramp):", st)
+
+
+def test_closed_loop_batched_prompts():
+    c = W.CONFIGS["batched_prompts"]
+    st = P.closed_loop(c, seed=1, T=24, G=8, kv_shape=(1, 2, 256 + 24 + 8, c.head_dim))
+    assert st.resample_events > 0
+    print("batched_prompts (8 prompts):", st)
+
+
+def test_eos_rows_freeze_and_are_not_read():
+    c = W.CONFIGS["tiny"]
+
+    def push_eos(t, lg):
+        if t == 5:
+            lg[1, c.eos_id] = 60.0                         # slot 1 is driven onto EOS at token 5
+
+    st = P.closed_loop(c, seed=5, T=20, kappa=0.05, logit_bias_fn=push_eos)
+    assert st.steps == 20
+
+
+def test_done_rows_logits_are_never_read():
+    V, N = 2048, 4
+    ps = B.Psmc(N, V, 4.0, 0.25, 0.01, 0, 3, V - 1, T_max=4)
+    ps.set_state(done=np.array([0, 1, 0, 1], dtype=np.uint8))
+    lg = torch.randn(N, V, device="cuda")
+    lg[1] = float("nan")
+    lg[3] = float("inf")
+    ps.step(lg)
+    assert ps.sync_status() == B.OK
+    assert ps.tokens.numpy()[[1, 3]].tolist() == [V - 1, V - 1] and ps.log_inc.numpy()[[1, 3]].tolist() == [0.0, 0.0]
+    ps.destroy()
+
+
+# ------------------------------------------------------------------ KV reindex
+@pytest.mark.parametrize("dtype,D", [(torch.bfloat16, 128), (torch.float32, 64), (torch.bfloat16, 20), (torch.float32, 3)])
+def test_reindex_out_of_place_is_index_select(dtype, D):
+    R, H, ML, L = 6, 3, 37, 2
+    ps = B.Psmc(R, 16, 2.0, 0.5, 0.5, 0, 1, 15, T_max=2)
+    ks = [torch.randn(R, H, ML, D, device="cuda").to(dtype) for _ in range(L)]
+    vs = [torch.randn(R, H, ML, D, device="cuda").to(dtype) for _ in range(L)]
+    kd = [torch.zeros_like(t) for t in ks]
+    vd = [torch.zeros_like(t) for t in vs]
+    idx = torch.tensor([4, 4, 0, 5, 1, 1], dtype=torch.int32, device="cuda")
+    ps.reindex_kv(ps.make_kv_desc(ks, vs), ps.make_kv_desc(kd, vd), idx)
+    assert ps.sync_status() == B.OK
+    for s, d in zip(ks + vs, kd + vd):
+        assert torch.equal(d, s[idx.long()])
+    ps.destroy()
+
+
+def test_reindex_in_place_override_and_hazard_detection():
+    R, H, ML, D = 6, 2, 16, 64
+    ps = B.Psmc(R, 16, 2.0, 0.5, 0.5, 0, 1, 15, T_max=2)
+    ks = [torch.randn(R, H, ML, D, device="cuda").to(torch.bfloat16)]
+    vs = [torch.randn(R, H, ML, D, device="cuda").to(torch.bfloat16)]
+    want_k, want_v = ks[0].clone(), vs[0].clone()
+    desc = ps.make_kv_desc(ks, vs)
+    good = torch.tensor([1, 1, 1, 3, 3, 5], dtype=torch.int32, device="cuda")
+    ps.reindex_kv(desc, None, good)
+    assert ps.sync_status() == B.OK
+    assert torch.equal(ks[0], want_k[good.long()]) and torch.equal(vs[0], want_v[good.long()])
+    before = ks[0].clone()
+    bad = torch.tensor([1, 2, 3, 3, 4, 5], dtype=torch.int32, device="cuda")   # row 1 is read and rewritten
+    ps.reindex_kv(desc, None, bad)
+    assert ps.sync_status() == B.E_HAZARD
+    assert torch.equal(ks[0], before)                       # nothing was written
+    ps.destroy()
+
+
+def test_reindex_strided_cache_and_misaligned_base():
+    """Caches that are views into larger buffers: row/head strides larger than the tight ones, odd offsets."""
+    R, H, ML, D = 4, 2, 9, 8
+    ps = B.Psmc(R, 16, 2.0, 0.5, 0.5, 0, 1, 15, T_max=2)
+    for off in (0, 1, 3):                                   # element offsets: 2-byte and 6-byte misalignment
+        big = torch.randn(R * (H + 1) * (ML + 2) * D + 8, device="cuda").to(torch.bfloat16)
+        view = big[off: off + R * (H + 1) * (ML + 2) * D].view(R, H + 1, ML + 2, D)[:, :H, :ML, :]
+        k, v = view, view.clone().contiguous()
+        ref_k, ref_v, ref_big = k.clone(), v.clone(), big.clone()
+        idx = torch.tensor([2, 1, 2, 2], dtype=torch.int32, device="cuda")
+        # once the strided view, once a tight tensor of the same shape (each as both K and V of one layer)
+        import ctypes as C
+        for t, ref in ((k, ref_k), (v, ref_v)):
+            arr = (C.c_void_p * 1)(t.data_ptr())
+            d = B.KvDesc(1, C.cast(arr, C.POINTER(C.c_void_p)), C.cast(arr, C.POINTER(C.c_void_p)), H, D, ML, B.BF16,
+                         t.stride(0), t.stride(1))
+            ps.reindex_kv(d, None, idx)
+            assert ps.sync_status() == B.OK
+            assert torch.equal(t, ref[idx.long()])
+        # the padding between heads/positions of the big buffer is untouched
+        mask = torch.ones_like(big, dtype=torch.bool)
+        mview = mask[off: off + R * (H + 1) * (ML + 2) * D].view(R, H + 1, ML + 2, D)
+        mview[:, :H, :ML, :] = False
+        assert torch.equal(big[mask], ref_big[mask])
+    ps.destroy()
+
+
+# ------------------------------------------------------------------ generators: CUDA twin vs numpy
+def test_cuda_generators_match_numpy():
+    seed, V, N = 4, 6000, 4
+    bias = W.vocab_bias(seed, V, 1.5)
+    prev = np.array([5, 5, 77, 4000, 1, 2, 3, 4], dtype=np.int32)
+    for dtype, tdt in (("f32", torch.float32), ("bf16", torch.bfloat16)):
+        dst = torch.empty(8, V, dtype=tdt, device="cuda")
+        WC.fill_logits(dst, seed, 3, N, torch.from_numpy(prev).cuda(), 3.0, torch.from_numpy(bias).cuda())
+        ref = W.logits_block(seed, 3, np.arange(8) // N, prev, V, 3.0, bias, dtype)
+        got = P.logits_to_numpy(dst)
+        flips = int((got != ref).sum())
+        assert flips <= 3, "%d of %d elements differ" % (flips, got.size)   # last-ulp libm differences only
+        if dtype == "f32":
+            assert np.abs(got - ref).max() <= 4e-6
+        kv = torch.empty(3, 2, 16, 32, dtype=tdt, device="cuda")
+        WC.fill_kv(kv, seed, 1, 1, row0=2)
+        ref = W.kv_block(seed, 1, 1, [2, 3, 4], 2, 16, 32, dtype)
+        got = (kv.view(torch.int16) if tdt == torch.bfloat16 else kv).cpu().numpy()
+        got = got.view(np.uint16) if dtype == "bf16" else got
+        assert int((got != ref).sum()) <= 2
+
+
+# ------------------------------------------------------------------ brute force through the C-ABI
+@pytest.mark.parametrize("N,runs", [(4, 3000), (32, 1500)])
+def test_power_distribution_and_normaliser_through_the_cabi(N, runs):
+    from test_oracle_pins import TinyLM
+    V, T, alpha = 3, 4, 3.0
+    lm = TinyLM(V, 31, spread=1.0)
+    strings, gam = lm.enumerate(T, alpha, V - 1)
+    pi, Z = gam / gam.sum(), gam.sum()
+    index = {s: k for k, s in enumerate(strings)}
+    G = 500                                                # 500 independent runs per context, batched as groups
+    table = torch.from_numpy(lm.table.astype(np.float32)).cuda()
+    counts = np.zeros(len(strings))
+    zs = []
+    for rep in range(runs // G):
+        ps = B.Psmc(N, V, alpha, 1.0 / alpha, 0.5, 0, 7000 + rep, V - 1, G=G, T_max=T)
+        last = ps.device_view("psmc_last_tokens", ps.R)
+        for t in range(T):
+            prev = torch.where(last < 0, torch.full_like(last, V), last).long()
+            ps.step(table[prev].contiguous())
+        toks, ln, ix = ps.select()
+        lw = ps.log_weights.numpy().reshape(G, N)
+        M = lw.max(axis=1)
+        zs.append(np.exp(ps.log_z.numpy() + M + np.log(np.exp(lw - M[:, None]).sum(axis=1) / N)))
+        for row in toks.cpu().numpy()[:, :T]:
+            counts[index[tuple(int(x) for x in row)]] += 1
+        assert ps.sync_status() == B.OK
+        ps.destroy()
+    n = counts.sum()
+    zs = np.concatenate(zs)
+    assert abs(zs.mean() - Z) < 4.0 * zs.std(ddof=1) / math.sqrt(zs.size)
+    tv = 0.5 * np.abs(counts / n - pi).sum()
+    noise = 0.5 * np.sum(np.sqrt(pi * (1 - pi) / n)) * math.sqrt(2 / math.pi)
+    if N >= 32:
+        assert tv < 3.0 * noise + 2.0 / N, (tv, noise)
+    else:
+        assert tv < 0.5
+
+
+# ------------------------------------------------------------------ host-visible errors
+def test_argument_errors_return_codes():
+    import ctypes as C
+    L = B.lib()
+    h = C.c_void_p()
+    assert L.psmc_init(C.byref(h), 0, 100, 4.0, 0.25, 0.5, 0, 1, 99) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 4, 1, 4.0, 0.25, 0.5, 0, 1, 0) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 4, 100, 0.5, 0.25, 0.5, 0, 1, 99) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 4, 100, 4.0, 0.0, 0.5, 0, 1, 99) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 4, 100, 4.0, 0.25, 1.5, 0, 1, 99) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 4, 100, 4.0, 0.25, 0.5, 0, 1, 100) == B.E_INVAL
+    assert L.psmc_init(C.byref(h), 2000, 100, 4.0, 0.25, 0.5, 0, 1, 99) == B.E_INVAL
+    assert L.psmc_step(None, None, 0, 0, None) == B.E_INVAL
+    ps = B.Psmc(4, 100, 4.0, 0.25, 0.5, 0, 1, 99, T_max=1)
+    lg = torch.zeros(4, 100, device="cuda")
+    assert L.psmc_step(ps._h, lg.data_ptr(), 7, 100, None) == B.E_INVAL
+    assert L.psmc_step(ps._h, lg.data_ptr(), 0, 99, None) == B.E_INVAL
+    ps.step(lg)
+    with pytest.raises(B.PsmcError) as e:
+        ps.step(lg)
+    assert e.value.code == B.E_STATE
+    ps.destroy()
+
+
+def test_step_host_matches_device_step():
+    c = W.CONFIGS["tiny"]
+    wl, ps, orc = P.make_pair(c, 9, T_max=6)
+    ps2 = B.Psmc(c.N, c.V, c.alpha, c.tau, c.kappa, c.ramp, 9, c.eos_id, T_max=6, prompt_len=wl.prompt_len)
+    lg = wl.new_logits()
+    prev = wl.first_prev.clone()
+    out = torch.empty(ps.R, dtype=torch.int32).pin_memory()
+    for t in range(1, 7):
+        wl.fill(lg, t, prev)
+        ps.step(lg)
+        host = lg.cpu().pin_memory()
+        ps2.step_host(host, out)
+        assert torch.equal(out, ps.last_tokens)
+        assert torch.equal(ps2.log_weights, ps.log_weights)
+        prev.copy_(ps.device_view("psmc_last_tokens", ps.R))
+    ps.destroy()
+    ps2.destroy()
