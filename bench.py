@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the Power-SMC hot path on B200: one "step" = one decoded token for every particle =
+logit pass + weights/ESS/resampling + KV-cache reindex, on synthetic inputs shaped like the paper's.
+
+  python bench.py --gpus 1 --steps 256 --warmup 8            # this repository's CUDA path
+  python bench.py --impl reference --steps 3 --warmup 1      # the CPU oracle as the reference arm
+
+Prints ONE JSON line.  `value` is particle-tokens/s with every input resident in HBM; `e2e` is the
+same metric through psmc_step_host (pinned host logits copied in, tokens copied out, every step).
+Multi-GPU (torchrun): every rank runs its own set of prompts (no data-path collective; weak scaling);
+time is the max over ranks of the device time of the K timed steps.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2602_10273_b200.workload import gen  # noqa: E402
+
+METRIC = "particle_tokens_per_s"
+UNIT = "particle-tokens/s"
+N_BLOCKS = 6           # distinct logit blocks rotated through (6 x 131 MB at the default workload: beyond L2)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons of one GPU through NVML while a region runs (read-only)."""
+
+    def __init__(self, local_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz, self._stop = [], set(), None, threading.Event()
+        self.period = period_s
+        self.thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            entry = vis.split(",")[local_index].strip() if vis else str(local_index)
+            if entry.isdigit():
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(int(entry))
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(entry.encode() if hasattr(entry, "encode") else entry)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                    nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                mask = get(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def logits_to_numpy(t: torch.Tensor) -> np.ndarray:
+    """Device logits -> host array the oracle reads (fp32 as is, bf16 as uint16 bit patterns)."""
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+def moved_bytes(slot_map, lens, G, N, bytes_per_pos):
+    """Algorithmic bytes of one KV reindex: each source with surplus offspring is read once, each rewritten slot
+    written once; lens are the post-step live lengths (a rewritten slot carries its source's length)."""
+    m = slot_map.reshape(G, N)
+    ln = lens.reshape(G, N)
+    moved = m != np.arange(N)[None, :]
+    wr = int(ln[moved].sum())
+    rd = 0
+    for g in np.nonzero(moved.any(axis=1))[0]:
+        srcs = np.unique(m[g][moved[g]])
+        rd += int(ln[g][srcs].sum())
+    return (rd + wr) * bytes_per_pos, int(moved.sum())
+
+
+def run_ours(args):
+    from paper_2602_10273_b200 import binding as B
+    from paper_2602_10273_b200.workload import cuda as WC
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    hbm_peak, peak_kind = load_peaks()
+
+    cfg = gen.CONFIGS[args.workload]
+    K, Wm = args.steps, args.warmup
+    T_total = K + Wm
+    if cfg.prompt_hi + T_total > cfg.max_len:
+        raise SystemExit("steps + warmup exceed the cache length of the workload")
+    # shrink the number of prompts only if the cache does not fit this GPU (never the shapes)
+    G = cfg.G if args.groups is None else args.groups
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    per_group = cfg.N * cfg.max_len * cfg.kv_bytes_per_pos_per_row
+    fixed = N_BLOCKS * cfg.N * cfg.logit_bytes_per_row  # per group
+    while G > 1 and G * (per_group + fixed) + (6 << 30) > free_b:
+        G -= 1
+    seed = 1 + rank
+    wl = WC.DeviceWorkload(cfg, seed, G=G, device=dev)
+    R, N = wl.R, cfg.N
+    ks, vs = wl.new_kv()
+    ps = B.Psmc(N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=G, T_max=T_total,
+                prompt_len=wl.prompt_len)
+    desc = ps.make_kv_desc(ks, vs)
+    last = ps.device_view("psmc_last_tokens", R)
+
+    # logit blocks: generated along a short closed loop, then reused cyclically by every pass below
+    blocks = [wl.new_logits() for _ in range(N_BLOCKS)]
+    prev = wl.first_prev.clone()
+    for t in range(1, N_BLOCKS + 1):
+        wl.fill(blocks[t - 1], t, prev)
+        ps.step(blocks[t - 1])
+        prev.copy_(last)
+    assert ps.sync_status() == B.OK
+    ps.reset(seed)
+
+    def one_pass(n_steps, first_t=1):
+        for t in range(first_t, first_t + n_steps):
+            ps.step(blocks[(t - 1) % N_BLOCKS])
+            ps.reindex_kv(desc)
+
+    # recording pass: per-step algorithmic KV bytes and live rows (deterministic, so the timed passes repeat it)
+    kv_bytes, moved_slots, live_rows = [], [], []
+    for t in range(1, T_total + 1):
+        live_rows.append(R - int(ps.done.numpy().sum()))  # rows that are live when step t starts
+        one_pass(1, t)
+        b, mv = moved_bytes(ps.slot_map.numpy(), ps.lens.numpy(), G, N, cfg.kv_bytes_per_pos_per_row)
+        kv_bytes.append(b)
+        moved_slots.append(mv)
+    assert ps.sync_status() == B.OK
+    live_timed = int(np.sum(live_rows[Wm:]))
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device=dev)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
+    def sum_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device=dev)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.SUM)
+            return float(t.item())
+        return float(x)
+
+    # ---- pass A: the headline. K steps, device-resident inputs, one pair of events around all of them ----
+    ps.reset(seed)
+    one_pass(Wm, 1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local) as clk:
+        e0.record()
+        one_pass(K, Wm + 1)
+        e1.record()
+        torch.cuda.synchronize(dev)
+    barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    assert ps.sync_status() == B.OK
+    value = sum_over_ranks(live_timed) / (ms_total * 1e-3)
+
+    # ---- pass B: same K steps with every kernel bracketed by events, for the roofline of each kernel ----
+    ps.reset(seed)
+    one_pass(Wm, 1)
+    torch.cuda.synchronize(dev)
+    ps.timing_enable(True)
+    one_pass(K, Wm + 1)
+    kms, kn = ps.timing_read()
+    ps.timing_enable(False)
+    k1_bytes = float(np.sum(live_rows[Wm:])) * cfg.logit_bytes_per_row
+    k3_bytes = float(np.sum(kv_bytes[Wm:]))
+    k1_gbs = k1_bytes / (kms[0] * 1e-3) / 1e9 if kms[0] > 0 else 0.0
+    k3_gbs = k3_bytes / (kms[2] * 1e-3) / 1e9 if kms[2] > 0 and k3_bytes > 0 else 0.0
+    shares = [m / max(sum(kms), 1e-12) for m in kms]
+    dominant = int(np.argmax(kms))
+    names = ["logits_pass_kernel", "weights_resample_kernel", "reindex_bulk_kernel"]
+    roofs = {
+        "logits_pass_kernel": {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
+                               "frac": k1_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                               "avg_launch_us": 1e3 * kms[0] / max(kn[0], 1), "time_share": shares[0],
+                               "bytes_per_launch": k1_bytes / max(kn[0], 1)},
+        "reindex_bulk_kernel": {"bound": "hbm", "achieved": k3_gbs, "peak": hbm_peak, "unit": "GB/s",
+                                "frac": k3_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                                "avg_launch_us": 1e3 * kms[2] / max(kn[2], 1), "time_share": shares[2],
+                                "bytes_per_launch": k3_bytes / max(kn[2], 1)},
+        "weights_resample_kernel": {"bound": "latency", "avg_launch_us": 1e3 * kms[1] / max(kn[1], 1),
+                                    "time_share": shares[1]},
+    }
+    roofline = dict(roofs[names[dominant]] if dominant != 1 else roofs["reindex_bulk_kernel"])
+    roofline["kernel"] = names[dominant] if dominant != 1 else "reindex_bulk_kernel"
+
+    # ---- e2e: host logits in, tokens out, every step, through psmc_step_host ----
+    Ke = min(K, args.e2e_steps)
+    host_blocks = [b.cpu().pin_memory() for b in blocks]
+    tok_host = torch.empty(R, dtype=torch.int32).pin_memory()
+    ps.reset(seed)
+    for t in range(1, Wm + 1):
+        ps.step_host(host_blocks[(t - 1) % N_BLOCKS], tok_host)
+        ps.reindex_kv(desc)
+    barrier()
+    e0.record()
+    for t in range(Wm + 1, Wm + Ke + 1):
+        ps.step_host(host_blocks[(t - 1) % N_BLOCKS], tok_host)
+        ps.reindex_kv(desc)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+    e2e_value = sum_over_ranks(float(np.sum(live_rows[Wm:Wm + Ke]))) / (ms_e2e * 1e-3)
+    assert ps.sync_status() == B.OK
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": "%s: %d prompts x %d particles, V=%d, KV %dx%dx%d max_len %d (%s)" % (
+                       cfg.name, G, N, cfg.V, cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, cfg.max_len, cfg.dtype),
+                   "prompts_per_gpu": G, "rows_per_gpu": R, "alpha": cfg.alpha, "tau": cfg.tau, "kappa": cfg.kappa,
+                   "ramp": cfg.ramp, "l2": "inputs larger than L2: %d logit blocks of %.0f MB rotated, KV %.1f GB" % (
+                       N_BLOCKS, R * cfg.logit_bytes_per_row / 1e6, G * per_group / 1e9),
+                   "parallelism": "replicas only (prompts sharded, no collective)"},
+        "clocks": clk.summary(),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": R * cfg.logit_bytes_per_row,
+                "d2h_bytes_per_step": R * 4, "steps": Ke, "ms_per_step": ms_e2e / Ke},
+        "gpu_launches": int(K * (2 + (cfg.n_layers + 63) // 64)),
+        "roofline": roofline,
+        "kernels": roofs,
+        "kv_reindex": {"gb_per_s": k3_gbs, "frac_of_hbm_peak": k3_gbs / hbm_peak,
+                       "slots_moved_per_step": float(np.mean(moved_slots[Wm:])),
+                       "gb_moved_per_step": k3_bytes / K / 1e9},
+        "step_without_kv": {"particle_tokens_per_s": float(np.sum(live_rows[Wm:])) / ((kms[0] + kms[1]) * 1e-3),
+                            "us_per_step": 1e3 * (kms[0] + kms[1]) / K},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(cfg, wl, blocks, G, float(np.mean(kv_bytes[Wm:])))
+    ps.destroy()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def oracle_step_rate(cfg, seed, G, logits_host_blocks, prompt_len, n_steps):
+    """Times the CPU oracle (as it stands) on n_steps of the given blocks; returns (rows/s, seconds, rows)."""
+    from oracle import oracle as O
+    o = O.Oracle(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=G, T_max=n_steps,
+                 prompt_len=prompt_len)
+    rows = 0
+    t0 = time.perf_counter()
+    for t in range(n_steps):
+        rows += G * cfg.N - int(o.done.sum())
+        o.step(logits_host_blocks[t % len(logits_host_blocks)])
+    return rows / (time.perf_counter() - t0), time.perf_counter() - t0, rows
+
+
+def oracle_copy_rate(cfg):
+    """GB/s (read + write) of the oracle's KV reindex loop on a 4-row slice of one layer tensor."""
+    from oracle import oracle as O
+    rng = np.random.default_rng(0)
+    t = rng.integers(0, 2**16, size=(4, cfg.n_kv_heads, cfg.max_len, cfg.head_dim), dtype=np.uint16)
+    if cfg.dtype == "f32":
+        t = t.astype(np.float32)
+    idx = np.array([1, 1, 3, 3], dtype=np.int32)
+    O.reindex_tensor(t, t, idx, None)  # touch
+    reps = 20
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        O.reindex_tensor(t, t, idx, None)
+    dt = time.perf_counter() - t0
+    return reps * 2 * 2 * t[0].nbytes / dt / 1e9
+
+
+def cpu_baseline(cfg, wl, blocks, G, kv_bytes_per_step):
+    cores = len(os.sched_getaffinity(0))
+    Gs = min(G, 8)                      # bounded sample: the first 8 prompts
+    host = [logits_to_numpy(b[: Gs * cfg.N]) for b in blocks[:3]]
+    rate, secs, rows = oracle_step_rate(cfg, wl.seed, Gs, host, wl.prompt_len[:Gs], 3)
+    copy_gbs = oracle_copy_rate(cfg)
+    # one full step on the CPU = the oracle's step for all rows + its memcpy loop over the step's KV bytes
+    t_step = (G * cfg.N) / rate + kv_bytes_per_step / (copy_gbs * 1e9)
+    return {"value": (G * cfg.N) / t_step, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "oracle step on the first %d prompts (%d rows) for 3 tokens: %.0f rows/s in %.1f s; oracle KV "
+                      "reindex loop on a 4-row slice of one layer: %.1f GB/s; combined for one full step of %d rows "
+                      "and %.2f GB of KV moves" % (Gs, Gs * cfg.N, rate, secs, copy_gbs, G * cfg.N,
+                                                  kv_bytes_per_step / 1e9),
+            "oracle_rows_per_s": rate, "oracle_copy_gb_per_s": copy_gbs}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = gen.CONFIGS[args.workload]
+    seed = 1
+    G = cfg.G if args.groups is None else args.groups
+    Gs = min(G, 2)                      # each step is a bounded sample: the first 2 prompts
+    bias = gen.vocab_bias(seed, cfg.V, cfg.slope)
+    plen = gen.prompt_lengths(seed, G, cfg.prompt_lo, cfg.prompt_hi)
+    prev = np.repeat(gen.prompt_last_token(seed, G, plen, cfg.V), cfg.N)[: Gs * cfg.N]
+    groups = np.repeat(np.arange(Gs), cfg.N)
+    host = [gen.logits_block(seed, t, groups, prev, cfg.V, cfg.scale, bias, cfg.dtype) for t in (1, 2)]
+    K, Wm = args.steps, args.warmup
+    from oracle import oracle as O
+    o = O.Oracle(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=Gs, T_max=K + Wm,
+                 prompt_len=plen[:Gs])
+    copy_gbs = oracle_copy_rate(cfg)
+    for t in range(Wm):
+        o.step(host[t % 2])
+    rows, kv_b = 0, 0.0
+    t0 = time.perf_counter()
+    for t in range(K):
+        rows += Gs * cfg.N - int(o.done.sum())
+        o.step(host[(Wm + t) % 2])
+        b, _ = moved_bytes(o.slot_map, o.lens, Gs, cfg.N, cfg.kv_bytes_per_pos_per_row)
+        kv_b += b
+    secs = time.perf_counter() - t0 + kv_b / (copy_gbs * 1e9)
+    value = rows / secs
+    cores = len(os.sched_getaffinity(0))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": K, "warmup": Wm, "ms_per_step": 1e3 * secs / K * (G / Gs), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s (CPU oracle on the first %d of %d prompts per step)" % (cfg.name, Gs, G)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "oracle step on %d prompts (%d rows) per step plus its KV reindex loop rate "
+                                   "(%.1f GB/s on a 4-row slice) applied to the step's moved bytes" % (
+                                       Gs, Gs * cfg.N, copy_gbs)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="batched_prompts", choices=sorted(gen.CONFIGS))
+    ap.add_argument("--groups", type=int, default=None, help="override the number of prompts (default: the workload's)")
+    ap.add_argument("--e2e-steps", type=int, default=24)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 256 if args.steps is None else args.steps
+        args.warmup = 8 if args.warmup is None else args.warmup
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

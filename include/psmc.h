@@ -183,6 +183,13 @@ int psmc_rows(const psmc_ctx*);              /* R                               
 psmc_status psmc_set_state(psmc_ctx*, const double* log_w, const double* cum_logp,
                            const uint8_t* done, const int32_t* lens);
 
+/* Profiling aid.  While enabled, every kernel launched by psmc_step / psmc_step_host /
+ * psmc_reindex_kv is bracketed by CUDA events on the caller's stream.  psmc_timing_read waits for
+ * the recorded events, adds up the device time per kernel (HOST arrays of 3: [0] logit pass,
+ * [1] weights/ESS/resampling, [2] KV reindex; milliseconds and launch counts) and clears the record. */
+psmc_status psmc_timing_enable(psmc_ctx*, int on);
+psmc_status psmc_timing_read(psmc_ctx*, double* ms_out, int64_t* launches_out);
+
 /* Synchronises `stream` and returns the sticky device status word (PSMC_OK if
  * nothing went wrong since the last reset). */
 psmc_status psmc_sync_status(psmc_ctx*, void* stream);

@@ -91,7 +91,8 @@ int orc_row(const double* l, int V, double beta, double alpha_t, double U, int f
     }
     double mg = 1.0;
     if (below > 0.0) mg = fmin(mg, fabs(U - below / total));
-    if (at < total) mg = fmin(mg, fabs(at / total - U));
+    /* the upper fence exists whenever a later token has mass, even one too small to move the fp64 prefix */
+    if (pick < last_pos) mg = fmin(mg, fabs(at / total - U));
 
     int tok = force >= 0 ? force : pick;
     double lp = l[tok] - l1;

@@ -80,6 +80,10 @@ def lib():
         L.psmc_set_state.argtypes = [vp, vp, vp, vp, vp]
         L.psmc_sync_status.restype = C.c_int
         L.psmc_sync_status.argtypes = [vp, vp]
+        L.psmc_timing_enable.restype = C.c_int
+        L.psmc_timing_enable.argtypes = [vp, C.c_int]
+        L.psmc_timing_read.restype = C.c_int
+        L.psmc_timing_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.psmc_strerror.restype = C.c_char_p
         L.psmc_strerror.argtypes = [C.c_int]
         _lib = L
@@ -219,6 +223,15 @@ class Psmc:
         c = None if done is None else np.ascontiguousarray(done, dtype=np.uint8)
         d = None if lens is None else np.ascontiguousarray(lens, dtype=np.int32)
         _check(lib().psmc_set_state(self._h, _ptr(a), _ptr(b), _ptr(c), _ptr(d)), "psmc_set_state")
+
+    def timing_enable(self, on: bool):
+        _check(lib().psmc_timing_enable(self._h, 1 if on else 0), "psmc_timing_enable")
+
+    def timing_read(self):
+        """(ms[3], launches[3]) for the logit pass, the weights/resampling kernel and the KV reindex."""
+        ms, n = (C.c_double * 3)(), (C.c_int64 * 3)()
+        _check(lib().psmc_timing_read(self._h, ms, n), "psmc_timing_read")
+        return list(ms), list(n)
 
     def sync_status(self, stream=None) -> int:
         return lib().psmc_sync_status(self._h, _stream(stream))

@@ -3,6 +3,7 @@
 // Section 4.3 for the token at hand and enqueues the kernels on the caller's stream.
 #include <new>
 #include <string.h>
+#include <vector>
 
 #include "internal.h"
 
@@ -31,6 +32,11 @@ struct psmc_ctx {
     void* scratch;       // logit-pass tickets and span triples
     void* staging;       // psmc_step_host: device copy of the host logits
     size_t staging_bytes;
+    // optional per-kernel timing (psmc_timing_enable): event pairs recorded around every launch
+    int timing_on;
+    struct Timed { cudaEvent_t a, b; int kind; };
+    std::vector<Timed> timed;
+    std::vector<cudaEvent_t> event_pool;
 };
 
 namespace {
@@ -77,8 +83,38 @@ psmc_status reset_device_state(psmc_ctx* c) {
     return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
+// Brackets one kernel launch with events on the caller's stream when timing is on.
+struct LaunchTimer {
+    psmc_ctx* c;
+    cudaStream_t s;
+    psmc_ctx::Timed t;
+    bool on;
+    LaunchTimer(psmc_ctx* ctx, cudaStream_t stream, int kind) : c(ctx), s(stream), on(ctx->timing_on != 0) {
+        if (!on) return;
+        cudaEvent_t ev[2];
+        for (int i = 0; i < 2; ++i) {
+            if (!c->event_pool.empty()) {
+                ev[i] = c->event_pool.back();
+                c->event_pool.pop_back();
+            } else if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+                on = false;
+                return;
+            }
+        }
+        t.a = ev[0]; t.b = ev[1]; t.kind = kind;
+        cudaEventRecord(t.a, s);
+    }
+    ~LaunchTimer() {
+        if (!on) return;
+        cudaEventRecord(t.b, s);
+        c->timed.push_back(t);
+    }
+};
+
 void free_ctx(psmc_ctx* c) {
     if (!c) return;
+    for (auto& t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+    for (auto e : c->event_pool) cudaEventDestroy(e);
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok_draw, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->scratch, c->staging};
@@ -101,7 +137,6 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     if ((int64_t)G * N > (1 << 24)) return PSMC_E_INVAL;
     psmc_ctx* c = new (std::nothrow) psmc_ctx();
     if (!c) return PSMC_E_NOMEM;
-    memset(c, 0, sizeof(*c));
     if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return PSMC_E_CUDA; }
     c->G = G; c->N = N; c->V = V; c->R = G * N; c->ramp = ramp; c->eos = eos_id; c->T_max = T_max;
     c->alpha = (double)alpha; c->tau = (double)tau; c->kappa = (double)ess_thresh; c->seed = seed;
@@ -168,7 +203,10 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     la.done = c->done; la.scratch = c->scratch; la.tok = c->tok_draw; la.logp = c->logp; la.loginc = c->loginc;
     la.status = c->status;
     la.zero_words = c->counts[0];  // the step's two move counters are cleared by the first kernel of the step
-    if (launch_logits_pass(la, s) != cudaSuccess) return PSMC_E_CUDA;
+    {
+        LaunchTimer lt(c, s, 0);
+        if (launch_logits_pass(la, s) != cudaSuccess) return PSMC_E_CUDA;
+    }
 
     WeightsArgs wa{};
     wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos;
@@ -182,7 +220,10 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     wa.sources = c->sources[0]; wa.dst_rows = c->dst_rows[0];
     wa.n_sources = c->counts[0]; wa.n_moves = c->counts[0] + 1;
     wa.status = c->status;
-    if (launch_weights_resample(wa, s) != cudaSuccess) return PSMC_E_CUDA;
+    {
+        LaunchTimer lt(c, s, 1);
+        if (launch_weights_resample(wa, s) != cudaSuccess) return PSMC_E_CUDA;
+    }
     c->t = t;
     return PSMC_OK;
 }
@@ -266,6 +307,7 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
             k.dst[2 * l + 1] = static_cast<char*>(d->v[l0 + l]);
         }
         k.n_ptrs = 2 * nl;
+        LaunchTimer lt(c, s, 2);
         if (launch_reindex_kv(k, s) != cudaSuccess) return PSMC_E_CUDA;
     }
     return PSMC_OK;
@@ -301,6 +343,28 @@ extern "C" psmc_status psmc_sync_status(psmc_ctx* c, void* stream) {
     int32_t w = 0;
     if (cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PSMC_E_CUDA;
     return (psmc_status)w;
+}
+
+extern "C" psmc_status psmc_timing_enable(psmc_ctx* c, int on) {
+    if (!c) return PSMC_E_INVAL;
+    c->timing_on = on ? 1 : 0;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_timing_read(psmc_ctx* c, double* ms_out, int64_t* launches_out) {
+    if (!c || !ms_out || !launches_out) return PSMC_E_INVAL;
+    for (int k = 0; k < 3; ++k) { ms_out[k] = 0.0; launches_out[k] = 0; }
+    psmc_status st = PSMC_OK;
+    for (auto& t : c->timed) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(t.b) != cudaSuccess || cudaEventElapsedTime(&ms, t.a, t.b) != cudaSuccess)
+            st = PSMC_E_CUDA;
+        if (t.kind >= 0 && t.kind < 3) { ms_out[t.kind] += (double)ms; launches_out[t.kind] += 1; }
+        c->event_pool.push_back(t.a);
+        c->event_pool.push_back(t.b);
+    }
+    c->timed.clear();
+    return st;
 }
 
 extern "C" const char* psmc_strerror(psmc_status s) {

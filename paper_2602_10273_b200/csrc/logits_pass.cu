@@ -323,11 +323,12 @@ __device__ void finish_row(const Params& p, int row, int lane) {
             p.loginc[row] = 0.0;
         } else {
             const double dl = (double)load_elem<DT>(rowp, y) - M;
-            const double lp = dl - log(S1);            // log p(y) = l_y - L1
-            const double lq = p.beta * dl - log(Sb);   // log q(y) = beta l_y - Lb
+            const double ln_s1 = log(S1), ln_sb = log(Sb);
             p.tok[row] = y;
-            p.logp[row] = lp;
-            p.loginc[row] = p.alpha_t * lp - lq;
+            p.logp[row] = dl - ln_s1;  // log p(y) = l_y - L1
+            // alpha_t log p(y) - log q(y) with log q(y) = beta l_y - Lb, grouped so that the token's own
+            // logit drops out exactly when beta = alpha_t (Theorem 1)
+            p.loginc[row] = (p.alpha_t - p.beta) * dl - p.alpha_t * ln_s1 + ln_sb;
         }
     }
 }
