@@ -103,8 +103,9 @@ psmc_status psmc_step_host(psmc_ctx*, const void* logits_host, psmc_dtype dt, in
  * logp[r] - (beta*l_y - Lb).  All pointers DEVICE.  u: [R] uniforms in (0,1).
  * done may be NULL (all live); rows with done[r]!=0 are left untouched.
  * scratch: at least psmc_logits_pass_scratch_bytes(R, V) bytes, 256-byte
- * aligned, zero-filled before the FIRST use (the pass leaves it zeroed again);
- * status_word: one int32, sticky PSMC_E_* code (0 = fine). */
+ * aligned, contents irrelevant on entry (it carries per-span partial sums from
+ * the streaming kernel to the finishing kernel of this call); status_word: one
+ * int32, sticky PSMC_E_* code (0 = fine).  A flagged row gets tok = -1. */
 size_t psmc_logits_pass_scratch_bytes(int R, int V);
 psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R, int V, int64_t ld,
                              double beta, double alpha_t, const double* u, const uint8_t* done,

@@ -20,7 +20,7 @@ struct psmc_ctx {
     uint8_t* done;
     int32_t* len;
     // results of the last step
-    int32_t *tok_draw, *tok, *last_tok, *anc, *map, *resampled;
+    int32_t *tok, *last_tok, *anc, *map, *resampled;
     double *logp, *loginc, *ess, *logZ;
     // ancestry log for psmc_select
     int32_t *hist_tok, *hist_map;  // [T_max][R]
@@ -60,7 +60,6 @@ psmc_status reset_device_state(psmc_ctx* c) {
     z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
     z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
     z(c->counts[0], 8); z(c->counts[1], 8); z(c->status, 4);
-    z(c->scratch, logits_pass_scratch_bytes(c->R, c->V));
     if (e != cudaSuccess) return PSMC_E_CUDA;
     // lens = prompt length of the group; identity maps; tokens -1; ESS = N
     int32_t* h = new (std::nothrow) int32_t[R];
@@ -73,7 +72,6 @@ psmc_status reset_device_state(psmc_ctx* c) {
     if (e == cudaSuccess) e = cudaMemcpy(c->map, h, 4 * R, cudaMemcpyHostToDevice);
     for (size_t r = 0; r < R; ++r) h[r] = -1;
     if (e == cudaSuccess) e = cudaMemcpy(c->tok, h, 4 * R, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemcpy(c->tok_draw, h, 4 * R, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(c->last_tok, h, 4 * R, cudaMemcpyHostToDevice);
     for (size_t g = 0; g < G; ++g) hd[g] = (double)c->N;
     if (e == cudaSuccess) e = cudaMemcpy(c->ess, hd, 8 * G, cudaMemcpyHostToDevice);
@@ -115,7 +113,7 @@ void free_ctx(psmc_ctx* c) {
     if (!c) return;
     for (auto& t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : c->event_pool) cudaEventDestroy(e);
-    void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok_draw, c->tok, c->last_tok, c->anc, c->map, c->resampled,
+    void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->scratch, c->staging};
     for (void* p : ptrs)
@@ -150,7 +148,7 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     cudaError_t e = cudaSuccess;
     auto ok = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
     ok(dev_alloc(&c->logW, R)); ok(dev_alloc(&c->S, R)); ok(dev_alloc(&c->done, R)); ok(dev_alloc(&c->len, R));
-    ok(dev_alloc(&c->tok_draw, R)); ok(dev_alloc(&c->tok, R)); ok(dev_alloc(&c->last_tok, R));
+    ok(dev_alloc(&c->tok, R)); ok(dev_alloc(&c->last_tok, R));
     ok(dev_alloc(&c->anc, R)); ok(dev_alloc(&c->map, R)); ok(dev_alloc(&c->resampled, (size_t)G));
     ok(dev_alloc(&c->logp, R)); ok(dev_alloc(&c->loginc, R)); ok(dev_alloc(&c->ess, (size_t)G));
     ok(dev_alloc(&c->logZ, (size_t)G));
@@ -197,21 +195,20 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     const double alpha_t = alpha_at(c, t), alpha_prev = alpha_at(c, t - 1);
     const double beta_t = alpha_t / (c->alpha * c->tau);  // tau = 1/alpha gives beta_t = alpha_t (Corollary 1)
 
-    LogitsPassArgs la{};
-    la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld;
-    la.beta = beta_t; la.alpha_t = alpha_t; la.u = nullptr; la.seed = c->seed; la.t = t; la.N = c->N;
-    la.done = c->done; la.scratch = c->scratch; la.tok = c->tok_draw; la.logp = c->logp; la.loginc = c->loginc;
-    la.status = c->status;
+    LogitsStreamArgs la{};
+    la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = beta_t;
+    la.done = c->done; la.scratch = c->scratch;
     la.zero_words = c->counts[0];  // the step's two move counters are cleared by the first kernel of the step
     {
         LaunchTimer lt(c, s, 0);
-        if (launch_logits_pass(la, s) != cudaSuccess) return PSMC_E_CUDA;
+        if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
     }
 
     WeightsArgs wa{};
     wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos;
-    wa.alpha_t = alpha_t; wa.delta = alpha_t - alpha_prev; wa.kappa = c->kappa; wa.seed = c->seed;
-    wa.tok_draw = c->tok_draw; wa.logp = c->logp; wa.loginc = c->loginc;
+    wa.alpha_t = alpha_t; wa.beta = beta_t; wa.delta = alpha_t - alpha_prev; wa.kappa = c->kappa; wa.seed = c->seed;
+    wa.logits = logits; wa.dt = dt; wa.V = c->V; wa.ld = ld; wa.scratch = c->scratch;
+    wa.logp = c->logp; wa.loginc = c->loginc;
     wa.logW = c->logW; wa.S = c->S; wa.done = c->done; wa.len = c->len;
     wa.tok = c->tok; wa.last_tok = c->last_tok; wa.anc = c->anc; wa.map = c->map;
     wa.resampled = c->resampled; wa.ess = c->ess; wa.logZ = c->logZ;

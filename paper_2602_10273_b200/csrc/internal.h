@@ -13,26 +13,24 @@ constexpr int kMaxParticles = 1024;  // one CTA per group in the weight/resample
 constexpr int kSMs = 148;            // B200
 
 // ---------------------------------------------------------------- logit pass (Eq. 7, Corollary 1)
-struct LogitsPassArgs {
+struct LogitsStreamArgs {
     const void* logits;
     int dt;          // psmc_dtype
     int R, V;
     int64_t ld;
-    double beta, alpha_t;
-    const double* u;       // [R] uniforms, or NULL to hash (seed, token stream, row / N, t, row % N)
-    uint64_t seed;
-    int t, N;
+    double beta;
     const uint8_t* done;   // may be NULL
-    void* scratch;         // counters + partials
-    int32_t* tok;
-    double* logp;
-    double* loginc;
-    int32_t* status;
-    int32_t* zero_words;   // optional: two consecutive words the pass clears before anything else (may be NULL)
+    void* scratch;         // span triples, logits_pass_scratch_bytes(R, V)
+    int32_t* zero_words;   // optional: two consecutive words the kernel clears before anything else (may be NULL)
 };
-int logits_pass_span(int R, int V);               // elements per warp task
+struct LogitsGeometry {    // how a [R, V] block is cut up; a pure function of the arguments
+    int span, n_spans, mode, vec;
+    float cb;
+};
+int logits_pass_span(int R, int V);               // logits per warp task
 size_t logits_pass_scratch_bytes(int R, int V);
-cudaError_t launch_logits_pass(const LogitsPassArgs& a, cudaStream_t stream);
+LogitsGeometry logits_geometry(const void* logits, int dt, int R, int V, int64_t ld, double beta);
+cudaError_t launch_logits_stream(const LogitsStreamArgs& a, cudaStream_t stream);
 
 // ---------------------------------------------------------------- weights, ESS, resampling
 struct MoveSource {      // one surviving particle with surplus offspring
@@ -43,11 +41,15 @@ struct MoveSource {      // one surviving particle with surplus offspring
 };
 struct WeightsArgs {
     int G, N, R, t, eos;
-    double alpha_t, delta, kappa;
+    double alpha_t, beta, delta, kappa;
     uint64_t seed;
-    // from the logit pass
-    const int32_t* tok_draw;
-    double* logp;      // zeroed here for finished rows
+    // the logit block of this step and the span triples the streaming kernel left
+    const void* logits;
+    int dt, V;
+    int64_t ld;
+    const void* scratch;
+    // per-row results of the finish (written here; zero for finished rows)
+    double* logp;
     double* loginc;
     // particle state, updated in place
     double* logW;

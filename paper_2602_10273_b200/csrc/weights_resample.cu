@@ -1,28 +1,36 @@
-// Weights, ESS and ESS-triggered systematic resampling for one token (Algorithm 1 rows 6-16,
-// Eq. 5, and the stage-boundary update of Section 4.3 / Appendix B).  One CTA per group, one
-// thread per particle (N <= 1024); reductions and prefix sums run on warp shuffles plus a
-// 33-entry shared array, in an order fixed by the thread index.
+// Second kernel of the step: per-row finish of the logit pass, then weights, ESS and ESS-triggered
+// systematic resampling (Algorithm 1 rows 5-16, Eq. 5, Eq. 7, and the stage-boundary update of
+// Section 4.3 / Appendix B).  One CTA per group.
 //
-// Per particle i of group g (row r = g*N + i):
+// Phase 1 (one warp per particle, looping when N > 32): finish_row() turns the span triples of the
+// streaming kernel into the drawn token y, log p(y) and log omega of the row.
+// Phase 2 (one thread per particle, N <= 1024); reductions and prefix sums run on warp shuffles plus a
+// 33-entry shared array, in an order fixed by the thread index:
 //   log W_r += (alpha_t - alpha_{t-1}) * S_r                     stage boundary (all rows)
 //   live:  log W_r += log omega_r;  S_r += log p(y);  len_r += 1;  done_r |= (y == EOS)
 //   done:  y = EOS, factor 1
-// Per group:  w_i = exp(log W_i - max), C = inclusive prefix of w, ESS = (sum w)^2 / sum w^2.
-// If ESS < kappa*N:  u0 = hash uniform, A_i = min{j : C_j * N >= (u0 + i) * C_{N-1}} (N-1 if none),
-// offspring counts -> hazard-free slot map (survivors stay; dead slots, in increasing order, take
-// the surplus offspring, sources in increasing order), state gathered by the map, log W <- 0,
-// log Z-hat += max + log(sum w / N).  Move records for the KV reindex are appended to global lists.
-#include "common.cuh"
+//   w_i = exp(log W_i - max), C = inclusive prefix of w, ESS = (sum w)^2 / sum w^2.
+//   If ESS < kappa*N:  u0 = hash uniform, A_i = min{j : C_j * N >= (u0 + i) * C_{N-1}} (N-1 if none),
+//   offspring counts -> hazard-free slot map (survivors stay; dead slots, in increasing order, take
+//   the surplus offspring, sources in increasing order), state gathered by the map, log W <- 0,
+//   log Z-hat += max + log(sum w / N).  Move records for the KV reindex are appended to global lists.
 #include "internal.h"
+#include "logits_common.cuh"
 
 namespace psmc {
 namespace {
 
-__global__ void weights_resample_kernel(const WeightsArgs a) {
+struct KernelArgs {
+    WeightsArgs a;
+    FinishParams f;
+};
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __grid_constant__ KernelArgs ka) {
     __shared__ double sh_red[33];
     __shared__ int sh_redi[33];
-    __shared__ double sh_C[kMaxParticles];
-    __shared__ double sh_S[kMaxParticles];
+    __shared__ double sh_C[kMaxParticles];    // phase 1: log omega; phase 2: weight prefix
+    __shared__ double sh_S[kMaxParticles];    // phase 1: log p(y);  phase 2: cumulative log p
     __shared__ int sh_off[kMaxParticles];
     __shared__ int sh_Einc[kMaxParticles];
     __shared__ int sh_len[kMaxParticles];
@@ -30,11 +38,28 @@ __global__ void weights_resample_kernel(const WeightsArgs a) {
     __shared__ unsigned char sh_done[kMaxParticles];
     __shared__ int sh_base[2];
 
+    const WeightsArgs& a = ka.a;
     const int g = blockIdx.x, i = threadIdx.x, N = a.N;
+    const int lane = i & 31, warp = i >> 5, n_warps = blockDim.x >> 5;
+
+    // ---- phase 1: one warp per live particle finishes its row ----
+    for (int k = warp; k < N; k += n_warps) {
+        const int row = g * N + k;
+        if (a.done[row]) continue;
+        const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)k));
+        const RowResult rr = finish_row<DT, MODE>(ka.f, row, U, lane);
+        if (lane == 0) {
+            if (rr.tok < 0) raise_status(a.status, PSMC_E_NUMERIC);
+            sh_tok[k] = rr.tok;
+            sh_S[k] = rr.logp;
+            sh_C[k] = rr.loginc;
+        }
+    }
+    __syncthreads();
+
+    // ---- phase 2: per-particle update ----
     const bool on = i < N;
     const int r = g * N + (on ? i : 0);
-
-    // ---- per-particle update ----
     double lw = -INFINITY, S = 0.0;
     int tk = a.eos, ln = 0;
     unsigned char dn = 1;
@@ -43,17 +68,23 @@ __global__ void weights_resample_kernel(const WeightsArgs a) {
         S = a.S[r];
         ln = a.len[r];
         lw = a.logW[r] + a.delta * S;
-        if (dn) {
-            a.logp[r] = 0.0;
-            a.loginc[r] = 0.0;
-        } else {
-            tk = a.tok_draw[r];
-            if (tk < 0) tk = a.eos;  // the logit pass flagged the row; keep indices valid
-            lw += a.loginc[r];
-            S += a.logp[r];
+        double lp = 0.0, inc = 0.0;
+        if (!dn) {
+            tk = sh_tok[i];
+            lp = sh_S[i];
+            inc = sh_C[i];
+            if (tk < 0) {  // the row was flagged: keep indices valid, leave the weight alone
+                tk = a.eos;
+                lp = 0.0;
+                inc = 0.0;
+            }
+            lw += inc;
+            S += lp;
             ln += 1;
             if (tk == a.eos) dn = 1;
         }
+        a.logp[r] = lp;
+        a.loginc[r] = inc;
         a.tok[r] = tk;
         a.hist_tok[r] = tk;
     }
@@ -101,7 +132,7 @@ __global__ void weights_resample_kernel(const WeightsArgs a) {
         const double pos = (u0 + (double)i) * s1;
         int lo = 0, hi = N;  // first j in [0,N) with C_j * N >= pos; C is non-decreasing
         while (lo < hi) {
-            int mid = (lo + hi) >> 1;
+            const int mid = (lo + hi) >> 1;
             if (sh_C[mid] * (double)N >= pos) hi = mid; else lo = mid + 1;
         }
         anc = lo < N ? lo : N - 1;
@@ -128,7 +159,7 @@ __global__ void weights_resample_kernel(const WeightsArgs a) {
         const int rank = dead_incl - 1;  // this dead slot takes surplus offspring number `rank`
         int lo = 0, hi = N;              // first j with Einc[j] > rank
         while (lo < hi) {
-            int mid = (lo + hi) >> 1;
+            const int mid = (lo + hi) >> 1;
             if (sh_Einc[mid] > rank) hi = mid; else lo = mid + 1;
         }
         mp = lo < N ? lo : N - 1;
@@ -157,11 +188,30 @@ __global__ void weights_resample_kernel(const WeightsArgs a) {
     if (i == 0) a.logZ[g] += M + log(s1 / (double)N);
 }
 
+typedef void (*Fn)(const KernelArgs);
+template <int DT>
+Fn pick(int mode) {
+    switch (mode) {
+        case kBeta1: return finish_weights_resample_kernel<DT, kBeta1>;
+        case kBeta2: return finish_weights_resample_kernel<DT, kBeta2>;
+        case kBeta4: return finish_weights_resample_kernel<DT, kBeta4>;
+        case kBeta8: return finish_weights_resample_kernel<DT, kBeta8>;
+        default: return finish_weights_resample_kernel<DT, kBetaAny>;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream) {
-    int threads = ((a.N + 31) / 32) * 32;
-    weights_resample_kernel<<<a.G, threads, 0, stream>>>(a);
+    const LogitsGeometry g = logits_geometry(a.logits, a.dt, a.R, a.V, a.ld, a.beta);
+    KernelArgs ka;
+    ka.a = a;
+    ka.f.logits = a.logits; ka.f.V = a.V; ka.f.ld = a.ld; ka.f.span = g.span; ka.f.n_spans = g.n_spans;
+    ka.f.partials = reinterpret_cast<const float4*>(a.scratch); ka.f.beta = a.beta; ka.f.alpha_t = a.alpha_t;
+    ka.f.cb = g.cb; ka.f.vec = g.vec;
+    const int warps = a.N < 32 ? a.N : 32;  // one warp per particle up to 32, then the warps loop
+    Fn fn = a.dt == PSMC_F32 ? pick<PSMC_F32>(g.mode) : pick<PSMC_BF16>(g.mode);
+    fn<<<a.G, warps * 32, 0, stream>>>(ka);
     return cudaGetLastError();
 }
 

@@ -28,7 +28,7 @@ def _to_double(t):
 def run_logits_pass(logits, beta, alpha_t, u, done=None):
     R, V = logits.shape
     dev = logits.device
-    scratch = torch.zeros(B.logits_pass_scratch_bytes(R, V) + 256, dtype=torch.uint8, device=dev)
+    scratch = torch.full((B.logits_pass_scratch_bytes(R, V) + 256,), 0xA5, dtype=torch.uint8, device=dev)
     off = (-scratch.data_ptr()) % 256
     scratch = scratch[off:off + B.logits_pass_scratch_bytes(R, V)]
     tok = torch.full((R,), -7, dtype=torch.int32, device=dev)
@@ -37,10 +37,9 @@ def run_logits_pass(logits, beta, alpha_t, u, done=None):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ud = torch.from_numpy(np.asarray(u, dtype=np.float64)).to(dev)
     dd = None if done is None else torch.from_numpy(np.asarray(done, dtype=np.uint8)).to(dev)
-    for _ in range(2):  # twice: the pass must leave its scratch ready for the next call
+    for _ in range(2):  # twice: nothing of the first call may leak into the second through the scratch
         B.logits_pass(logits, beta, alpha_t, ud, dd, scratch, tok, logp, loginc, status)
     torch.cuda.synchronize()
-    assert int(scratch[: 4 * R].view(torch.int32).abs().sum()) == 0
     return tok.cpu().numpy(), logp.cpu().numpy(), loginc.cpu().numpy(), int(status.item())
 
 
