@@ -49,7 +49,8 @@ typedef enum {
     PSMC_E_STATE = 4,   /* call out of order (e.g. step beyond T_max)              */
     PSMC_E_NUMERIC = 5, /* NaN / +inf logit, or a row with no finite logit         */
     PSMC_E_TIMEOUT = 6, /* a bounded device-side wait gave up                      */
-    PSMC_E_HAZARD = 7   /* in-place gather vector reads a row that is also written */
+    PSMC_E_HAZARD = 7,  /* in-place gather vector reads a row that is also written */
+    PSMC_E_TOO_LARGE = 8 /* problem needs more than the fixed scratch of psmc_logits_pass_static */
 } psmc_status;
 
 typedef enum { PSMC_F32 = 0, PSMC_BF16 = 1 } psmc_dtype;
@@ -111,6 +112,43 @@ psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R, int V, in
                              double beta, double alpha_t, const double* u, const uint8_t* done,
                              void* scratch, size_t scratch_bytes, int32_t* tok, double* logp,
                              double* loginc, int32_t* status_word, void* stream);
+
+/* The logit pass for callers that cannot allocate device memory.  (The paper
+ * has no counterpart: this is a packaging variant of psmc_logits_pass.)
+ *
+ * Some hosts of this library are handed raw input and output pointers and
+ * nothing else: a custom-op hook inside a serving runtime whose memory pool
+ * belongs to the runtime, a plug-in running under a framework that forbids
+ * cudaMalloc while its own allocator is active (cudaMalloc synchronises the
+ * device and would stall every other stream), a real-time loop with a "no
+ * allocation after start-up" rule.  They have nowhere to get the scratch
+ * buffer psmc_logits_pass asks for, and psmc_init is closed to them too.
+ *
+ * This entry point takes the same inputs and outputs as psmc_logits_pass but
+ * no scratch: the per-span partial sums go to a fixed array of
+ * PSMC_STATIC_SCRATCH_BYTES that is part of the library's device image, so
+ * every GPU that loads the library carries it (4 MiB) until the process exits.
+ * The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   - Limit: psmc_logits_pass_scratch_bytes(R, V) must not exceed
+ *     PSMC_STATIC_SCRATCH_BYTES (16 bytes per span of 1024-4096 logits per row;
+ *     e.g. 512 rows x 128256 logits need 516,096 bytes).  Larger problems are
+ *     refused with PSMC_E_TOO_LARGE and nothing is enqueued.
+ *   - First call on each device: looks up the array's device address (a
+ *     runtime symbol query, with that device current) and caches it.  Make that
+ *     first call outside any stream capture.
+ *   - One array per device, shared by every call and every stream: two calls
+ *     that overlap on the GPU (different streams, or different host threads
+ *     without ordering) race on it and corrupt each other's results.  Issue
+ *     calls on one stream or order them yourself.  The array keeps the previous
+ *     call's contents; nothing in it needs clearing, because each call
+ *     overwrites every entry it later reads.
+ * Results are identical to psmc_logits_pass on the same inputs. */
+#define PSMC_STATIC_SCRATCH_BYTES (4u << 20)
+psmc_status psmc_logits_pass_static(const void* logits, psmc_dtype dt, int R, int V, int64_t ld,
+                                    double beta, double alpha_t, const double* u,
+                                    const uint8_t* done, int32_t* tok, double* logp, double* loginc,
+                                    int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------- */
 /* KV-cache reindex (Algorithm 1 row 14, Appendix C)                          */

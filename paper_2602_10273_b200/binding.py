@@ -15,7 +15,8 @@ import torch
 
 from . import build as _build
 
-OK, E_INVAL, E_NOMEM, E_CUDA, E_STATE, E_NUMERIC, E_TIMEOUT, E_HAZARD = range(8)
+OK, E_INVAL, E_NOMEM, E_CUDA, E_STATE, E_NUMERIC, E_TIMEOUT, E_HAZARD, E_TOO_LARGE = range(9)
+STATIC_SCRATCH_BYTES = 4 << 20
 F32, BF16 = 0, 1
 
 _lib = None
@@ -62,6 +63,9 @@ def lib():
         L.psmc_logits_pass.restype = C.c_int
         L.psmc_logits_pass.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_double, C.c_double, f64p, u8p,
                                        vp, C.c_size_t, i32p, f64p, f64p, i32p, vp]
+        L.psmc_logits_pass_static.restype = C.c_int
+        L.psmc_logits_pass_static.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_double, C.c_double, f64p,
+                                              u8p, i32p, f64p, f64p, i32p, vp]
         L.psmc_reindex_kv.restype = C.c_int
         L.psmc_reindex_kv.argtypes = [vp, C.POINTER(KvDesc), C.POINTER(KvDesc), i32p, vp]
         L.psmc_select.restype = C.c_int
@@ -292,3 +296,17 @@ def logits_pass(logits: torch.Tensor, beta: float, alpha_t: float, u: torch.Tens
                                   u.data_ptr(), _ptr(done), scratch.data_ptr(), scratch.numel() * scratch.element_size(),
                                   tok.data_ptr(), logp.data_ptr(), loginc.data_ptr(), status_word.data_ptr(),
                                   _stream(stream)), "psmc_logits_pass")
+
+
+def logits_pass_static(logits: torch.Tensor, beta: float, alpha_t: float, u: torch.Tensor, done, tok: torch.Tensor,
+                       logp: torch.Tensor, loginc: torch.Tensor, status_word: torch.Tensor, stream=None):
+    """psmc_logits_pass_static: the logit pass without a scratch argument, for callers that cannot allocate.
+
+    The span partials live in a fixed 4 MiB array inside the library; calls share it, so keep them on one
+    stream.  Raises PsmcError(E_TOO_LARGE) when logits_pass_scratch_bytes(R, V) exceeds STATIC_SCRATCH_BYTES."""
+    R, V = logits.shape
+    assert logits.stride(1) == 1 and u.dtype == torch.float64 and tok.dtype == torch.int32
+    _check(lib().psmc_logits_pass_static(logits.data_ptr(), _dtype_code(logits), R, V, logits.stride(0), beta,
+                                         alpha_t, u.data_ptr(), _ptr(done), tok.data_ptr(), logp.data_ptr(),
+                                         loginc.data_ptr(), status_word.data_ptr(), _stream(stream)),
+           "psmc_logits_pass_static")

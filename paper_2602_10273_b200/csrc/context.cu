@@ -374,6 +374,7 @@ extern "C" const char* psmc_strerror(psmc_status s) {
         case PSMC_E_NUMERIC: return "NaN/+inf logit or a row without finite logits";
         case PSMC_E_TIMEOUT: return "bounded device wait ran out";
         case PSMC_E_HAZARD: return "in-place gather vector reads a row that is also written";
+        case PSMC_E_TOO_LARGE: return "problem needs more than the fixed scratch of psmc_logits_pass_static";
     }
     return "unknown status";
 }

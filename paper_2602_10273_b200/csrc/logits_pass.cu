@@ -8,6 +8,8 @@
 // (m, s1, sb) triple and stores it; nothing else leaves the kernel.  No atomics, no fences, no waits:
 // spans are dealt round-robin to a grid that exactly fills the machine, so every warp does the same
 // amount of work.  The per-row finish (logits_common.cuh) runs in the kernel that follows.
+#include <mutex>
+
 #include "internal.h"
 #include "logits_common.cuh"
 
@@ -293,6 +295,70 @@ extern "C" psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R
     if (scratch_bytes < logits_pass_scratch_bytes(R, V) || reinterpret_cast<uintptr_t>(scratch) % 256 != 0)
         return PSMC_E_INVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LogitsStreamArgs a{};
+    a.logits = logits; a.dt = dt; a.R = R; a.V = V; a.ld = ld; a.beta = beta; a.done = done; a.scratch = scratch;
+    a.zero_words = nullptr;
+    if (launch_logits_stream(a, s) != cudaSuccess) return PSMC_E_CUDA;
+
+    const LogitsGeometry g = logits_geometry(logits, dt, R, V, ld, beta);
+    FinishKernelParams p;
+    p.f.logits = logits; p.f.V = V; p.f.ld = ld; p.f.span = g.span; p.f.n_spans = g.n_spans;
+    p.f.partials = reinterpret_cast<const float4*>(scratch); p.f.beta = beta; p.f.alpha_t = alpha_t; p.f.cb = g.cb;
+    p.f.vec = g.vec;
+    p.R = R; p.u = u; p.done = done; p.tok = tok; p.logp = logp; p.loginc = loginc; p.status = status_word;
+    FinishFn fn = dt == PSMC_F32 ? pick_finish<PSMC_F32>(g.mode) : pick_finish<PSMC_BF16>(g.mode);
+    fn<<<(unsigned)((R + kWarpsPerCta - 1) / kWarpsPerCta), kThreads, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The logit pass for callers that must not allocate: same two kernels, span triples kept in a
+// fixed array that lives in the library's device image instead of in caller memory.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Fixed scratch: room for PSMC_STATIC_SCRATCH_BYTES / 16 span triples.  It is part of the module, so
+// every GPU on which the library gets loaded carries these 4 MiB until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[PSMC_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices];  // device address of g_static_scratch, looked up once per device
+
+// `g_static_scratch` names a host-side handle in host code, not memory a kernel could use; the address
+// the kernels need comes from the runtime, per device, with that device current.
+cudaError_t static_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" psmc_status psmc_logits_pass_static(const void* logits, psmc_dtype dt, int R, int V, int64_t ld,
+                                               double beta, double alpha_t, const double* u, const uint8_t* done,
+                                               int32_t* tok, double* logp, double* loginc, int32_t* status_word,
+                                               void* stream) {
+    using namespace psmc;
+    if (!logits || !u || !tok || !logp || !loginc || !status_word) return PSMC_E_INVAL;
+    if (R < 1 || V < 2 || ld < V || !(beta > 0.0) || !(alpha_t >= 1.0)) return PSMC_E_INVAL;
+    if (dt != PSMC_F32 && dt != PSMC_BF16) return PSMC_E_INVAL;
+    if (logits_pass_scratch_bytes(R, V) > (size_t)PSMC_STATIC_SCRATCH_BYTES) return PSMC_E_TOO_LARGE;
+    void* scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess) return PSMC_E_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Nothing in the array has to start at zero: the streaming kernel writes every triple the finishing
+    // kernel reads, so whatever an earlier call left behind is never looked at.
     LogitsStreamArgs a{};
     a.logits = logits; a.dt = dt; a.R = R; a.V = V; a.ld = ld; a.beta = beta; a.done = done; a.scratch = scratch;
     a.zero_words = nullptr;
