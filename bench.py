@@ -121,9 +121,11 @@ def run_ours(args):
     from paper_2602_10273_b200 import binding as B
     from paper_2602_10273_b200.workload import cuda as WC
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2602_10273_b200 import replicas
+
+    cfg = gen.CONFIGS[args.workload]
+    plan = replicas.rank_plan(cfg.G if args.groups is None else args.groups)
+    world, rank, local = plan.world, plan.rank, plan.local_rank
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -131,7 +133,6 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     hbm_peak, peak_kind = load_peaks()
 
-    cfg = gen.CONFIGS[args.workload]
     K, Wm = args.steps, args.warmup
     T_total = K + Wm
     if cfg.prompt_hi + T_total > cfg.max_len:
@@ -143,7 +144,7 @@ def run_ours(args):
     fixed = N_BLOCKS * cfg.N * cfg.logit_bytes_per_row  # per group
     while G > 1 and G * (per_group + fixed) + (6 << 30) > free_b:
         G -= 1
-    seed = 1 + rank
+    seed = plan.seed
     wl = WC.DeviceWorkload(cfg, seed, G=G, device=dev)
     R, N = wl.R, cfg.N
     ks, vs = wl.new_kv()
@@ -179,23 +180,14 @@ def run_ours(args):
     live_timed = int(np.sum(live_rows[Wm:]))
 
     def barrier():
-        if world > 1:
-            torch.distributed.barrier()
+        replicas.barrier()
         torch.cuda.synchronize(dev)
 
     def max_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], dtype=torch.float64, device=dev)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            return float(t.item())
-        return x
+        return replicas.max_over_ranks(x, dev)
 
     def sum_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], dtype=torch.float64, device=dev)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.SUM)
-            return float(t.item())
-        return float(x)
+        return replicas.sum_over_ranks(x, dev)
 
     # ---- pass A: the headline. K steps, device-resident inputs, one pair of events around all of them ----
     ps.reset(seed)
@@ -323,19 +315,20 @@ def oracle_copy_rate(cfg):
     return reps * 2 * 2 * t[0].nbytes / dt / 1e9
 
 
-def cpu_baseline(cfg, wl, blocks, G, kv_bytes_per_step):
+def cpu_baseline(cfg, wl, blocks, G, kv_bytes_per_step, n_steps=24):
+    """The oracle as it stands on the host cores: every row of the workload for n_steps tokens (the logit blocks
+    the CUDA path was timed on, downloaded), plus the rate of its KV reindex loop applied to one step's moves."""
     cores = len(os.sched_getaffinity(0))
-    Gs = min(G, 8)                      # bounded sample: the first 8 prompts
-    host = [logits_to_numpy(b[: Gs * cfg.N]) for b in blocks[:3]]
-    rate, secs, rows = oracle_step_rate(cfg, wl.seed, Gs, host, wl.prompt_len[:Gs], 3)
+    host = [logits_to_numpy(b) for b in blocks]
+    rate, secs, rows = oracle_step_rate(cfg, wl.seed, G, host, wl.prompt_len, n_steps)
     copy_gbs = oracle_copy_rate(cfg)
     # one full step on the CPU = the oracle's step for all rows + its memcpy loop over the step's KV bytes
     t_step = (G * cfg.N) / rate + kv_bytes_per_step / (copy_gbs * 1e9)
     return {"value": (G * cfg.N) / t_step, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "oracle step on the first %d prompts (%d rows) for 3 tokens: %.0f rows/s in %.1f s; oracle KV "
-                      "reindex loop on a 4-row slice of one layer: %.1f GB/s; combined for one full step of %d rows "
-                      "and %.2f GB of KV moves" % (Gs, Gs * cfg.N, rate, secs, copy_gbs, G * cfg.N,
-                                                  kv_bytes_per_step / 1e9),
+            "sample": "oracle step on all %d prompts (%d rows) for %d tokens: %.0f rows/s in %.1f s wall on %d threads; "
+                      "oracle KV reindex loop on a 4-row slice of one layer: %.1f GB/s; combined for one full step of "
+                      "%d rows and %.2f GB of KV moves" % (G, G * cfg.N, n_steps, rate, secs, cores, copy_gbs,
+                                                          G * cfg.N, kv_bytes_per_step / 1e9),
             "oracle_rows_per_s": rate, "oracle_copy_gb_per_s": copy_gbs}
 
 
@@ -346,7 +339,7 @@ def run_reference(args):
     cfg = gen.CONFIGS[args.workload]
     seed = 1
     G = cfg.G if args.groups is None else args.groups
-    Gs = min(G, 2)                      # each step is a bounded sample: the first 2 prompts
+    Gs = min(G, 8)                      # each step is a bounded sample: the first 8 prompts
     bias = gen.vocab_bias(seed, cfg.V, cfg.slope)
     plen = gen.prompt_lengths(seed, G, cfg.prompt_lo, cfg.prompt_hi)
     prev = np.repeat(gen.prompt_last_token(seed, G, plen, cfg.V), cfg.N)[: Gs * cfg.N]
