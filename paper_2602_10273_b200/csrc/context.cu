@@ -29,6 +29,7 @@ struct psmc_ctx {
     int32_t* dst_rows[2];
     int32_t* counts[2];  // {n_sources, n_moves}
     int32_t* status;
+    int32_t* kv_work;    // [2] unit queue of the reindex kernels (kept at zero between launches by the kernels)
     void* scratch;       // logit-pass tickets and span triples
     void* staging;       // psmc_step_host: device copy of the host logits
     size_t staging_bytes;
@@ -59,7 +60,7 @@ psmc_status reset_device_state(psmc_ctx* c) {
     auto z = [&](void* p, size_t bytes) { if (e == cudaSuccess) e = cudaMemset(p, 0, bytes); };
     z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
     z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
-    z(c->counts[0], 8); z(c->counts[1], 8); z(c->status, 4);
+    z(c->counts[0], 8); z(c->counts[1], 8); z(c->status, 4); z(c->kv_work, 8);
     if (e != cudaSuccess) return PSMC_E_CUDA;
     // lens = prompt length of the group; identity maps; tokens -1; ESS = N
     int32_t* h = new (std::nothrow) int32_t[R];
@@ -115,7 +116,7 @@ void free_ctx(psmc_ctx* c) {
     for (auto e : c->event_pool) cudaEventDestroy(e);
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
-                    c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->scratch, c->staging};
+                    c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->kv_work, c->scratch, c->staging};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete[] c->prompt_len_host;
@@ -157,6 +158,7 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
         ok(dev_alloc(&c->sources[s], R)); ok(dev_alloc(&c->dst_rows[s], R)); ok(dev_alloc(&c->counts[s], 2));
     }
     ok(dev_alloc(&c->status, 1));
+    ok(dev_alloc(&c->kv_work, 2));
     ok(cudaMalloc(&c->scratch, logits_pass_scratch_bytes(c->R, c->V)));
     if (e != cudaSuccess) { free_ctx(c); return e == cudaErrorMemoryAllocation ? PSMC_E_NOMEM : PSMC_E_CUDA; }
     psmc_status st = reset_device_state(c);
@@ -287,6 +289,7 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
     k.dst_rows = c->dst_rows[set];
     k.n_sources = c->counts[set];
     k.status = c->status;
+    k.work = c->kv_work;
     uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |
                     (uint64_t)k.dst_head_bytes_stride | (uint64_t)k.pos_bytes;
     for (int l = 0; l < src->n_layers; ++l) {

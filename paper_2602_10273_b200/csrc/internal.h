@@ -90,6 +90,7 @@ struct KvLaunch {
     const int32_t* dst_rows;
     const int32_t* n_sources;
     int32_t* status;
+    int32_t* work;   // [2] unit queue of the copy kernels: next unit, CTAs that have left; both zero between launches
     int bulk_ok;     // 16-byte alignment holds everywhere
 };
 cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream);

@@ -67,7 +67,11 @@ __device__ __forceinline__ void bulk_wait_read() {
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Work item w -> (source record, pointer/head segment, chunk) and its byte range.
+// Work is handed out in units of one (source record, pointer/head segment): the live prefix of one head of one
+// K or V tensor of one surviving row.  Lengths differ from row to row, so a static deal of fixed-size pieces
+// leaves CTAs with unequal loads; instead every CTA takes the next unit from a global counter when it runs
+// out (the fetch of the unit after that is already in flight, so its latency stays off the copy pipeline).
+// A unit is streamed in chunks of kChunk bytes.
 struct Item {
     const char* src;
     int64_t dst_off;  // byte offset inside a destination row-head segment = chunk * kChunk
@@ -75,30 +79,47 @@ struct Item {
     int dst_begin, n_dst;
     uint32_t bytes;
 };
-__device__ __forceinline__ bool decode(const KvLaunch& k, int64_t w, int n_seg, int n_chunk, int chunk_bytes, Item& it) {
-    const int chunk = (int)(w % n_chunk);
-    const int64_t q = w / n_chunk;
-    const int seg = (int)(q % n_seg);
-    const int s = (int)(q / n_seg);
+struct UnitCursor {
+    int seg_ptr, seg_head, dst_begin, n_dst;
+    const char* src;     // start of the source segment
+    int64_t seg_bytes;   // live bytes of the segment
+    int64_t off;         // next byte to hand out
+};
+__device__ __forceinline__ void open_unit(const KvLaunch& k, int u, int n_seg, UnitCursor& c) {
+    const int s = u / n_seg, seg = u - s * n_seg;
     const MoveSource ms = k.sources[s];
-    int len = ms.len < k.max_len ? ms.len : k.max_len;
-    const int64_t seg_bytes = (int64_t)len * k.pos_bytes;
-    const int64_t off = (int64_t)chunk * chunk_bytes;
-    if (off >= seg_bytes) return false;
-    it.seg_ptr = seg / k.H;
-    it.seg_head = seg - it.seg_ptr * k.H;
-    it.src = k.src[it.seg_ptr] + (int64_t)ms.src_row * k.row_bytes_stride + (int64_t)it.seg_head * k.head_bytes_stride + off;
-    it.dst_off = off;
-    it.dst_begin = ms.dst_begin;
-    it.n_dst = ms.n_dst;
-    const int64_t left = seg_bytes - off;
-    it.bytes = (uint32_t)(left < chunk_bytes ? left : chunk_bytes);
-    return true;
+    const int len = ms.len < k.max_len ? ms.len : k.max_len;
+    c.seg_ptr = seg / k.H;
+    c.seg_head = seg - c.seg_ptr * k.H;
+    c.dst_begin = ms.dst_begin;
+    c.n_dst = ms.n_dst;
+    c.src = k.src[c.seg_ptr] + (int64_t)ms.src_row * k.row_bytes_stride + (int64_t)c.seg_head * k.head_bytes_stride;
+    c.seg_bytes = (int64_t)(len > 0 ? len : 0) * k.pos_bytes;
+    c.off = 0;
+}
+__device__ __forceinline__ void take_chunk(UnitCursor& c, Item& it) {
+    it.src = c.src + c.off;
+    it.dst_off = c.off;
+    it.seg_ptr = c.seg_ptr;
+    it.seg_head = c.seg_head;
+    it.dst_begin = c.dst_begin;
+    it.n_dst = c.n_dst;
+    const int64_t left = c.seg_bytes - c.off;
+    it.bytes = (uint32_t)(left < kChunk ? left : kChunk);
+    c.off += it.bytes;
 }
 __device__ __forceinline__ char* dst_addr(const KvLaunch& k, const Item& it, int d) {
     const int row = k.dst_rows[it.dst_begin + d];
     return k.dst[it.seg_ptr] + (int64_t)row * k.dst_row_bytes_stride + (int64_t)it.seg_head * k.dst_head_bytes_stride +
            it.dst_off;
+}
+// Last CTA out puts the unit counter back to zero for the next launch (launches on one context are stream-ordered).
+__device__ __forceinline__ void leave_queue(int32_t* work) {
+    __threadfence();
+    if (atomicInc(reinterpret_cast<unsigned int*>(work + 1), gridDim.x - 1) == gridDim.x - 1) {
+        work[0] = 0;
+        __threadfence();
+    }
 }
 
 __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant__ KvLaunch k) {
@@ -115,12 +136,24 @@ __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant_
     fence_async_smem();
 
     const int n_seg = k.n_ptrs * k.H;
-    const int n_chunk = (int)(((int64_t)k.max_len * k.pos_bytes + kChunk - 1) / kChunk);
-    const int64_t total = (int64_t)n_src * n_seg * n_chunk;
+    const int n_units = n_src * n_seg;   // < 2^31: rows <= 2^24 is checked at init, and segments per launch <= 128 * H
 
-    int64_t pw = blockIdx.x;
+    // unit queue: `next_u` is always one fetch ahead of the unit being streamed
+    UnitCursor cur;
+    cur.seg_bytes = 0;
+    cur.off = 0;
+    int next_u = atomicAdd(k.work, 1);
     Item cand;
-    while (pw < total && !decode(k, pw, n_seg, n_chunk, kChunk, cand)) pw += gridDim.x;
+    auto advance = [&]() -> bool {  // next chunk into `cand`; false when the queue is dry
+        while (cur.off >= cur.seg_bytes) {
+            if (next_u >= n_units) return false;
+            open_unit(k, next_u, n_seg, cur);
+            next_u = atomicAdd(k.work, 1);
+        }
+        take_chunk(cur, cand);
+        return true;
+    };
+    bool more = advance();
 
     int issued = 0, consumed = 0;
     bool failed = false;
@@ -140,15 +173,14 @@ __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant_
             ++consumed;
         }
         // produce item i into slot i % kStages, last used by item i-kStages
-        if (pw < total) {
+        if (more) {
             const int slot = i % kStages;
             if (i >= kStages) bulk_wait_read<1>();  // all store groups but the newest have read their stage
             ring[slot] = cand;
             mbar_expect_tx(&bars[slot], cand.bytes);
             bulk_load(smem + (size_t)slot * kChunk, cand.src, cand.bytes, &bars[slot]);
             ++issued;
-            pw += gridDim.x;
-            while (pw < total && !decode(k, pw, n_seg, n_chunk, kChunk, cand)) pw += gridDim.x;
+            more = advance();
         } else if (consumed == issued) {
             break;
         }
@@ -159,26 +191,35 @@ __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant_
         for (int j = consumed; j < issued; ++j) mbar_wait(&bars[j % kStages], (uint32_t)((j / kStages) & 1));
     }
     bulk_wait_all();
+    leave_queue(k.work);
 }
 
 // ---- plain path: ordinary loads and stores of unit type U ----
 template <typename U>
 __global__ void __launch_bounds__(256) reindex_plain_kernel(const __grid_constant__ KvLaunch k) {
+    __shared__ int sh_u;
     const int n_src = *reinterpret_cast<const volatile int32_t*>(k.n_sources);
     if (n_src <= 0) return;
     const int n_seg = k.n_ptrs * k.H;
-    const int n_chunk = (int)(((int64_t)k.max_len * k.pos_bytes + kChunk - 1) / kChunk);
-    const int64_t total = (int64_t)n_src * n_seg * n_chunk;
-    for (int64_t w = blockIdx.x; w < total; w += gridDim.x) {
+    const int n_units = n_src * n_seg;
+    for (;;) {
+        __syncthreads();  // everyone has read the previous sh_u
+        if (threadIdx.x == 0) sh_u = atomicAdd(k.work, 1);
+        __syncthreads();
+        const int u = sh_u;
+        if (u >= n_units) break;
+        UnitCursor c;
+        open_unit(k, u, n_seg, c);
         Item it;
-        if (!decode(k, w, n_seg, n_chunk, kChunk, it)) continue;
-        const int n_units = it.bytes / (int)sizeof(U);
-        const U* s = reinterpret_cast<const U*>(it.src);
-        for (int e = threadIdx.x; e < n_units; e += blockDim.x) {
+        it.seg_ptr = c.seg_ptr; it.seg_head = c.seg_head; it.dst_begin = c.dst_begin; it.n_dst = c.n_dst; it.dst_off = 0;
+        const int64_t n_units_u = c.seg_bytes / (int64_t)sizeof(U);
+        const U* s = reinterpret_cast<const U*>(c.src);
+        for (int64_t e = threadIdx.x; e < n_units_u; e += blockDim.x) {
             const U v = s[e];
             for (int d = 0; d < it.n_dst; ++d) reinterpret_cast<U*>(dst_addr(k, it, d))[e] = v;
         }
     }
+    if (threadIdx.x == 0) leave_queue(k.work);
 }
 
 // ---- arbitrary gather vector -> move records, with the in-place hazard check ----
