@@ -74,14 +74,15 @@ __device__ __forceinline__ T warp_scan_incl(T v, int lane) {
 }
 
 // ---- block collectives for up to 1024 threads (32 warps); `sh` holds 33 items ----
+// Every thread of the CTA calls them; only the first `nwarp` warps carry data (the others pass the identity).
 // Inclusive scan over threadIdx.x order.  Also returns the block total.  The order of additions is
 // fixed by the thread index, so results do not depend on scheduling.
 template <typename T>
-__device__ __forceinline__ T block_scan_incl(T v, T* sh, T* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+__device__ __forceinline__ T block_scan_incl(T v, T* sh, T* total, int nwarp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     T incl = warp_scan_incl(v, lane);
     __syncthreads();  // sh may still be read by a previous call
-    if (lane == 31) sh[warp] = incl;
+    if (lane == 31 && warp < nwarp) sh[warp] = incl;
     __syncthreads();
     T before = T(0), all = T(0);
     for (int w = 0; w < nwarp; ++w) {
@@ -93,21 +94,21 @@ __device__ __forceinline__ T block_scan_incl(T v, T* sh, T* total) {
     return before + incl;
 }
 template <typename T>
-__device__ __forceinline__ T block_max(T v, T* sh) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+__device__ __forceinline__ T block_max(T v, T* sh, int nwarp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     v = warp_max(v);
     __syncthreads();
-    if (lane == 0) sh[warp] = v;
+    if (lane == 0 && warp < nwarp) sh[warp] = v;
     __syncthreads();
     T m = sh[0];
     for (int w = 1; w < nwarp; ++w) m = m > sh[w] ? m : sh[w];
     return m;
 }
-__device__ __forceinline__ double block_sum(double v, double* sh) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+__device__ __forceinline__ double block_sum(double v, double* sh, int nwarp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     v = warp_sum(v);
     __syncthreads();
-    if (lane == 0) sh[warp] = v;
+    if (lane == 0 && warp < nwarp) sh[warp] = v;
     __syncthreads();
     double s = 0.0;
     for (int w = 0; w < nwarp; ++w) s += sh[w];

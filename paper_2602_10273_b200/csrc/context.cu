@@ -200,6 +200,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     LogitsStreamArgs la{};
     la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = beta_t;
     la.done = c->done; la.scratch = c->scratch;
+    la.status = c->status;
     la.zero_words = c->counts[0];  // the step's two move counters are cleared by the first kernel of the step
     {
         LaunchTimer lt(c, s, 0);

@@ -22,10 +22,11 @@ struct LogitsStreamArgs {
     const uint8_t* done;   // may be NULL
     void* scratch;         // span triples, logits_pass_scratch_bytes(R, V)
     int32_t* zero_words;   // optional: two consecutive words the kernel clears before anything else (may be NULL)
+    int32_t* status;       // sticky status word for a bounded wait that ran out (may be NULL)
 };
 struct LogitsGeometry {    // how a [R, V] block is cut up; a pure function of the arguments
     int span, n_spans, mode, vec;
-    float cb;
+    float bf;             // (float)beta
 };
 int logits_pass_span(int R, int V);               // logits per warp task
 size_t logits_pass_scratch_bytes(int R, int V);

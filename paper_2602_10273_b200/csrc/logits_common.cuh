@@ -6,9 +6,13 @@
 //   Lb = logsumexp(beta l)     normaliser of the tempered proposal q of Corollary 1
 //   y  = min{v : sum_{u<=v} exp(beta l_u) >= U sum_all}
 //   log p(y) = l_y - L1,  log omega = alpha_t log p(y) - (beta l_y - Lb)     (Eq. 7 in logs)
-// The streaming kernel cuts a row into spans and writes one triple (m, s1, sb) per span:
-//   m = max l over the span, s1 = sum exp(l - m), sb = sum exp(beta (l - m)).
-// finish_row() rescales the triples to the row maximum in fp64, in span order, finds the span
+// All exponentials are taken in base 2 (the hardware's ex2): with x_v = l_v * log2(e),
+//   exp(l_v) = 2^{x_v}.  x_v - c is formed as fma(l, k_lo, fma(l, k_hi, -c)) with log2(e) = k_hi + k_lo split
+// over two floats, so the product carries no representation error of log2(e) and the big parts cancel
+// before the small one is added.  The streaming kernel cuts a row into spans and writes one triple (c, s1, sb)
+// per span:   c = a reference exponent (close to the span's largest x),  s1 = sum 2^{x - c},
+//   sb = sum 2^{beta (x - c)}.
+// The finish rescales the triples to the row's largest c in fp64, in span order, finds the span
 // that holds U * sum_all by a prefix sum over the sb terms, and re-reads only that span.
 #pragma once
 
@@ -19,7 +23,10 @@
 namespace psmc {
 
 constexpr float kNegBig = -3.3895313892515355e38f;  // most negative finite bf16; start value of a running maximum
-constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRefFloor = -3.0e38f;               // reference exponent of a lane or span that saw no finite logit
+constexpr float kLog2eHi = 1.4426950216293335f;     // float(log2 e)
+constexpr float kLog2eLo = 1.925963033500011e-8f;   // float(log2 e - kLog2eHi)
+constexpr double kLn2 = 0.6931471805599453;
 
 enum BetaMode { kBeta1 = 0, kBeta2 = 1, kBeta4 = 2, kBeta8 = 3, kBetaAny = 4 };
 
@@ -37,17 +44,29 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// exp(beta * d) for d = l - m <= 0.  One MUFU: for beta in {1,2,4,8} exp(d) is squared up.
+// x - c for one logit: l * log2(e) - c
+__device__ __forceinline__ float rel_exponent(float l, float neg_c) {
+    return fmaf(l, kLog2eLo, fmaf(l, kLog2eHi, neg_c));
+}
+// reference exponent for a logit value m: about m * log2(e), kept finite
+__device__ __forceinline__ float ref_exponent(float m) { return fmaxf(m * kLog2eHi, kRefFloor); }
+
+// 2^{beta d} for d = x - c.  One MUFU: for beta in {1,2,4,8} 2^d is squared up; bf = (float)beta otherwise.
 template <int MODE>
-__device__ __forceinline__ float mass_beta(float d, float cb) {
-    if (MODE == kBetaAny) return ex2(d * cb);
-    float e = ex2(d * kLog2e);
+__device__ __forceinline__ float mass_beta(float d, float bf) {
+    if (MODE == kBetaAny) return ex2(d * bf);
+    float e = ex2(d);
     if (MODE == kBeta1) return e;
     e *= e;
     if (MODE == kBeta2) return e;
     e *= e;
     if (MODE == kBeta4) return e;
     return e * e;
+}
+// mass 2^{beta (x - C)} of one logit
+template <int MODE>
+__device__ __forceinline__ float logit_mass(float l, float neg_C, float bf) {
+    return mass_beta<MODE>(rel_exponent(l, neg_C), bf);
 }
 
 template <int DT>
@@ -62,9 +81,9 @@ struct FinishParams {
     int V;
     int64_t ld;
     int span, n_spans;
-    const float4* partials;  // [R][n_spans] = (m, s1, sb, -)
+    const float4* partials;  // [R][n_spans] = (c, s1, sb, -)
     double beta, alpha_t;
-    float cb;                // beta * log2(e)
+    float bf;                // (float)beta
     int vec;                 // rows are 16-byte aligned
 };
 
@@ -74,34 +93,44 @@ struct RowResult {
     double loginc; // log omega
 };
 
-// One warp finishes one row.  Every lane returns the same RowResult.
-template <int DT, int MODE>
-__device__ __forceinline__ RowResult finish_row(const FinishParams& p, int row, double U, int lane) {
-    RowResult bad{-1, 0.0, 0.0};
+// What one warp learns from a row's span triples.  Every lane holds the same values.
+struct RowTotals {
+    bool ok;        // false: NaN, +inf, or no finite logit
+    float C;        // the row's largest reference exponent
+    double S1, Sb;  // sum 2^{x - C}, sum 2^{beta (x - C)}
+    double target;  // U * Sb
+    double base;    // mass of the spans before span `jsel`
+    int jsel;       // span that holds the target
+};
+
+template <int MODE>
+__device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane) {
+    RowTotals t;
+    t.ok = false;
     const int n = p.n_spans;
     const float4* P = p.partials + (size_t)row * n;
-    const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
 
-    // row maximum
-    float mf = kNegBig;
-    for (int j = lane; j < n; j += 32) mf = fmaxf(mf, __ldcg(&P[j]).x);
-    mf = warp_max(mf);
-    const double M = (double)mf;
+    float cf = kRefFloor;
+    for (int j = lane; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
+    cf = warp_max(cf);
+    t.C = cf;
+    const double C = (double)cf;
 
-    // totals, every term rescaled to the row maximum in fp64
+    // totals, every term rescaled to the row's reference in fp64
     double a_sum = 0.0, b_sum = 0.0;
     for (int j = lane; j < n; j += 32) {
         const float4 f = __ldcg(&P[j]);
-        const double dm = (double)f.x - M;
-        const double a = (double)f.y * exp(dm);
+        const double dc = (double)f.x - C;
+        const double a = (double)f.y * exp2(dc);
         a_sum += a;
-        b_sum += (MODE == kBeta1) ? a : (double)f.z * exp(p.beta * dm);
+        b_sum += (MODE == kBeta1) ? a : (double)f.z * exp2(p.beta * dc);
     }
-    const double S1 = warp_sum(a_sum), Sb = warp_sum(b_sum);
-    if (!(S1 > 0.0) || !(Sb > 0.0) || isinf(S1) || isinf(Sb)) return bad;  // NaN, +inf, or nothing finite
+    t.S1 = warp_sum(a_sum);
+    t.Sb = warp_sum(b_sum);
+    if (!(t.S1 > 0.0) || !(t.Sb > 0.0) || isinf(t.S1) || isinf(t.Sb)) return t;
 
     // span that holds the target: inclusive prefix over spans in order, 32 spans per round
-    const double target = U * Sb;
+    t.target = U * t.Sb;
     double carry = 0.0, base = 0.0, last_base = 0.0;
     int jsel = -1, last_pos = -1;
     for (int c = 0; c < n && jsel < 0; c += 32) {
@@ -109,11 +138,11 @@ __device__ __forceinline__ RowResult finish_row(const FinishParams& p, int row, 
         double b = 0.0;
         if (j < n) {
             const float4 f = __ldcg(&P[j]);
-            const double dm = (double)f.x - M;
-            b = (MODE == kBeta1) ? (double)f.y * exp(dm) : (double)f.z * exp(p.beta * dm);
+            const double dc = (double)f.x - C;
+            b = (MODE == kBeta1) ? (double)f.y * exp2(dc) : (double)f.z * exp2(p.beta * dc);
         }
         const double incl = carry + warp_scan_incl(b, lane);
-        const unsigned hit = __ballot_sync(kFull, b > 0.0 && incl >= target);
+        const unsigned hit = __ballot_sync(kFull, b > 0.0 && incl >= t.target);
         const unsigned pos = __ballot_sync(kFull, b > 0.0);
         if (hit) {
             const int src = __ffs(hit) - 1;
@@ -130,67 +159,97 @@ __device__ __forceinline__ RowResult finish_row(const FinishParams& p, int row, 
         jsel = last_pos;
         base = last_base;
     }
-    if (jsel < 0) return bad;
+    if (jsel < 0) return t;
+    t.jsel = jsel;
+    t.base = base;
+    t.ok = true;
+    return t;
+}
 
-    // re-read that span in vocabulary order: lane owns `sub` consecutive logits
-    const int a0 = jsel * p.span, b0 = min(p.V, a0 + p.span);
-    const int sub = p.span >> 5;
-    const int e0 = a0 + lane * sub;
-    float lane_mass = 0.f;
-    int lane_last = -1;
-    if (DT == PSMC_BF16 && p.vec && e0 + sub <= b0) {
-        const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(rowp) + e0);
-        for (int k = 0; k < (sub >> 3); k += 2) {  // sub is a multiple of 16 (span >= 512)
-            const uint4 v0 = q[k], v1 = q[k + 1];
-            const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-            float g = 0.f;
+// One lane's share of the selected span: `E` consecutive logits from e0 (clipped to b0).  Returns their mass
+// (eight logits summed in fp32 at a time, then in fp64) and the last position with mass (-1 if none).
+template <int DT, int MODE>
+__device__ __forceinline__ double lane_share(const FinishParams& p, const void* rowp, int e0, int E, int b0, float neg_C,
+                                            int& lane_last) {
+    constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;  // logits per 16 bytes
+    double lm = 0.0;
+    lane_last = -1;
+    if (e0 >= b0) return lm;
+    if (p.vec && e0 + E <= b0) {
+        const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)e0 * (16 / kPer));
+        const int Q = E / kPer;
+        for (int q0 = 0; q0 < Q; q0 += 4) {  // four loads in flight
+            uint4 v[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float m0 = mass_beta<MODE>(__uint_as_float(w[i] << 16) - mf, p.cb);
-                const float m1 = mass_beta<MODE>(__uint_as_float(w[i] & 0xffff0000u) - mf, p.cb);
-                if (m0 > 0.f) lane_last = e0 + (k << 3) + 2 * i;
-                if (m1 > 0.f) lane_last = e0 + (k << 3) + 2 * i + 1;
-                g += m0 + m1;
+            for (int i = 0; i < 4; ++i)
+                if (q0 + i < Q) v[i] = q[q0 + i];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (q0 + i >= Q) break;
+                const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                const int at = e0 + (q0 + i) * kPer;
+                float g[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (DT == PSMC_BF16) {
+                        const float m0 = logit_mass<MODE>(__uint_as_float(w[j] << 16), neg_C, p.bf);
+                        const float m1 = logit_mass<MODE>(__uint_as_float(w[j] & 0xffff0000u), neg_C, p.bf);
+                        if (m0 > 0.f) lane_last = at + 2 * j;
+                        if (m1 > 0.f) lane_last = at + 2 * j + 1;
+                        g[j] = m0 + m1;
+                    } else {
+                        g[j] = logit_mass<MODE>(__uint_as_float(w[j]), neg_C, p.bf);
+                        if (g[j] > 0.f) lane_last = at + j;
+                    }
+                }
+                lm += (double)((g[0] + g[1]) + (g[2] + g[3]));
             }
-            lane_mass += g;
         }
     } else {
-        const int e1 = min(b0, e0 + sub);
+        const int e1 = min(b0, e0 + E);
         for (int i = e0; i < e1; ++i) {
-            const float e = mass_beta<MODE>(load_elem<DT>(rowp, i) - mf, p.cb);
+            const float e = logit_mass<MODE>(load_elem<DT>(rowp, i), neg_C, p.bf);
             if (e > 0.f) lane_last = i;
-            lane_mass += e;
+            lm += (double)e;
         }
     }
-    const double lm = (double)lane_mass;
-    const double r_incl = base + warp_scan_incl(lm, lane);
-    const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= target);
-    int y = -1;
-    if (hit2) {
-        // the owner's `sub` logits, 32 at a time across the warp, in order
-        const int owner = __ffs(hit2) - 1;
-        double run = __shfl_sync(kFull, r_incl - lm, owner);
-        const int o0 = a0 + owner * sub, o1 = min(b0, o0 + sub);
-        int last_in_owner = -1;
-        for (int c = o0; c < o1 && y < 0; c += 32) {
-            const int i = c + lane;
-            const float e = i < o1 ? mass_beta<MODE>(load_elem<DT>(rowp, i) - mf, p.cb) : 0.f;
+    return lm;
+}
+
+// Token inside the owner lane's logits [o0, o1): 32 at a time across the warp, in vocabulary order, the loads of
+// up to four rounds issued together.  `run` is the mass before o0.  Returns -1 only if nothing there has mass.
+template <int DT, int MODE>
+__device__ __forceinline__ int locate_in_lane(const FinishParams& p, const void* rowp, int o0, int o1, double run,
+                                              double target, float neg_C, int lane) {
+    int y = -1, last_with_mass = -1;
+    for (int c0 = o0; c0 < o1 && y < 0; c0 += 128) {
+        float l[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int i = c0 + 32 * b + lane;
+            l[b] = i < o1 ? load_elem<DT>(rowp, i) : -INFINITY;
+        }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if (c0 + 32 * b >= o1 || y >= 0) break;
+            const float e = logit_mass<MODE>(l[b], neg_C, p.bf);  // -inf gives mass 0
             const double incl = run + warp_scan_incl((double)e, lane);
             const unsigned h3 = __ballot_sync(kFull, e > 0.f && incl >= target);
             const unsigned p3 = __ballot_sync(kFull, e > 0.f);
-            if (h3) y = c + __ffs(h3) - 1;
-            else if (p3) last_in_owner = c + 31 - __clz(p3);
+            if (h3) y = c0 + 32 * b + __ffs(h3) - 1;
+            else if (p3) last_with_mass = c0 + 32 * b + 31 - __clz(p3);
             run = __shfl_sync(kFull, incl, 31);
         }
-        if (y < 0) y = last_in_owner;  // the finer sums fell a rounding error short
-    } else {
-        y = warp_max(lane_last);       // the re-read sums fall short of the target: last token with mass
     }
-    if (y < 0) return bad;
+    return y >= 0 ? y : last_with_mass;  // the finer sums may fall a rounding error short of the lane's total
+}
 
+template <int DT>
+__device__ __forceinline__ RowResult row_result(const FinishParams& p, const void* rowp, const RowTotals& t, int y) {
     RowResult r;
-    const double dl = (double)load_elem<DT>(rowp, y) - M;
-    const double ln_s1 = log(S1), ln_sb = log(Sb);
+    // l_y - C ln 2: the token's logit relative to the row's reference, in natural units
+    const double dl = (double)load_elem<DT>(rowp, y) - (double)t.C * kLn2;
+    const double ln_s1 = log(t.S1), ln_sb = log(t.Sb);
     r.tok = y;
     r.logp = dl - ln_s1;  // log p(y) = l_y - L1
     // alpha_t log p(y) - log q(y), log q(y) = beta l_y - Lb, grouped so that the token's own logit drops out
@@ -199,15 +258,89 @@ __device__ __forceinline__ RowResult finish_row(const FinishParams& p, int row, 
     return r;
 }
 
-// run-time dispatch of finish_row over the beta mode (the dtype stays a template parameter of the caller)
-template <int DT>
-__device__ __forceinline__ RowResult finish_row_mode(int mode, const FinishParams& p, int row, double U, int lane) {
-    switch (mode) {
-        case kBeta1: return finish_row<DT, kBeta1>(p, row, U, lane);
-        case kBeta2: return finish_row<DT, kBeta2>(p, row, U, lane);
-        case kBeta4: return finish_row<DT, kBeta4>(p, row, U, lane);
-        case kBeta8: return finish_row<DT, kBeta8>(p, row, U, lane);
-        default: return finish_row<DT, kBetaAny>(p, row, U, lane);
+// ---- the finish at CTA level: several warps share a row ----
+constexpr int kFinishMaxWarps = 32;
+struct FinishShared {
+    double tot[kFinishMaxWarps];  // mass of the part of the selected span each warp re-read
+    int last[kFinishMaxWarps];    // last position with mass in that part (-1 if none)
+};
+
+// warps per row: as many as the CTA can spare, each part of the span at least 256 logits (8 per lane)
+__host__ __device__ inline int finish_warps_per_row(int n_rows, int span, int n_warps) {
+    int w = 1;
+    while (w * 2 * n_rows <= n_warps && w * 2 <= 8 && span / (w * 2) >= 256) w *= 2;
+    return w;
+}
+
+// Every thread of the CTA calls this (it synchronises the CTA).  Finishes rows row0 .. row0+n_rows-1, `wpr` warps
+// (a power of two) per row, n_warps/wpr rows at a time.  live(k): does row k need finishing; uniform(k): its U;
+// emit(k, result) is called by lane 0 of one warp per finished row.
+template <int DT, int MODE, class LiveFn, class UniformFn, class EmitFn>
+__device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared& sh, int row0, int n_rows, int wpr,
+                                            LiveFn live, UniformFn uniform, EmitFn emit) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int rows_per_pass = n_warps / wpr;
+    const int q = warp & (wpr - 1);
+    for (int k0 = 0; k0 < n_rows; k0 += rows_per_pass) {
+        const int k = k0 + warp / wpr;
+        const bool active = warp < rows_per_pass * wpr && k < n_rows && live(k);
+        const int row = row0 + k;
+        const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
+        RowTotals t;
+        t.ok = false;
+        double lm = 0.0, incl = 0.0;
+        int a0 = 0, b0 = 0, E = 0, sub = 0;
+        float neg_C = 0.f;
+        if (active) {
+            t = combine_spans<MODE>(p, row, uniform(k), lane);
+            int wl = -1;
+            if (t.ok) {
+                neg_C = -t.C;
+                a0 = t.jsel * p.span;
+                b0 = min(p.V, a0 + p.span);
+                sub = p.span / wpr;
+                E = sub >> 5;
+                int lane_last;
+                lm = lane_share<DT, MODE>(p, rowp, a0 + q * sub + lane * E, E, b0, neg_C, lane_last);
+                incl = warp_scan_incl(lm, lane);
+                wl = warp_max(lane_last);
+            }
+            if (lane == 31) sh.tot[warp] = incl;
+            if (lane == 0) sh.last[warp] = wl;
+        }
+        __syncthreads();
+        if (active) {
+            const int w0 = warp - q;  // first warp of this row
+            if (!t.ok) {
+                if (q == 0 && lane == 0) emit(k, RowResult{-1, 0.0, 0.0});
+            } else {
+                // which part of the span reaches the target: same additions, in the same order, in every warp
+                double cum = t.base, before = t.base;
+                int first_hit = -1;
+                for (int i = 0; i < wpr; ++i) {
+                    if (i == q) before = cum;
+                    const double ti = sh.tot[w0 + i];
+                    cum += ti;
+                    if (first_hit < 0 && ti > 0.0 && cum >= t.target) first_hit = i;
+                }
+                int y = -1;
+                bool mine = false;
+                if (first_hit == q) {
+                    mine = true;
+                    const double r_incl = before + incl;
+                    const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+                    const int owner = hit2 ? __ffs(hit2) - 1 : 31;
+                    const double run = __shfl_sync(kFull, r_incl - lm, owner);
+                    const int o0 = a0 + q * sub + owner * E;
+                    y = locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+                } else if (first_hit < 0 && q == 0) {
+                    mine = true;  // the re-read sums fall short of the target: last token with mass in the span
+                    for (int i = 0; i < wpr; ++i) y = max(y, sh.last[w0 + i]);
+                }
+                if (mine && lane == 0) emit(k, y >= 0 ? row_result<DT>(p, rowp, t, y) : RowResult{-1, 0.0, 0.0});
+            }
+        }
+        __syncthreads();  // sh is reused by the next pass
     }
 }
 

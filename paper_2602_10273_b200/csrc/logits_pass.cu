@@ -1,147 +1,214 @@
 // Streaming half of the logit pass: ONE sweep over the [R, V] logits, HBM-bound.
 //
-// A row is cut into spans of `span` consecutive logits; one warp streams one span with 128-bit
-// loads (8 bf16 / 4 fp32 per lane per load, up to eight loads in flight per lane) and keeps, per
-// lane, a running maximum m and the sums  s1 = sum exp(l - m),  sb = sum exp(beta (l - m)).
-// One MUFU.EX2 per logit: for beta in {1,2,4,8} exp(beta d) is exp(d) squared up; other beta
-// (exponent-bridging steps, Section 4.3) pay a second EX2.  The warp reduces its lanes to one
-// (m, s1, sb) triple and stores it; nothing else leaves the kernel.  No atomics, no fences, no waits:
-// spans are dealt round-robin to a grid that exactly fills the machine, so every warp does the same
-// amount of work.  The per-row finish (logits_common.cuh) runs in the kernel that follows.
+// A row is cut into spans of `span` consecutive logits; one warp sums one span and stores one (c, s1, sb)
+// triple for it (logits_common.cuh); nothing else leaves the kernel.  The per-row finish runs in the kernel
+// that follows.
+//
+// Data movement: one persistent CTA per SM, up to 16 warps, each warp with a private ring of kDepth stages of
+// kStageBytes in shared memory.  Lane 0 of a warp keeps kDepth-1 bulk asynchronous copies (TMA, untiled,
+// completion on an mbarrier) in flight for the pieces the warp will need next -- across span boundaries, so
+// the memory pipe never drains -- while the warp sums the piece that has landed, reading it back with
+// conflict-free 128-bit shared loads.  About 128 KB per SM are in flight at any time, independent of how the
+// warps are scheduled.  No cross-warp synchronisation, no atomics; every mbarrier wait is bounded.
+//
+// Arithmetic per pair of logits: two unpack operations, two packed fp32x2 FMAs for x - c, two MUFU.EX2, one
+// packed add for s1 and, for beta in {2,4,8}, one to three packed multiply/FMA for sb (2^{beta d} is 2^d
+// squared up); other beta (exponent-bridging steps, Section 4.3) pay a second EX2 per logit.  The reference
+// exponent c is common to the lanes of a warp and is carried from span to span inside a row.  It follows the
+// largest logit the warp has seen with a slack of kRefSlack: it moves (a warp-uniform, rare path) only when some
+// logit exceeds it by more than that, which keeps |x - c| of the dominant terms small -- the fp32 rounding of
+// x - c is what limits their accuracy -- without rescaling the sums at every load.
 #include <mutex>
 
+#include "bulk_copy.cuh"
 #include "internal.h"
 #include "logits_common.cuh"
 
 namespace psmc {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarpsPerCta = kThreads / 32;
-constexpr int kCtasPerSm = 3;
+constexpr int kMaxWarps = 16;        // warps per CTA of the streaming kernel
+constexpr int kStageBytes = 4096;    // one bulk copy
+constexpr int kDepth = 3;            // stages per warp: one being summed, two in flight
+constexpr float kRefSlack = 2.0f;    // natural units a logit may exceed the warp's reference point by (less for beta > 31)
 
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+// ---- packed pairs of fp32 in one 64-bit register (fp32x2 instructions of sm_100) ----
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float2 unpack2(f32x2 v) {
+    float2 r;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// 2^x on both halves
+__device__ __forceinline__ f32x2 ex2_2(f32x2 x) {
+    f32x2 r;
+    asm("{\n\t.reg .f32 lo, hi;\n\t"
+        "mov.b64 {lo, hi}, %1;\n\t"
+        "ex2.approx.ftz.f32 lo, lo;\n\t"
+        "ex2.approx.ftz.f32 hi, hi;\n\t"
+        "mov.b64 %0, {lo, hi};\n\t}"
+        : "=l"(r)
+        : "l"(x));
+    return r;
+}
+// the two bf16 of a word, widened to fp32: low half in the low lane
+__device__ __forceinline__ f32x2 widen_bf16x2(uint32_t w) {
+    return ((f32x2)(w & 0xffff0000u) << 32) | (f32x2)(w << 16);
 }
 
+// Per-lane running state.  Two accumulators per sum (a, b) shorten the dependent chains; each holds a packed pair.
 struct LaneSums {
-    float m, s1, sb;
+    float thr;    // logits above this move the reference exponent (the same in every lane of the warp)
+    float neg_c;  // minus the reference exponent in use (the same in every lane of the warp)
+    f32x2 s1a, s1b, sba, sbb;
 };
+__device__ __forceinline__ LaneSums lane_sums_init() {
+    LaneSums a;
+    a.thr = kNegBig;
+    a.neg_c = -kRefFloor;
+    a.s1a = a.s1b = a.sba = a.sbb = 0ull;
+    return a;
+}
+__device__ __forceinline__ float pair_sum(f32x2 v) {
+    const float2 f = unpack2(v);
+    return f.x + f.y;
+}
+__device__ __forceinline__ f32x2 pair_scale(f32x2 v, float f) { return mul2(v, pack2(f, f)); }
 
-// one logit into the two running sums; d = l - m
+// The packed operations take no immediates; the constants they need live in registers for the whole kernel.
+struct PackedConsts {
+    f32x2 k_hi, k_lo, bf;
+    float bf1;
+    float slack;  // min(kRefSlack, 62 / beta): keeps 2^{beta slack log2 e} below 2^90
+};
+__device__ __forceinline__ PackedConsts packed_consts(float bf) {
+    PackedConsts k;
+    k.k_hi = pack2(kLog2eHi, kLog2eHi);
+    k.k_lo = pack2(kLog2eLo, kLog2eLo);
+    k.bf = pack2(bf, bf);
+    k.bf1 = bf;
+    k.slack = fminf(kRefSlack, 62.f / fmaxf(bf, 1.f));
+    // hide the values from constant propagation so that they are not rebuilt at every use
+    asm volatile("" : "+l"(k.k_hi), "+l"(k.k_lo), "+l"(k.bf));
+    return k;
+}
+__device__ __forceinline__ f32x2 rel_exponent2(f32x2 l, f32x2 neg_c, const PackedConsts& k) {
+    return fma2(l, k.k_lo, fma2(l, k.k_hi, neg_c));
+}
+// two logits, already as exponents d = x - c, into one accumulator pair
 template <int MODE>
-__device__ __forceinline__ void accumulate(float d, float cb, float& s1, float& sb) {
-    const float e = ex2(d * kLog2e);
-    s1 += e;
+__device__ __forceinline__ void add_pair(f32x2 d, const PackedConsts& k, f32x2& s1, f32x2& sb) {
+    const f32x2 e = ex2_2(d);
+    s1 = add2(s1, e);
     if (MODE == kBeta2) {
-        sb = fmaf(e, e, sb);
+        sb = fma2(e, e, sb);
     } else if (MODE == kBeta4) {
-        const float e2 = e * e;
-        sb = fmaf(e2, e2, sb);
+        const f32x2 e2 = mul2(e, e);
+        sb = fma2(e2, e2, sb);
     } else if (MODE == kBeta8) {
-        const float e2 = e * e;
-        const float e4 = e2 * e2;
-        sb = fmaf(e4, e4, sb);
+        const f32x2 e2 = mul2(e, e);
+        const f32x2 e4 = mul2(e2, e2);
+        sb = fma2(e4, e4, sb);
     } else if (MODE == kBetaAny) {
-        sb += ex2(d * cb);
+        sb = add2(sb, ex2_2(mul2(d, k.bf)));
     }
 }
+// Some lane met a logit above the threshold; cm is this lane's largest candidate.  The warp moves its reference
+// exponent to the largest of them and shrinks the sums accordingly.  Called by all 32 lanes together.
+// Logits up to the new maximum + slack then pass without another move: a term stays below
+// 2^{beta slack log2 e} <= 2^90 and whatever underflows is smaller than 2^-126 against a largest term of about 1.
 template <int MODE>
-__device__ __forceinline__ void raise_max(float cm, float cb, LaneSums& a) {
-    if (cm > a.m) {
-        const float d0 = a.m - cm;  // <= 0; hugely negative on the first call, which zeroes the (empty) sums
-        a.s1 *= ex2(d0 * kLog2e);
-        if (MODE != kBeta1) a.sb *= mass_beta<MODE>(d0, cb);
-        a.m = cm;
+__device__ __forceinline__ void move_reference(float cm, float bf, float slack, LaneSums& a) {
+    cm = warp_max(cm);
+    const float new_neg_c = -ref_exponent(cm);
+    const float d0 = new_neg_c - a.neg_c;  // c_old - c_new < 0; hugely negative the first time, when the sums are empty
+    const float f1 = ex2(d0);
+    a.s1a = pair_scale(a.s1a, f1);
+    a.s1b = pair_scale(a.s1b, f1);
+    if (MODE != kBeta1) {
+        const float fb = mass_beta<MODE>(d0, bf);
+        a.sba = pair_scale(a.sba, fb);
+        a.sbb = pair_scale(a.sbb, fb);
     }
+    a.thr = cm + slack;
+    a.neg_c = new_neg_c;
+}
+// one logit per lane (ragged ends, unaligned rows); all 32 lanes call it, lanes without a logit pass -inf
+template <int MODE>
+__device__ __forceinline__ void add_one(float l, float bf, float slack, LaneSums& a) {
+    if (__any_sync(kFull, l > a.thr)) move_reference<MODE>(l, bf, slack, a);
+    const float d = rel_exponent(l, a.neg_c);  // -inf for a lane without a logit: mass 0
+    a.s1a = add2(a.s1a, pack2(ex2(d), 0.f));
+    if (MODE != kBeta1) a.sba = add2(a.sba, pack2(mass_beta<MODE>(d, bf), 0.f));
 }
 
 // ---- bf16: NW 32-bit words = 2*NW logits ----
 template <int MODE, int NW>
-__device__ __forceinline__ void consume_bf16(const uint32_t (&w)[NW], float cb, LaneSums& a, __nv_bfloat162& m2) {
+__device__ __forceinline__ void consume_bf16(const uint32_t (&w)[NW], const PackedConsts& k, LaneSums& a,
+                                             __nv_bfloat162& thr2) {
     __nv_bfloat162 pm = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
 #pragma unroll
     for (int i = 1; i < NW; ++i) pm = __hmax2(pm, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
-    if (!__hble2(pm, m2)) {  // some logit exceeds the running maximum (rare after the first loads)
-        raise_max<MODE>(fmaxf(__low2float(pm), __high2float(pm)), cb, a);
-        m2 = __float2bfloat162_rn(a.m);  // exact: m is itself a bf16 value
+    if (__any_sync(kFull, !__hble2(pm, thr2))) {  // some logit of the warp is above the threshold
+        move_reference<MODE>(fmaxf(__low2float(pm), __high2float(pm)), k.bf1, k.slack, a);
+        thr2 = __float2bfloat162_rn(a.thr);
     }
+    const f32x2 nc = pack2(a.neg_c, a.neg_c);
 #pragma unroll
     for (int i = 0; i < NW; ++i) {
-        accumulate<MODE>(__uint_as_float(w[i] << 16) - a.m, cb, a.s1, a.sb);
-        accumulate<MODE>(__uint_as_float(w[i] & 0xffff0000u) - a.m, cb, a.s1, a.sb);
+        const f32x2 d = rel_exponent2(widen_bf16x2(w[i]), nc, k);
+        if (i & 1) add_pair<MODE>(d, k, a.s1b, a.sbb);
+        else add_pair<MODE>(d, k, a.s1a, a.sba);
     }
 }
-// ---- fp32: NW words = NW logits ----
+// ---- fp32: NW words = NW logits (NW even) ----
 template <int MODE, int NW>
-__device__ __forceinline__ void consume_f32(const uint32_t (&w)[NW], float cb, LaneSums& a) {
+__device__ __forceinline__ void consume_f32(const uint32_t (&w)[NW], const PackedConsts& k, LaneSums& a) {
     float cm = __uint_as_float(w[0]);
 #pragma unroll
     for (int i = 1; i < NW; ++i) cm = fmaxf(cm, __uint_as_float(w[i]));
-    raise_max<MODE>(cm, cb, a);
+    if (__any_sync(kFull, cm > a.thr)) move_reference<MODE>(cm, k.bf1, k.slack, a);
+    const f32x2 nc = pack2(a.neg_c, a.neg_c);
 #pragma unroll
-    for (int i = 0; i < NW; ++i) accumulate<MODE>(__uint_as_float(w[i]) - a.m, cb, a.s1, a.sb);
+    for (int i = 0; i < NW; i += 2) {
+        const f32x2 d = rel_exponent2(((f32x2)w[i + 1] << 32) | (f32x2)w[i], nc, k);
+        if (i & 2) add_pair<MODE>(d, k, a.s1b, a.sbb);
+        else add_pair<MODE>(d, k, a.s1a, a.sba);
+    }
 }
 template <int DT, int MODE, int NW>
-__device__ __forceinline__ void consume(const uint32_t (&w)[NW], float cb, LaneSums& a, __nv_bfloat162& m2) {
-    if (DT == PSMC_BF16) consume_bf16<MODE, NW>(w, cb, a, m2);
-    else consume_f32<MODE, NW>(w, cb, a);
-}
-
-// 16-byte aligned span [a0, b0) of a row: chunks of 16 bytes, lane-strided
-template <int DT, int MODE>
-__device__ __forceinline__ void span_vec(const void* rowp, int a0, int b0, float cb, int lane, LaneSums& acc) {
-    constexpr int kPerChunk = DT == PSMC_BF16 ? 8 : 4;
-    constexpr int kShift = DT == PSMC_BF16 ? 3 : 2;
-    const int n = b0 - a0, n_chunks = n >> kShift;
-    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)a0 * (16 / kPerChunk));
-    __nv_bfloat162 m2 = __float2bfloat162_rn(acc.m);
-    int c = lane;
-    for (; c + 224 < n_chunks; c += 256) {  // eight loads in flight per lane
-        uint4 v[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = ld_stream16(p + c + 32 * i);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t w[16] = {v[4 * h].x,     v[4 * h].y,     v[4 * h].z,     v[4 * h].w,
-                                    v[4 * h + 1].x, v[4 * h + 1].y, v[4 * h + 1].z, v[4 * h + 1].w,
-                                    v[4 * h + 2].x, v[4 * h + 2].y, v[4 * h + 2].z, v[4 * h + 2].w,
-                                    v[4 * h + 3].x, v[4 * h + 3].y, v[4 * h + 3].z, v[4 * h + 3].w};
-            consume<DT, MODE, 16>(w, cb, acc, m2);
-        }
-    }
-    for (; c + 96 < n_chunks; c += 128) {
-        const uint4 v0 = ld_stream16(p + c), v1 = ld_stream16(p + c + 32), v2 = ld_stream16(p + c + 64),
-                    v3 = ld_stream16(p + c + 96);
-        const uint32_t w[16] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w,
-                                v2.x, v2.y, v2.z, v2.w, v3.x, v3.y, v3.z, v3.w};
-        consume<DT, MODE, 16>(w, cb, acc, m2);
-    }
-    for (; c < n_chunks; c += 32) {
-        const uint4 v0 = ld_stream16(p + c);
-        const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
-        consume<DT, MODE, 4>(w, cb, acc, m2);
-    }
-    const int tail = n & (kPerChunk - 1);  // ragged end of the row
-    if (lane < tail) {
-        const float x = load_elem<DT>(rowp, (int64_t)a0 + (n_chunks << kShift) + lane);
-        raise_max<MODE>(x, cb, acc);
-        accumulate<MODE>(x - acc.m, cb, acc.s1, acc.sb);
-    }
+__device__ __forceinline__ void consume(const uint32_t (&w)[NW], const PackedConsts& k, LaneSums& a,
+                                        __nv_bfloat162& thr2) {
+    if (DT == PSMC_BF16) consume_bf16<MODE, NW>(w, k, a, thr2);
+    else consume_f32<MODE, NW>(w, k, a);
 }
 
 // any alignment: one logit per lane per load
 template <int DT, int MODE>
-__device__ __forceinline__ void span_scalar(const void* rowp, int a0, int b0, float cb, int lane, LaneSums& acc) {
-    for (int i = a0 + lane; i < b0; i += 32) {
-        const float x = load_elem<DT>(rowp, i);
-        raise_max<MODE>(x, cb, acc);
-        accumulate<MODE>(x - acc.m, cb, acc.s1, acc.sb);
-    }
+__device__ __forceinline__ void span_scalar(const void* rowp, int a0, int b0, const PackedConsts& k, int lane,
+                                            LaneSums& acc) {
+    for (int i0 = a0; i0 < b0; i0 += 32)  // the same trip count in every lane
+        add_one<MODE>(i0 + lane < b0 ? load_elem<DT>(rowp, i0 + lane) : -INFINITY, k.bf1, k.slack, acc);
 }
 
 struct StreamParams {
@@ -149,42 +216,220 @@ struct StreamParams {
     int R, V;
     int64_t ld;
     int span, n_spans;
-    float cb;
+    float bf;     // (float)beta
     const uint8_t* done;
     float4* partials;
     int32_t* zero_words;
+    int32_t* status;  // may be NULL
 };
 
-template <int DT, int MODE, bool VEC>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) logits_stream_kernel(const StreamParams p) {
-    const int lane = threadIdx.x & 31;
-    const int warp_global = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const int n_warps = gridDim.x * kWarpsPerCta;
+// one (row, span) task as the streaming loop sees it
+struct TaskDesc {
+    int row, sp;
+    int bytes16;        // bytes of the span that bulk copies can fetch (a multiple of 16)
+    int tail;           // ragged logits after them (only a row's last span can have any)
+    const char* base;   // first byte of the span
+};
+// Walks the tasks first, first+1, ... in (row, span) order without dividing at every step.
+template <int DT>
+struct TaskWalker {
+    int task, end, row, sp;
+    __device__ __forceinline__ void start(const StreamParams& p, int first, int last) {
+        task = first;
+        end = last;
+        row = first / p.n_spans;
+        sp = first - row * p.n_spans;
+    }
+    __device__ __forceinline__ bool at_end() const { return task >= end; }
+    __device__ __forceinline__ void next(const StreamParams& p) {
+        ++task;
+        if (++sp == p.n_spans) {
+            sp = 0;
+            ++row;
+        }
+    }
+    // false: the row is finished and its logits are not to be read (absorbing state)
+    __device__ __forceinline__ bool describe(const StreamParams& p, TaskDesc& d) const {
+        constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;  // logits per 16 bytes
+        if (p.done && p.done[row]) return false;
+        d.row = row;
+        d.sp = sp;
+        const int a0 = sp * p.span;
+        const int n = min(p.V, a0 + p.span) - a0;
+        d.bytes16 = (n / kPer) * 16;
+        d.tail = n % kPer;
+        d.base = reinterpret_cast<const char*>(p.logits) + ((size_t)row * p.ld + a0) * (16 / kPer);
+        return true;
+    }
+};
+
+// one triple per span: the lanes share the reference exponent, so their sums add up as they are
+template <int MODE>
+__device__ __forceinline__ void store_triple(const StreamParams& p, int row, int sp, const LaneSums& acc, int lane) {
+    const float s1 = warp_sum(pair_sum(add2(acc.s1a, acc.s1b)));
+    const float sb = (MODE == kBeta1) ? 0.f : warp_sum(pair_sum(add2(acc.sba, acc.sbb)));
+    if (lane == 0) __stcg(&p.partials[(size_t)row * p.n_spans + sp], make_float4(-acc.neg_c, s1, sb, 0.f));
+}
+
+// Rows that start on 16-byte boundaries: the bulk-copy pipeline described at the top of the file.  Each warp owns
+// a contiguous run of tasks, so it mostly stays inside one row and its copies walk forward through memory.
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1) logits_stream_kernel(const __grid_constant__ StreamParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bars[kMaxWarps * kDepth];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps_per_cta = blockDim.x >> 5;
+    const int warp_global = blockIdx.x * warps_per_cta + warp;
+    const int n_warps = gridDim.x * warps_per_cta;
+    const int n_tasks = p.R * p.n_spans;  // < 2^31, checked by the host
+    const int per_warp = (n_tasks + n_warps - 1) / n_warps;
+    const int first = min(n_tasks, warp_global * per_warp), last = min(n_tasks, first + per_warp);
     if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
 
-    const int64_t n_tasks = (int64_t)p.R * p.n_spans;
-    for (int64_t task = warp_global; task < n_tasks; task += n_warps) {
-        const int row = (int)(task / p.n_spans), sp = (int)(task - (int64_t)row * p.n_spans);
-        if (p.done && p.done[row]) continue;  // absorbing state: the row's logits are never read
-        const int a0 = sp * p.span, b0 = min(p.V, a0 + p.span);
-        const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
+    const PackedConsts kc = packed_consts(p.bf);
+    unsigned char* ring = smem + (size_t)warp * kDepth * kStageBytes;
+    uint64_t* full = bars + warp * kDepth;
+    if (lane == 0) {
+        for (int d = 0; d < kDepth; ++d) mbar_init(&full[d], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    __syncwarp();
 
-        LaneSums acc{kNegBig, 0.f, 0.f};
-        if (VEC) span_vec<DT, MODE>(rowp, a0, b0, p.cb, lane, acc);
-        else span_scalar<DT, MODE>(rowp, a0, b0, p.cb, lane, acc);
+    // producer cursor (the same in every lane; lane 0 issues): the next piece to fetch
+    TaskWalker<DT> pw;
+    pw.start(p, first, last);
+    const char* p_src = nullptr;
+    int p_left = 0;
+    auto prod_seek = [&]() {
+        for (; !pw.at_end(); pw.next(p)) {
+            TaskDesc d;
+            if (pw.describe(p, d) && d.bytes16 > 0) {
+                p_src = d.base;
+                p_left = d.bytes16;
+                return;
+            }
+        }
+    };
+    int issued = 0;
+    auto issue = [&]() {  // next piece into stage issued % kDepth
+        if (pw.at_end()) return;
+        const int bytes = p_left < kStageBytes ? p_left : kStageBytes;
+        if (lane == 0) {
+            const int slot = issued % kDepth;
+            fence_async_smem();  // the stage's previous contents were read through the generic proxy
+            mbar_expect_tx(&full[slot], (uint32_t)bytes);
+            bulk_load(ring + (size_t)slot * kStageBytes, p_src, (uint32_t)bytes, &full[slot]);
+        }
+        ++issued;
+        p_src += bytes;
+        p_left -= bytes;
+        if (p_left == 0) {
+            pw.next(p);
+            prod_seek();
+        }
+    };
 
-        // one triple per span: rescale every lane to the warp's maximum, then add
-        const float wm = warp_max(acc.m);
-        const float d0 = acc.m - wm;
-        float s1 = acc.s1 * ex2(d0 * kLog2e);
-        float sb = (MODE == kBeta1) ? 0.f : acc.sb * mass_beta<MODE>(d0, p.cb);
-        s1 = warp_sum(s1);
-        sb = warp_sum(sb);
-        if (lane == 0) __stcg(&p.partials[(size_t)row * p.n_spans + sp], make_float4(wm, s1, sb, 0.f));
+    // consumer cursor: the task being summed
+    TaskWalker<DT> cw;
+    cw.start(p, first, last);
+    int c_left = 0, c_row = -1;
+    TaskDesc c_d = {};
+    LaneSums acc = lane_sums_init();
+    __nv_bfloat162 thr2 = __float2bfloat162_rn(acc.thr);
+    auto finish_task = [&]() {
+        if (c_d.tail > 0)  // ragged end of the row
+            add_one<MODE>(lane < c_d.tail ? load_elem<DT>(c_d.base + c_d.bytes16, lane) : -INFINITY, kc.bf1, kc.slack, acc);
+        store_triple<MODE>(p, c_d.row, c_d.sp, acc, lane);
+    };
+    auto cons_seek = [&]() {  // next live task; tasks without a whole 16-byte chunk are done on the spot
+        for (; !cw.at_end(); cw.next(p)) {
+            if (cw.describe(p, c_d)) {
+                if (c_d.row != c_row) {  // a new row: forget the reference point of the old one
+                    acc = lane_sums_init();
+                    thr2 = __float2bfloat162_rn(acc.thr);
+                    c_row = c_d.row;
+                } else {                 // same row: keep the reference point, start new sums
+                    acc.s1a = acc.s1b = acc.sba = acc.sbb = 0ull;
+                }
+                c_left = c_d.bytes16;
+                if (c_left > 0) return;
+                finish_task();
+            }
+        }
+    };
+
+    prod_seek();
+    cons_seek();
+    for (int d = 0; d < kDepth - 1; ++d) issue();
+
+    bool failed = false;
+    int consumed = 0;
+    while (!cw.at_end()) {
+        __syncwarp();  // every lane is done with the stage that is about to be refilled
+        issue();
+        const int slot = consumed % kDepth;
+        if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // uniform verdict
+            failed = true;
+            break;
+        }
+        const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
+        const int bytes = c_left < kStageBytes ? c_left : kStageBytes;
+        if (bytes == kStageBytes) {
+#pragma unroll
+            for (int h = 0; h < kStageBytes / 2048; ++h) {  // 2 KB = four 16-byte chunks per lane at a time
+                const uint4 v0 = st[h * 128 + lane], v1 = st[h * 128 + 32 + lane], v2 = st[h * 128 + 64 + lane],
+                            v3 = st[h * 128 + 96 + lane];
+                const uint32_t w[16] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w,
+                                        v2.x, v2.y, v2.z, v2.w, v3.x, v3.y, v3.z, v3.w};
+                consume<DT, MODE, 16>(w, kc, acc, thr2);
+            }
+        } else {
+            constexpr uint32_t kNoLogit = DT == PSMC_BF16 ? 0xff80ff80u : 0xff800000u;  // -inf: no mass, never a maximum
+            for (int c0 = 0; c0 < (bytes >> 4); c0 += 32) {  // the same trip count in every lane
+                const bool in = c0 + lane < (bytes >> 4);
+                const uint4 v0 = in ? st[c0 + lane] : make_uint4(kNoLogit, kNoLogit, kNoLogit, kNoLogit);
+                const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+                consume<DT, MODE, 4>(w, kc, acc, thr2);
+            }
+        }
+        ++consumed;
+        c_left -= bytes;
+        if (c_left == 0) {
+            finish_task();
+            cw.next(p);
+            cons_seek();
+        }
+    }
+    if (failed) {
+        if (lane == 0) raise_status(p.status, PSMC_E_TIMEOUT);
+        // do not leave with copies still landing in this CTA's shared memory: bounded second wait
+        for (int j = consumed; j < issued; ++j) mbar_wait(&full[j % kDepth], (uint32_t)((j / kDepth) & 1));
     }
 }
 
-// one warp per row: the finish as a kernel of its own (stateless entry point)
+// Rows of any alignment: plain loads, one logit per lane per load.
+template <int DT, int MODE>
+__global__ void __launch_bounds__(256) logits_stream_scalar_kernel(const __grid_constant__ StreamParams p) {
+    const int lane = threadIdx.x & 31;
+    const int warp_global = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int n_warps = gridDim.x * (blockDim.x >> 5);
+    if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
+    const PackedConsts kc = packed_consts(p.bf);
+    const int n_tasks = p.R * p.n_spans;
+    for (int task = warp_global; task < n_tasks; task += n_warps) {
+        const int row = task / p.n_spans, sp = task - row * p.n_spans;
+        if (p.done && p.done[row]) continue;
+        const int a0 = sp * p.span, b0 = min(p.V, a0 + p.span);
+        const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
+        LaneSums acc = lane_sums_init();
+        span_scalar<DT, MODE>(rowp, a0, b0, kc, lane, acc);
+        store_triple<MODE>(p, row, sp, acc, lane);
+    }
+}
+
+// the finish as a kernel of its own (stateless entry points): kFinishRows rows per CTA, four warps each
+constexpr int kFinishRows = 8;
 struct FinishKernelParams {
     FinishParams f;
     int R;
@@ -196,28 +441,40 @@ struct FinishKernelParams {
     int32_t* status;
 };
 template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads) logits_finish_kernel(const FinishKernelParams p) {
-    const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    if (row >= p.R || (p.done && p.done[row])) return;
-    const RowResult r = finish_row<DT, MODE>(p.f, row, p.u[row], lane);
-    if (lane == 0) {
-        if (r.tok < 0) raise_status(p.status, PSMC_E_NUMERIC);
-        p.tok[row] = r.tok;
-        p.logp[row] = r.logp;
-        p.loginc[row] = r.loginc;
-    }
+__global__ void __launch_bounds__(1024) logits_finish_kernel(const __grid_constant__ FinishKernelParams p) {
+    __shared__ FinishShared sh;
+    const int row0 = blockIdx.x * kFinishRows;
+    const int n_rows = min(kFinishRows, p.R - row0);
+    const int wpr = finish_warps_per_row(kFinishRows, p.f.span, blockDim.x >> 5);
+    finish_rows<DT, MODE>(
+        p.f, sh, row0, n_rows, wpr, [&](int k) { return !(p.done && p.done[row0 + k]); },
+        [&](int k) { return p.u[row0 + k]; },
+        [&](int k, const RowResult& r) {
+            if (r.tok < 0) raise_status(p.status, PSMC_E_NUMERIC);
+            p.tok[row0 + k] = r.tok;
+            p.logp[row0 + k] = r.logp;
+            p.loginc[row0 + k] = r.loginc;
+        });
 }
 
 typedef void (*StreamFn)(const StreamParams);
 template <int DT, bool VEC>
 StreamFn pick_stream(int mode) {
+    if (VEC) {
+        switch (mode) {
+            case kBeta1: return logits_stream_kernel<DT, kBeta1>;
+            case kBeta2: return logits_stream_kernel<DT, kBeta2>;
+            case kBeta4: return logits_stream_kernel<DT, kBeta4>;
+            case kBeta8: return logits_stream_kernel<DT, kBeta8>;
+            default: return logits_stream_kernel<DT, kBetaAny>;
+        }
+    }
     switch (mode) {
-        case kBeta1: return logits_stream_kernel<DT, kBeta1, VEC>;
-        case kBeta2: return logits_stream_kernel<DT, kBeta2, VEC>;
-        case kBeta4: return logits_stream_kernel<DT, kBeta4, VEC>;
-        case kBeta8: return logits_stream_kernel<DT, kBeta8, VEC>;
-        default: return logits_stream_kernel<DT, kBetaAny, VEC>;
+        case kBeta1: return logits_stream_scalar_kernel<DT, kBeta1>;
+        case kBeta2: return logits_stream_scalar_kernel<DT, kBeta2>;
+        case kBeta4: return logits_stream_scalar_kernel<DT, kBeta4>;
+        case kBeta8: return logits_stream_scalar_kernel<DT, kBeta8>;
+        default: return logits_stream_scalar_kernel<DT, kBetaAny>;
     }
 }
 typedef void (*FinishFn)(const FinishKernelParams);
@@ -236,7 +493,7 @@ FinishFn pick_finish(int mode) {
 
 int logits_pass_span(int R, int V) {
     // about four spans per resident warp when the problem is large enough, between 1024 and 4096 logits each
-    const int64_t resident_warps = (int64_t)kSMs * kCtasPerSm * kWarpsPerCta;
+    const int64_t resident_warps = (int64_t)kSMs * kMaxWarps;
     const int64_t want = ((int64_t)R * V) / (resident_warps * 4);
     int span = 1024;
     while (span < 4096 && span * 2 <= want) span *= 2;
@@ -254,7 +511,7 @@ LogitsGeometry logits_geometry(const void* logits, int dt, int R, int V, int64_t
     g.span = logits_pass_span(R, V);
     g.n_spans = (V + g.span - 1) / g.span;
     g.mode = beta_mode(beta);
-    g.cb = (float)(beta * 1.4426950408889634);
+    g.bf = (float)beta;
     const size_t esize = dt == PSMC_F32 ? 4 : 2;
     g.vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((ld * esize) % 16 == 0) ? 1 : 0;
     return g;
@@ -263,17 +520,39 @@ LogitsGeometry logits_geometry(const void* logits, int dt, int R, int V, int64_t
 cudaError_t launch_logits_stream(const LogitsStreamArgs& a, cudaStream_t stream) {
     const LogitsGeometry g = logits_geometry(a.logits, a.dt, a.R, a.V, a.ld, a.beta);
     StreamParams p;
-    p.logits = a.logits; p.R = a.R; p.V = a.V; p.ld = a.ld; p.span = g.span; p.n_spans = g.n_spans; p.cb = g.cb;
+    p.logits = a.logits; p.R = a.R; p.V = a.V; p.ld = a.ld; p.span = g.span; p.n_spans = g.n_spans; p.bf = g.bf;
     p.done = a.done; p.partials = reinterpret_cast<float4*>(a.scratch); p.zero_words = a.zero_words;
+    p.status = a.status;
     StreamFn fn;
     if (a.dt == PSMC_F32) fn = g.vec ? pick_stream<PSMC_F32, true>(g.mode) : pick_stream<PSMC_F32, false>(g.mode);
     else fn = g.vec ? pick_stream<PSMC_BF16, true>(g.mode) : pick_stream<PSMC_BF16, false>(g.mode);
     const int64_t n_tasks = (int64_t)a.R * g.n_spans;
-    int64_t blocks = (n_tasks + kWarpsPerCta - 1) / kWarpsPerCta;
-    const int64_t max_blocks = (int64_t)kSMs * kCtasPerSm;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (blocks < 1) blocks = 1;
-    fn<<<(unsigned)blocks, kThreads, 0, stream>>>(p);
+    if (n_tasks >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    if (!g.vec) {
+        int64_t blocks = (n_tasks + 7) / 8;
+        if (blocks > (int64_t)kSMs * 8) blocks = (int64_t)kSMs * 8;
+        fn<<<(unsigned)(blocks < 1 ? 1 : blocks), 256, 0, stream>>>(p);
+        return cudaGetLastError();
+    }
+    // one CTA per SM; as many warps per CTA as it takes to give every task a warp, up to kMaxWarps
+    int64_t warps = (n_tasks + kSMs - 1) / kSMs;
+    if (warps > kMaxWarps) warps = kMaxWarps;
+    if (warps < 1) warps = 1;
+    int64_t blocks = (n_tasks + warps - 1) / warps;
+    if (blocks > kSMs) blocks = kSMs;
+    const size_t smem = (size_t)warps * kDepth * kStageBytes;
+    {
+        static std::mutex mu;
+        static bool configured[2][5] = {};
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[a.dt][g.mode]) {
+            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 kMaxWarps * kDepth * kStageBytes);
+            if (e != cudaSuccess) return e;
+            configured[a.dt][g.mode] = true;
+        }
+    }
+    fn<<<(unsigned)blocks, (unsigned)(warps * 32), smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -298,16 +577,17 @@ extern "C" psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R
     LogitsStreamArgs a{};
     a.logits = logits; a.dt = dt; a.R = R; a.V = V; a.ld = ld; a.beta = beta; a.done = done; a.scratch = scratch;
     a.zero_words = nullptr;
+    a.status = status_word;
     if (launch_logits_stream(a, s) != cudaSuccess) return PSMC_E_CUDA;
 
     const LogitsGeometry g = logits_geometry(logits, dt, R, V, ld, beta);
     FinishKernelParams p;
     p.f.logits = logits; p.f.V = V; p.f.ld = ld; p.f.span = g.span; p.f.n_spans = g.n_spans;
-    p.f.partials = reinterpret_cast<const float4*>(scratch); p.f.beta = beta; p.f.alpha_t = alpha_t; p.f.cb = g.cb;
+    p.f.partials = reinterpret_cast<const float4*>(scratch); p.f.beta = beta; p.f.alpha_t = alpha_t; p.f.bf = g.bf;
     p.f.vec = g.vec;
     p.R = R; p.u = u; p.done = done; p.tok = tok; p.logp = logp; p.loginc = loginc; p.status = status_word;
     FinishFn fn = dt == PSMC_F32 ? pick_finish<PSMC_F32>(g.mode) : pick_finish<PSMC_BF16>(g.mode);
-    fn<<<(unsigned)((R + kWarpsPerCta - 1) / kWarpsPerCta), kThreads, 0, s>>>(p);
+    fn<<<(unsigned)((R + kFinishRows - 1) / kFinishRows), 1024, 0, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
@@ -362,15 +642,16 @@ extern "C" psmc_status psmc_logits_pass_static(const void* logits, psmc_dtype dt
     LogitsStreamArgs a{};
     a.logits = logits; a.dt = dt; a.R = R; a.V = V; a.ld = ld; a.beta = beta; a.done = done; a.scratch = scratch;
     a.zero_words = nullptr;
+    a.status = status_word;
     if (launch_logits_stream(a, s) != cudaSuccess) return PSMC_E_CUDA;
 
     const LogitsGeometry g = logits_geometry(logits, dt, R, V, ld, beta);
     FinishKernelParams p;
     p.f.logits = logits; p.f.V = V; p.f.ld = ld; p.f.span = g.span; p.f.n_spans = g.n_spans;
-    p.f.partials = reinterpret_cast<const float4*>(scratch); p.f.beta = beta; p.f.alpha_t = alpha_t; p.f.cb = g.cb;
+    p.f.partials = reinterpret_cast<const float4*>(scratch); p.f.beta = beta; p.f.alpha_t = alpha_t; p.f.bf = g.bf;
     p.f.vec = g.vec;
     p.R = R; p.u = u; p.done = done; p.tok = tok; p.logp = logp; p.loginc = loginc; p.status = status_word;
     FinishFn fn = dt == PSMC_F32 ? pick_finish<PSMC_F32>(g.mode) : pick_finish<PSMC_BF16>(g.mode);
-    fn<<<(unsigned)((R + kWarpsPerCta - 1) / kWarpsPerCta), kThreads, 0, s>>>(p);
+    fn<<<(unsigned)((R + kFinishRows - 1) / kFinishRows), 1024, 0, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a)
     // weights relative to the largest, then the inverse CDF over slots in order
     double mx = -INFINITY;
     for (int i = tid; i < N; i += blockDim.x) mx = fmax(mx, lw[i]);
-    mx = block_max(mx, sh_red);
+    mx = block_max(mx, sh_red, (int)(blockDim.x >> 5));
     for (int i = tid; i < N; i += blockDim.x) sh_w[i] = exp(lw[i] - mx);
     __syncthreads();
     if (tid == 0) {

@@ -2,8 +2,8 @@
 // systematic resampling (Algorithm 1 rows 5-16, Eq. 5, Eq. 7, and the stage-boundary update of
 // Section 4.3 / Appendix B).  One CTA per group.
 //
-// Phase 1 (one warp per particle, looping when N > 32): finish_row() turns the span triples of the
-// streaming kernel into the drawn token y, log p(y) and log omega of the row.
+// Phase 1 (finish_rows: up to eight warps per particle, the CTA's warps shared among the group's rows):
+// the span triples of the streaming kernel become the drawn token y, log p(y) and log omega of each row.
 // Phase 2 (one thread per particle, N <= 1024); reductions and prefix sums run on warp shuffles plus a
 // 33-entry shared array, in an order fixed by the thread index:
 //   log W_r += (alpha_t - alpha_{t-1}) * S_r                     stage boundary (all rows)
@@ -23,6 +23,7 @@ namespace {
 struct KernelArgs {
     WeightsArgs a;
     FinishParams f;
+    int wpr;  // warps per row in the finish
 };
 
 template <int DT, int MODE>
@@ -37,27 +38,25 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     __shared__ int sh_tok[kMaxParticles];
     __shared__ unsigned char sh_done[kMaxParticles];
     __shared__ int sh_base[2];
+    __shared__ FinishShared sh_fin;
 
     const WeightsArgs& a = ka.a;
     const int g = blockIdx.x, i = threadIdx.x, N = a.N;
-    const int lane = i & 31, warp = i >> 5, n_warps = blockDim.x >> 5;
 
-    // ---- phase 1: one warp per live particle finishes its row ----
-    for (int k = warp; k < N; k += n_warps) {
-        const int row = g * N + k;
-        if (a.done[row]) continue;
-        const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)k));
-        const RowResult rr = finish_row<DT, MODE>(ka.f, row, U, lane);
-        if (lane == 0) {
+    // ---- phase 1: the CTA's warps finish the rows of the group's live particles ----
+    finish_rows<DT, MODE>(
+        ka.f, sh_fin, g * N, N, ka.wpr, [&](int k) { return a.done[g * N + k] == 0; },
+        [&](int k) { return hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)k)); },
+        [&](int k, const RowResult& rr) {
             if (rr.tok < 0) raise_status(a.status, PSMC_E_NUMERIC);
             sh_tok[k] = rr.tok;
             sh_S[k] = rr.logp;
             sh_C[k] = rr.loginc;
-        }
-    }
-    __syncthreads();
+        });
+    // finish_rows ends on a CTA-wide barrier: the results are visible to every thread
 
     // ---- phase 2: per-particle update ----
+    const int nw = (N + 31) >> 5;  // warps that hold particles
     const bool on = i < N;
     const int r = g * N + (on ? i : 0);
     double lw = -INFINITY, S = 0.0;
@@ -90,11 +89,11 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     }
 
     // ---- normalise, ESS (Eq. 5) ----
-    const double M = block_max(lw, sh_red);
+    const double M = block_max(lw, sh_red, nw);
     const double w = on ? exp(lw - M) : 0.0;
     double s1;
-    const double C = block_scan_incl(w, sh_red, &s1);
-    const double s2 = block_sum(w * w, sh_red);
+    const double C = block_scan_incl(w, sh_red, &s1, nw);
+    const double s2 = block_sum(w * w, sh_red, nw);
     const double ess = s1 * s1 / s2;
     const bool fire = ess < a.kappa * (double)N;
     if (i == 0) {
@@ -145,9 +144,9 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     const int dead = (on && off == 0) ? 1 : 0;
     const int surplus = (on && off > 1) ? off - 1 : 0;
     int n_dead, n_src;
-    const int dead_incl = block_scan_incl(dead, sh_redi, &n_dead);
-    const int sur_incl = block_scan_incl(surplus, sh_redi, (int*)nullptr);
-    const int src_incl = block_scan_incl(surplus > 0 ? 1 : 0, sh_redi, &n_src);
+    const int dead_incl = block_scan_incl(dead, sh_redi, &n_dead, nw);
+    const int sur_incl = block_scan_incl(surplus, sh_redi, (int*)nullptr, nw);
+    const int src_incl = block_scan_incl(surplus > 0 ? 1 : 0, sh_redi, &n_src, nw);
     if (on) sh_Einc[i] = sur_incl;
     if (i == 0) {
         sh_base[0] = atomicAdd(a.n_moves, n_dead);
@@ -208,8 +207,11 @@ cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream) {
     ka.a = a;
     ka.f.logits = a.logits; ka.f.V = a.V; ka.f.ld = a.ld; ka.f.span = g.span; ka.f.n_spans = g.n_spans;
     ka.f.partials = reinterpret_cast<const float4*>(a.scratch); ka.f.beta = a.beta; ka.f.alpha_t = a.alpha_t;
-    ka.f.cb = g.cb; ka.f.vec = g.vec;
-    const int warps = a.N < 32 ? a.N : 32;  // one warp per particle up to 32, then the warps loop
+    ka.f.bf = g.bf; ka.f.vec = g.vec;
+    // up to eight warps per particle while the CTA has room for them; beyond 32 particles the warps loop over rows
+    const int wpr = finish_warps_per_row(a.N, g.span, kFinishMaxWarps);
+    const int warps = a.N * wpr < kFinishMaxWarps ? a.N * wpr : kFinishMaxWarps;
+    ka.wpr = wpr;
     Fn fn = a.dt == PSMC_F32 ? pick<PSMC_F32>(g.mode) : pick<PSMC_BF16>(g.mode);
     fn<<<a.G, warps * 32, 0, stream>>>(ka);
     return cudaGetLastError();

@@ -102,7 +102,7 @@ def case_step(a):
     G = cfg.G if a.groups is None else a.groups
     wl = WC.DeviceWorkload(cfg, 1, G=G)
     n_buf = min(64, max(2, -(-2 * L2_BYTES // (wl.R * cfg.logit_bytes_per_row))))
-    T = a.iters + 2
+    T = 2 * a.iters + 4
     ps = B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
                 T_max=T, prompt_len=wl.prompt_len)
     bufs = [wl.new_logits() for _ in range(n_buf)]
@@ -115,8 +115,16 @@ def case_step(a):
 
     us = _time(run, a.iters)
     assert ps.sync_status() == B.OK
+    # the two kernels of the step, each bracketed by events on the stream
+    ps.reset(1)
+    ps.timing_enable(True)
+    for i in range(a.iters):
+        run(i)
+    kms, kn = ps.timing_read()
+    ps.timing_enable(False)
     ps.destroy()
     return {"case": "step", "workload": cfg.name, "rows": wl.R, "vocab": cfg.V, "buffers": n_buf, "us": us,
+            "logits_stream_us": 1e3 * kms[0] / max(kn[0], 1), "finish_weights_us": 1e3 * kms[1] / max(kn[1], 1),
             "us_median": float(np.median(us)), "bytes": wl.R * cfg.logit_bytes_per_row,
             "gb_per_s": wl.R * cfg.logit_bytes_per_row / (np.median(us) * 1e-6) / 1e9}
 
