@@ -11,6 +11,15 @@ namespace psmc {
 constexpr int kWarp = 32;
 constexpr unsigned kFull = 0xffffffffu;
 
+// ---- programmatic dependent launch: a kernel launched with launch_chained() may be scheduled while the kernel
+// before it on the stream is still running.  chain_begin() lets the next kernel of the stream be scheduled early in
+// turn, then waits until the previous kernel has completed and its writes are visible; nothing that reads or
+// writes global memory may come before it.  Both are no-ops in a kernel launched the ordinary way. ----
+__device__ __forceinline__ void chain_begin() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- sticky device status word: the first error wins ----
 __device__ __forceinline__ void raise_status(int32_t* word, int code) {
     if (word) atomicCAS(word, 0, code);
@@ -75,12 +84,17 @@ __device__ __forceinline__ T warp_scan_incl(T v, int lane) {
 
 // ---- block collectives for up to 1024 threads (32 warps); `sh` holds 33 items ----
 // Every thread of the CTA calls them; only the first `nwarp` warps carry data (the others pass the identity).
+// With nwarp == 1 they are plain warp collectives without any CTA barrier, to be called by warp 0 alone.
 // Inclusive scan over threadIdx.x order.  Also returns the block total.  The order of additions is
 // fixed by the thread index, so results do not depend on scheduling.
 template <typename T>
 __device__ __forceinline__ T block_scan_incl(T v, T* sh, T* total, int nwarp) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     T incl = warp_scan_incl(v, lane);
+    if (nwarp == 1) {
+        if (total) *total = __shfl_sync(kFull, incl, 31);
+        return incl;
+    }
     __syncthreads();  // sh may still be read by a previous call
     if (lane == 31 && warp < nwarp) sh[warp] = incl;
     __syncthreads();
@@ -97,6 +111,7 @@ template <typename T>
 __device__ __forceinline__ T block_max(T v, T* sh, int nwarp) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     v = warp_max(v);
+    if (nwarp == 1) return v;
     __syncthreads();
     if (lane == 0 && warp < nwarp) sh[warp] = v;
     __syncthreads();
@@ -107,12 +122,19 @@ __device__ __forceinline__ T block_max(T v, T* sh, int nwarp) {
 __device__ __forceinline__ double block_sum(double v, double* sh, int nwarp) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     v = warp_sum(v);
+    if (nwarp == 1) return v;
     __syncthreads();
     if (lane == 0 && warp < nwarp) sh[warp] = v;
     __syncthreads();
     double s = 0.0;
     for (int w = 0; w < nwarp; ++w) s += sh[w];
     return s;
+}
+
+// CTA barrier, or a warp barrier when a single warp is at work
+__device__ __forceinline__ void group_sync(int nwarp) {
+    if (nwarp == 1) __syncwarp();
+    else __syncthreads();
 }
 
 }  // namespace psmc

@@ -9,6 +9,26 @@
 
 namespace psmc {
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled (and run up to its chain_begin())
+// while the previous kernel of the stream drains, which hides launch latency between the kernels of a step.
+// Every kernel launched this way calls chain_begin() before it touches global memory, and every grid of the
+// step fits the GPU in one wave, so early CTAs never keep a predecessor's CTAs from being scheduled.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int kMaxParticles = 1024;  // one CTA per group in the weight/resample kernel
 constexpr int kSMs = 148;            // B200
 

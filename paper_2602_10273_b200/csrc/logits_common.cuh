@@ -11,7 +11,7 @@
 // over two floats, so the product carries no representation error of log2(e) and the big parts cancel
 // before the small one is added.  The streaming kernel cuts a row into spans and writes one triple (c, s1, sb)
 // per span:   c = a reference exponent (close to the span's largest x),  s1 = sum 2^{x - c},
-//   sb = sum 2^{beta (x - c)}.
+//   sb = sum 2^{beta (x - c)}.  Reference exponents are whole numbers.
 // The finish rescales the triples to the row's largest c in fp64, in span order, finds the span
 // that holds U * sum_all by a prefix sum over the sb terms, and re-reads only that span.
 #pragma once
@@ -48,8 +48,9 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ float rel_exponent(float l, float neg_c) {
     return fmaf(l, kLog2eLo, fmaf(l, kLog2eHi, neg_c));
 }
-// reference exponent for a logit value m: about m * log2(e), kept finite
-__device__ __forceinline__ float ref_exponent(float m) { return fmaxf(m * kLog2eHi, kRefFloor); }
+// reference exponent for a logit value m: m * log2(e) rounded up to a whole number (so that rescaling between
+// reference points is an exact power of two), kept finite
+__device__ __forceinline__ float ref_exponent(float m) { return fmaxf(ceilf(m * kLog2eHi), kRefFloor); }
 
 // 2^{beta d} for d = x - c.  One MUFU: for beta in {1,2,4,8} 2^d is squared up; bf = (float)beta otherwise.
 template <int MODE>
@@ -103,8 +104,22 @@ struct RowTotals {
     int jsel;       // span that holds the target
 };
 
+// 2^{dc} and 2^{beta dc} for a span whose reference exponent lies dc <= 0 below the row's.  dc is a whole number,
+// so for whole beta both factors are exact powers of two (ldexp); other beta take one fp64 exp2.
+template <int MODE>
+__device__ __forceinline__ void span_scales(float dcf, double beta, double& f1, double& fb) {
+    const int dc = (int)fmaxf(dcf, -4000.f);  // below -2100 or so every factor is 0 anyway
+    f1 = ldexp(1.0, dc);
+    if (MODE == kBeta1) fb = f1;
+    else if (MODE == kBeta2) fb = ldexp(1.0, 2 * dc);
+    else if (MODE == kBeta4) fb = ldexp(1.0, 4 * dc);
+    else if (MODE == kBeta8) fb = ldexp(1.0, 8 * dc);
+    else fb = exp2(beta * (double)dc);
+}
+
 template <int MODE>
 __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane) {
+    constexpr int kKeep = 8;  // span masses a lane keeps in registers between the two sweeps (rows of <= 256 spans)
     RowTotals t;
     t.ok = false;
     const int n = p.n_spans;
@@ -114,16 +129,23 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     for (int j = lane; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
     cf = warp_max(cf);
     t.C = cf;
-    const double C = (double)cf;
 
     // totals, every term rescaled to the row's reference in fp64
     double a_sum = 0.0, b_sum = 0.0;
-    for (int j = lane; j < n; j += 32) {
+    double keep[kKeep];
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) keep[i] = 0.0;
+    for (int j = lane, i = 0; j < n; j += 32, ++i) {
         const float4 f = __ldcg(&P[j]);
-        const double dc = (double)f.x - C;
-        const double a = (double)f.y * exp2(dc);
+        double f1, fb;
+        span_scales<MODE>(f.x - cf, p.beta, f1, fb);
+        const double a = (double)f.y * f1;
+        const double b = (MODE == kBeta1) ? a : (double)f.z * fb;
         a_sum += a;
-        b_sum += (MODE == kBeta1) ? a : (double)f.z * exp2(p.beta * dc);
+        b_sum += b;
+#pragma unroll
+        for (int q = 0; q < kKeep; ++q)
+            if (q == i) keep[q] = b;
     }
     t.S1 = warp_sum(a_sum);
     t.Sb = warp_sum(b_sum);
@@ -133,13 +155,18 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     t.target = U * t.Sb;
     double carry = 0.0, base = 0.0, last_base = 0.0;
     int jsel = -1, last_pos = -1;
-    for (int c = 0; c < n && jsel < 0; c += 32) {
+    for (int c = 0, i = 0; c < n && jsel < 0; c += 32, ++i) {
         const int j = c + lane;
         double b = 0.0;
-        if (j < n) {
+        if (i < kKeep) {
+#pragma unroll
+            for (int q = 0; q < kKeep; ++q)
+                if (q == i) b = keep[q];
+        } else if (j < n) {
             const float4 f = __ldcg(&P[j]);
-            const double dc = (double)f.x - C;
-            b = (MODE == kBeta1) ? (double)f.y * exp2(dc) : (double)f.z * exp2(p.beta * dc);
+            double f1, fb;
+            span_scales<MODE>(f.x - cf, p.beta, f1, fb);
+            b = (MODE == kBeta1) ? (double)f.y * f1 : (double)f.z * fb;
         }
         const double incl = carry + warp_scan_incl(b, lane);
         const unsigned hit = __ballot_sync(kFull, b > 0.0 && incl >= t.target);
@@ -261,8 +288,10 @@ __device__ __forceinline__ RowResult row_result(const FinishParams& p, const voi
 // ---- the finish at CTA level: several warps share a row ----
 constexpr int kFinishMaxWarps = 32;
 struct FinishShared {
-    double tot[kFinishMaxWarps];  // mass of the part of the selected span each warp re-read
-    int last[kFinishMaxWarps];    // last position with mass in that part (-1 if none)
+    RowTotals row[kFinishMaxWarps];  // per row of the current pass: what its first warp learnt from the triples
+    bool live[kFinishMaxWarps];      // does the row need finishing at all
+    double tot[kFinishMaxWarps];     // mass of the part of the selected span each warp re-read
+    int last[kFinishMaxWarps];       // last position with mass in that part (-1 if none)
 };
 
 // warps per row: as many as the CTA can spare, each part of the span at least 256 logits (8 per lane)
@@ -272,27 +301,41 @@ __host__ __device__ inline int finish_warps_per_row(int n_rows, int span, int n_
     return w;
 }
 
-// Every thread of the CTA calls this (it synchronises the CTA).  Finishes rows row0 .. row0+n_rows-1, `wpr` warps
-// (a power of two) per row, n_warps/wpr rows at a time.  live(k): does row k need finishing; uniform(k): its U;
-// emit(k, result) is called by lane 0 of one warp per finished row.
+// Every thread of the CTA calls this (it synchronises the CTA).  Finishes rows row0 .. row0+n_rows-1, n_warps/wpr
+// rows at a time: one warp per row combines the span triples, then `wpr` warps (a power of two) share the re-read of
+// the selected span, then the warp whose part holds the target pins the token down.  live(k): does row k need
+// finishing; uniform(k): its U; emit(k, result) is called by lane 0 of one warp per finished row.
 template <int DT, int MODE, class LiveFn, class UniformFn, class EmitFn>
 __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared& sh, int row0, int n_rows, int wpr,
                                             LiveFn live, UniformFn uniform, EmitFn emit) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const int rows_per_pass = n_warps / wpr;
-    const int q = warp & (wpr - 1);
+    const int q = warp & (wpr - 1), kk = warp / wpr;  // this warp's part of the span, and its row within the pass
     for (int k0 = 0; k0 < n_rows; k0 += rows_per_pass) {
-        const int k = k0 + warp / wpr;
-        const bool active = warp < rows_per_pass * wpr && k < n_rows && live(k);
-        const int row = row0 + k;
-        const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
+        // ---- one warp per row: totals, target, span ----
+        if (warp < rows_per_pass) {
+            const int k = k0 + warp;
+            const bool lv = k < n_rows && live(k);
+            RowTotals t;
+            t.ok = false;
+            if (lv) t = combine_spans<MODE>(p, row0 + k, uniform(k), lane);
+            if (lane == 0) {
+                sh.live[warp] = lv;
+                sh.row[warp] = t;
+            }
+        }
+        __syncthreads();
+        // ---- wpr warps per row: mass of each part of the selected span ----
+        const int k = k0 + kk;
+        const bool active = kk < rows_per_pass && sh.live[kk];
+        const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)(row0 + k) * p.ld * (DT == PSMC_F32 ? 4 : 2);
         RowTotals t;
         t.ok = false;
         double lm = 0.0, incl = 0.0;
         int a0 = 0, b0 = 0, E = 0, sub = 0;
         float neg_C = 0.f;
         if (active) {
-            t = combine_spans<MODE>(p, row, uniform(k), lane);
+            t = sh.row[kk];
             int wl = -1;
             if (t.ok) {
                 neg_C = -t.C;
@@ -309,6 +352,7 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
             if (lane == 0) sh.last[warp] = wl;
         }
         __syncthreads();
+        // ---- the warp whose part reaches the target: the token ----
         if (active) {
             const int w0 = warp - q;  // first warp of this row
             if (!t.ok) {
@@ -340,7 +384,7 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
                 if (mine && lane == 0) emit(k, y >= 0 ? row_result<DT>(p, rowp, t, y) : RowResult{-1, 0.0, 0.0});
             }
         }
-        __syncthreads();  // sh is reused by the next pass
+        __syncthreads();  // sh is reused by the next pass; the emitted results are visible to the CTA
     }
 }
 

@@ -284,7 +284,6 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) logits_stream_kernel(const 
     const int n_tasks = p.R * p.n_spans;  // < 2^31, checked by the host
     const int per_warp = (n_tasks + n_warps - 1) / n_warps;
     const int first = min(n_tasks, warp_global * per_warp), last = min(n_tasks, first + per_warp);
-    if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
 
     const PackedConsts kc = packed_consts(p.bf);
     unsigned char* ring = smem + (size_t)warp * kDepth * kStageBytes;
@@ -295,6 +294,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) logits_stream_kernel(const 
         fence_async_smem();
     }
     __syncwarp();
+    chain_begin();  // everything above is local set-up; global memory from here on
+    if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
 
     // producer cursor (the same in every lane; lane 0 issues): the next piece to fetch
     TaskWalker<DT> pw;
@@ -552,8 +553,7 @@ cudaError_t launch_logits_stream(const LogitsStreamArgs& a, cudaStream_t stream)
             configured[a.dt][g.mode] = true;
         }
     }
-    fn<<<(unsigned)blocks, (unsigned)(warps * 32), smem, stream>>>(p);
-    return cudaGetLastError();
+    return launch_chained(fn, dim3((unsigned)blocks), dim3((unsigned)(warps * 32)), smem, stream, p);
 }
 
 }  // namespace psmc

@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant_
     __shared__ __align__(8) uint64_t bars[kStages];
     __shared__ Item ring[kStages];
 
+    chain_begin();
     const int n_src = *reinterpret_cast<const volatile int32_t*>(k.n_sources);
     if (n_src <= 0) return;  // nothing resampled this step
     if (threadIdx.x != 0) return;
@@ -234,8 +235,7 @@ cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream) {
             if (e != cudaSuccess) return e;
             configured = true;
         }
-        reindex_bulk_kernel<<<kSMs * kBulkCtasPerSm, 32, smem, stream>>>(k);
-        return cudaGetLastError();
+        return launch_chained(reindex_bulk_kernel, dim3(kSMs * kBulkCtasPerSm), dim3(32), (size_t)smem, stream, k);
     }
     // widest unit that divides every address, stride and row size
     uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |

@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     const WeightsArgs& a = ka.a;
     const int g = blockIdx.x, i = threadIdx.x, N = a.N;
 
+    chain_begin();
     // ---- phase 1: the CTA's warps finish the rows of the group's live particles ----
     finish_rows<DT, MODE>(
         ka.f, sh_fin, g * N, N, ka.wpr, [&](int k) { return a.done[g * N + k] == 0; },
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
 
     // ---- phase 2: per-particle update ----
     const int nw = (N + 31) >> 5;  // warps that hold particles
+    if (nw == 1 && i >= 32) return;  // up to 32 particles: warp 0 finishes alone, on warp collectives only
     const bool on = i < N;
     const int r = g * N + (on ? i : 0);
     double lw = -INFINITY, S = 0.0;
@@ -124,7 +126,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
         sh_done[i] = dn;
         sh_off[i] = 0;
     }
-    __syncthreads();
+    group_sync(nw);
     int anc = N - 1;
     if (on) {
         const double u0 = hash_uniform(hash5(a.seed, kStreamResample, (uint64_t)g, (uint64_t)a.t, 0));
@@ -137,7 +139,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
         anc = lo < N ? lo : N - 1;
         atomicAdd(&sh_off[anc], 1);
     }
-    __syncthreads();
+    group_sync(nw);
 
     // ---- slot map ----
     const int off = on ? sh_off[i] : 1;
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
         sh_base[0] = atomicAdd(a.n_moves, n_dead);
         sh_base[1] = atomicAdd(a.n_sources, n_src);
     }
-    __syncthreads();
+    group_sync(nw);
     int mp = i;
     if (dead) {
         const int rank = dead_incl - 1;  // this dead slot takes surplus offspring number `rank`
@@ -213,8 +215,7 @@ cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream) {
     const int warps = a.N * wpr < kFinishMaxWarps ? a.N * wpr : kFinishMaxWarps;
     ka.wpr = wpr;
     Fn fn = a.dt == PSMC_F32 ? pick<PSMC_F32>(g.mode) : pick<PSMC_BF16>(g.mode);
-    fn<<<a.G, warps * 32, 0, stream>>>(ka);
-    return cudaGetLastError();
+    return launch_chained(fn, dim3((unsigned)a.G), dim3((unsigned)(warps * 32)), 0, stream, ka);
 }
 
 }  // namespace psmc

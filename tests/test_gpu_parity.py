@@ -74,7 +74,7 @@ def test_logits_pass_matches_oracle(dtype, beta, V):
     tok, logp, loginc, status = run_logits_pass(logits, beta, beta, u)
     assert status == B.OK
     check_rows_against_oracle(logits, beta, beta, u, tok, logp, loginc)
-    assert tok[5] == V - 3 and abs(loginc[5]) < 1e-12
+    assert tok[5] == V - 3 and abs(loginc[5]) < 1e-6      # one-hot row: log omega = 0 (closed form), one approximate ex2 away
     assert abs(loginc[4] - (1.0 - beta) * math.log(V)) < 1e-5
 
 
