@@ -31,6 +31,11 @@ from paper_2602_10273_b200.workload import gen  # noqa: E402
 METRIC = "particle_tokens_per_s"
 UNIT = "particle-tokens/s"
 N_BLOCKS = 6           # distinct logit blocks rotated through (6 x 131 MB at the default workload: beyond L2)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte, from the ncu captures summarised
+# under profiles/ (logits_stream_kernel__batched_prompts.md, reindex_bulk_kernel__64rows_8layers_len1024.md; the
+# reindex capture ran on a smaller cache and its traffic scales with the bytes moved).  An entry goes back to None
+# when its kernel changes, until the counters are taken again.
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"logits_stream_kernel": 1.032, "reindex_bulk_kernel": 0.978}
 
 
 def load_peaks():
@@ -217,18 +222,25 @@ def run_ours(args):
     k1_gbs = k1_bytes / (kms[0] * 1e-3) / 1e9 if kms[0] > 0 else 0.0
     k3_gbs = k3_bytes / (kms[2] * 1e-3) / 1e9 if kms[2] > 0 and k3_bytes > 0 else 0.0
     shares = [m / max(sum(kms), 1e-12) for m in kms]
+
+    def traffic(kernel, algorithmic_bytes, launches):
+        r = TRAFFIC_PER_ALGORITHMIC_BYTE.get(kernel)
+        return None if r is None or launches < 1 else r * algorithmic_bytes / launches
+
     dominant = int(np.argmax(kms))
-    names = ["logits_pass_kernel", "weights_resample_kernel", "reindex_bulk_kernel"]
+    names = ["logits_stream_kernel", "finish_weights_resample_kernel", "reindex_bulk_kernel"]
     roofs = {
-        "logits_pass_kernel": {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
-                               "frac": k1_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+        "logits_stream_kernel": {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
+                               "frac": k1_gbs / hbm_peak, "traffic": traffic("logits_stream_kernel", k1_bytes, kn[0]),
+                               "peak_kind": peak_kind,
                                "avg_launch_us": 1e3 * kms[0] / max(kn[0], 1), "time_share": shares[0],
                                "bytes_per_launch": k1_bytes / max(kn[0], 1)},
         "reindex_bulk_kernel": {"bound": "hbm", "achieved": k3_gbs, "peak": hbm_peak, "unit": "GB/s",
-                                "frac": k3_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                                "frac": k3_gbs / hbm_peak, "traffic": traffic("reindex_bulk_kernel", k3_bytes, kn[2]),
+                                "peak_kind": peak_kind,
                                 "avg_launch_us": 1e3 * kms[2] / max(kn[2], 1), "time_share": shares[2],
                                 "bytes_per_launch": k3_bytes / max(kn[2], 1)},
-        "weights_resample_kernel": {"bound": "latency", "avg_launch_us": 1e3 * kms[1] / max(kn[1], 1),
+        "finish_weights_resample_kernel": {"bound": "latency", "avg_launch_us": 1e3 * kms[1] / max(kn[1], 1),
                                     "time_share": shares[1]},
     }
     roofline = dict(roofs[names[dominant]] if dominant != 1 else roofs["reindex_bulk_kernel"])
