@@ -27,7 +27,9 @@ struct psmc_ctx {
     // move records: [0] from the step, [1] from an idx_override
     MoveSource* sources[2];
     int32_t* dst_rows[2];
-    int32_t* counts[2];  // {n_sources, n_moves}
+    int32_t* counts[3];  // {n_sources, n_moves}: [0]/[1] steps of even/odd index (they alternate), [2] idx_override
+    int32_t* row_arrivals;    // [R] arrival counters of the fused step kernel (zero between launches)
+    int32_t* group_arrivals;  // [G]
     int32_t* status;
     int32_t* kv_work;    // [2] unit queue of the reindex kernels (kept at zero between launches by the kernels)
     void* scratch;       // logit-pass tickets and span triples
@@ -60,7 +62,8 @@ psmc_status reset_device_state(psmc_ctx* c) {
     auto z = [&](void* p, size_t bytes) { if (e == cudaSuccess) e = cudaMemset(p, 0, bytes); };
     z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
     z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
-    z(c->counts[0], 8); z(c->counts[1], 8); z(c->status, 4); z(c->kv_work, 8);
+    z(c->counts[0], 8); z(c->counts[1], 8); z(c->counts[2], 8); z(c->status, 4); z(c->kv_work, 8);
+    z(c->row_arrivals, 4 * R); z(c->group_arrivals, 4 * G);
     if (e != cudaSuccess) return PSMC_E_CUDA;
     // lens = prompt length of the group; identity maps; tokens -1; ESS = N
     int32_t* h = new (std::nothrow) int32_t[R];
@@ -116,7 +119,8 @@ void free_ctx(psmc_ctx* c) {
     for (auto e : c->event_pool) cudaEventDestroy(e);
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
-                    c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->status, c->kv_work, c->scratch, c->staging};
+                    c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
+                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete[] c->prompt_len_host;
@@ -155,8 +159,10 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     ok(dev_alloc(&c->logZ, (size_t)G));
     ok(dev_alloc(&c->hist_tok, R * (size_t)T_max)); ok(dev_alloc(&c->hist_map, R * (size_t)T_max));
     for (int s = 0; s < 2; ++s) {
-        ok(dev_alloc(&c->sources[s], R)); ok(dev_alloc(&c->dst_rows[s], R)); ok(dev_alloc(&c->counts[s], 2));
+        ok(dev_alloc(&c->sources[s], R)); ok(dev_alloc(&c->dst_rows[s], R));
     }
+    for (int s = 0; s < 3; ++s) ok(dev_alloc(&c->counts[s], 2));
+    ok(dev_alloc(&c->row_arrivals, R)); ok(dev_alloc(&c->group_arrivals, (size_t)G));
     ok(dev_alloc(&c->status, 1));
     ok(dev_alloc(&c->kv_work, 2));
     ok(cudaMalloc(&c->scratch, logits_pass_scratch_bytes(c->R, c->V)));
@@ -201,11 +207,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = beta_t;
     la.done = c->done; la.scratch = c->scratch;
     la.status = c->status;
-    la.zero_words = c->counts[0];  // the step's two move counters are cleared by the first kernel of the step
-    {
-        LaunchTimer lt(c, s, 0);
-        if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
-    }
+    la.zero_words = c->counts[(t + 1) & 1];  // each step clears the pair of move counters the next step will use
 
     WeightsArgs wa{};
     wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos;
@@ -218,9 +220,16 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     wa.hist_tok = c->hist_tok + (size_t)(t - 1) * c->R;
     wa.hist_map = c->hist_map + (size_t)(t - 1) * c->R;
     wa.sources = c->sources[0]; wa.dst_rows = c->dst_rows[0];
-    wa.n_sources = c->counts[0]; wa.n_moves = c->counts[0] + 1;
+    wa.n_sources = c->counts[t & 1]; wa.n_moves = c->counts[t & 1] + 1;
     wa.status = c->status;
-    {
+    if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
+        LaunchTimer lt(c, s, 0);
+        if (launch_step_fused(la, wa, c->row_arrivals, c->group_arrivals, s) != cudaSuccess) return PSMC_E_CUDA;
+    } else {
+        {
+            LaunchTimer lt(c, s, 0);
+            if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
+        }
         LaunchTimer lt(c, s, 1);
         if (launch_weights_resample(wa, s) != cudaSuccess) return PSMC_E_CUDA;
     }
@@ -273,7 +282,7 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
     const int set = idx_override ? 1 : 0;
     if (idx_override) {
         if (launch_build_moves(idx_override, c->R, src->max_len, dst ? 0 : 1, c->sources[1], c->dst_rows[1],
-                               c->counts[1], c->counts[1] + 1, c->status, s) != cudaSuccess)
+                               c->counts[2], c->counts[2] + 1, c->status, s) != cudaSuccess)
             return PSMC_E_CUDA;
     }
     const psmc_kv_desc* d = dst ? dst : src;
@@ -288,7 +297,7 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
     k.max_len = src->max_len;
     k.sources = c->sources[set];
     k.dst_rows = c->dst_rows[set];
-    k.n_sources = c->counts[set];
+    k.n_sources = idx_override ? c->counts[2] : c->counts[c->t & 1];
     k.status = c->status;
     k.work = c->kv_work;
     uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |
@@ -396,6 +405,6 @@ extern "C" const double* psmc_ess(psmc_ctx* c) { return c ? c->ess : nullptr; }
 extern "C" const double* psmc_log_z(psmc_ctx* c) { return c ? c->logZ : nullptr; }
 extern "C" const int32_t* psmc_lens(psmc_ctx* c) { return c ? c->len : nullptr; }
 extern "C" const uint8_t* psmc_done(psmc_ctx* c) { return c ? c->done : nullptr; }
-extern "C" const int32_t* psmc_move_count(psmc_ctx* c) { return c ? c->counts[0] + 1 : nullptr; }
+extern "C" const int32_t* psmc_move_count(psmc_ctx* c) { return c ? c->counts[c->t & 1] + 1 : nullptr; }
 extern "C" int psmc_step_index(const psmc_ctx* c) { return c ? c->t : -1; }
 extern "C" int psmc_rows(const psmc_ctx* c) { return c ? c->R : -1; }

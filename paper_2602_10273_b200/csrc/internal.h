@@ -96,6 +96,12 @@ struct WeightsArgs {
 };
 cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream);
 
+// The logit pass and the per-group update as one kernel: possible for groups of up to 32 particles whose logit
+// rows start on 16-byte boundaries.  row_arrivals [R] and group_arrivals [G] are zero between launches.
+bool step_can_fuse(const LogitsStreamArgs& la, int N);
+cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, int32_t* row_arrivals,
+                              int32_t* group_arrivals, cudaStream_t stream);
+
 // ---------------------------------------------------------------- KV reindex (Appendix C)
 constexpr int kMaxKvPtrs = 128;  // K and V pointers per launch (64 layers); more layers take more launches
 struct KvLaunch {

@@ -285,6 +285,34 @@ __device__ __forceinline__ RowResult row_result(const FinishParams& p, const voi
     return r;
 }
 
+// ---- the finish of one row by one warp on its own (no shared memory, no CTA barrier) ----
+// Every lane returns the same RowResult.
+template <int DT, int MODE>
+__device__ __forceinline__ RowResult finish_row_warp(const FinishParams& p, int row, double U, int lane) {
+    const RowResult bad{-1, 0.0, 0.0};
+    const RowTotals t = combine_spans<MODE>(p, row, U, lane);
+    if (!t.ok) return bad;
+    const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
+    const float neg_C = -t.C;
+    const int a0 = t.jsel * p.span, b0 = min(p.V, a0 + p.span);
+    const int E = p.span >> 5;
+    int lane_last;
+    const double lm = lane_share<DT, MODE>(p, rowp, a0 + lane * E, E, b0, neg_C, lane_last);
+    const double r_incl = t.base + warp_scan_incl(lm, lane);
+    const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+    int y;
+    if (hit2) {
+        const int owner = __ffs(hit2) - 1;
+        const double run = __shfl_sync(kFull, r_incl - lm, owner);
+        const int o0 = a0 + owner * E;
+        y = locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+    } else {
+        y = warp_max(lane_last);  // the re-read sums fall short of the target: last token with mass in the span
+    }
+    if (y < 0) return bad;
+    return row_result<DT>(p, rowp, t, y);
+}
+
 // ---- the finish at CTA level: several warps share a row ----
 constexpr int kFinishMaxWarps = 32;
 struct FinishShared {
