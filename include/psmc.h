@@ -55,6 +55,14 @@ typedef enum {
 
 typedef enum { PSMC_F32 = 0, PSMC_BF16 = 1 } psmc_dtype;
 
+/* Resampling schemes (Appendix E, "Resampling Choices": any unbiased scheme preserves the target). */
+typedef enum {
+    PSMC_RESAMPLE_SYSTEMATIC = 0,  /* Algorithm 1 row 13: positions (u0 + i)/N, one uniform per group and step */
+    PSMC_RESAMPLE_STRATIFIED = 1,  /* positions (u_i + i)/N, one uniform per particle                            */
+    PSMC_RESAMPLE_MULTINOMIAL = 2, /* positions u_i: N independent draws from Categorical(W)                     */
+    PSMC_RESAMPLE_RESIDUAL = 3     /* floor(N W_j) copies of j, the rest drawn from the residual weights          */
+} psmc_resampler;
+
 /* ------------------------------------------------------------------------- */
 /* Context (inputs of Algorithm 1: alpha, N, kappa, T_max, proposal)          */
 /* ------------------------------------------------------------------------- */
@@ -74,6 +82,11 @@ psmc_status psmc_init(psmc_ctx** out, int N, int V, float alpha, float tau, floa
 psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, float alpha, float tau,
                               float ess_thresh, int ramp, uint64_t seed, int eos_id, int T_max,
                               const int32_t* prompt_len_host);
+
+/* Scheme used by the following steps (default PSMC_RESAMPLE_SYSTEMATIC).  Uniforms: H(seed,2,group,t,0) for the
+ * systematic offset, H(seed,2,group,t,1+i) for particle (or residual draw) i of the others.  For multinomial and
+ * residual resampling the ancestor vector is in drawing order, not sorted. */
+psmc_status psmc_set_resampler(psmc_ctx*, psmc_resampler kind);
 
 psmc_status psmc_destroy(psmc_ctx*);                 /* syncs the device, frees everything   */
 psmc_status psmc_reset(psmc_ctx*, uint64_t seed);    /* t=0, weights 1, S=0, done=0; syncs    */
@@ -212,7 +225,8 @@ const double*  psmc_ess(psmc_ctx*);          /* [G] ESS of Eq. 5 before resampli
 const double*  psmc_log_z(psmc_ctx*);        /* [G] running log of the normaliser estimate               */
 const int32_t* psmc_lens(psmc_ctx*);         /* [R] live KV length                                       */
 const uint8_t* psmc_done(psmc_ctx*);         /* [R]                                                      */
-const int32_t* psmc_move_count(psmc_ctx*);   /* [1] slots rewritten by the last step's maps              */
+const int32_t* psmc_move_count(psmc_ctx*);   /* [1] slots rewritten by the last step's maps (ask again after each step:
+                                                    the counter alternates between two words)                */
 
 int psmc_step_index(const psmc_ctx*);        /* t: tokens decoded so far                                 */
 int psmc_rows(const psmc_ctx*);              /* R                                                        */

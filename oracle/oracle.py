@@ -63,6 +63,12 @@ def lib():
         L.orc_ess.argtypes = [_f64p, C.c_int] + [_f64p] * 4
         L.orc_systematic.restype = None
         L.orc_systematic.argtypes = [_f64p, C.c_int, C.c_double, C.c_double, _i32p, _f64p]
+        for name in ("orc_stratified", "orc_multinomial", "orc_residual"):
+            f = getattr(L, name)
+            f.restype = None
+            f.argtypes = [_f64p, C.c_int, C.c_double, _f64p, _i32p, _f64p]
+        L.orc_set_resampler.restype = C.c_int
+        L.orc_set_resampler.argtypes = [C.c_void_p, C.c_int]
         L.orc_slot_map.restype = None
         L.orc_slot_map.argtypes = [_i32p, C.c_int, _i32p]
         L.orc_create.restype = C.c_void_p
@@ -158,6 +164,25 @@ def systematic(w, u0: float):
     return A, mg.value
 
 
+SYSTEMATIC, STRATIFIED, MULTINOMIAL, RESIDUAL = 0, 1, 2, 3
+
+
+def resample(kind: int, w, u):
+    """Ancestors under the stratified / multinomial / residual scheme for unnormalised weights w and
+    uniforms u (one per particle); returns (A, margin)."""
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    assert u.size == w.size
+    s1 = 0.0
+    for x in w:  # sequential, as in the C loop
+        s1 += float(x)
+    A = np.zeros(w.size, dtype=np.int32)
+    mg = C.c_double()
+    f = {STRATIFIED: lib().orc_stratified, MULTINOMIAL: lib().orc_multinomial, RESIDUAL: lib().orc_residual}[kind]
+    f(_ptr(w, _f64p), w.size, s1, _ptr(u, _f64p), _ptr(A, _i32p), C.byref(mg))
+    return A, mg.value
+
+
 def slot_map(A):
     A = np.ascontiguousarray(A, dtype=np.int32)
     m = np.zeros_like(A)
@@ -194,6 +219,10 @@ class Oracle:
     def reset(self, seed):
         self.seed = seed
         lib().orc_reset(self._h, seed)
+
+    def set_resampler(self, kind: int):
+        if lib().orc_set_resampler(self._h, kind):
+            raise ValueError("unknown resampling scheme")
 
     def step(self, logits, dtype=None, ld=None, force_tok=None, force_resample=None, force_anc=None):
         """logits: numpy [R, V] of float64 / float32, or uint16 holding bf16 bit patterns."""

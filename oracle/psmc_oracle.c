@@ -156,6 +156,90 @@ void orc_systematic(const double* w, int N, double s1, double u0, int32_t* A, do
     free(C);
 }
 
+/* ------------------------------------------------------------------ */
+/* the other unbiased schemes of Appendix E ("Resampling Choices")     */
+/* ------------------------------------------------------------------ */
+/* first index j whose inclusive prefix C_j reaches `level` (both in the units of C), N-1 if rounding leaves none */
+static int first_reaching(const double* C, int N, double level) {
+    for (int j = 0; j < N; ++j)
+        if (C[j] >= level) return j;
+    return N - 1;
+}
+static void note_margin(const double* C, int N, double total, int a, double p, double* mg) {
+    *mg = fmin(*mg, fabs(C[a] / total - p));
+    if (a > 0) *mg = fmin(*mg, fabs(p - C[a - 1] / total));
+}
+
+/* stratified: one position per stratum, p_i = (i + u_i) / N with its own uniform u_i */
+void orc_stratified(const double* w, int N, double s1, const double* u, int32_t* A, double* margin) {
+    double* C = (double*)malloc(sizeof(double) * (size_t)N);
+    double c = 0.0, mg = 1.0;
+    for (int j = 0; j < N; ++j) { c += w[j]; C[j] = c; }
+    for (int i = 0; i < N; ++i) {
+        double pos = (u[i] + (double)i) * s1; /* p_i * N * s1, compared with C_j * N as in the systematic scheme */
+        int a = N - 1;
+        for (int j = 0; j < N; ++j)
+            if (C[j] * (double)N >= pos) { a = j; break; }
+        A[i] = a;
+        note_margin(C, N, s1, a, (u[i] + (double)i) / (double)N, &mg);
+    }
+    if (margin) *margin = mg;
+    free(C);
+}
+
+/* multinomial: N independent draws from Categorical(W), p_i = u_i */
+void orc_multinomial(const double* w, int N, double s1, const double* u, int32_t* A, double* margin) {
+    double* C = (double*)malloc(sizeof(double) * (size_t)N);
+    double c = 0.0, mg = 1.0;
+    for (int j = 0; j < N; ++j) { c += w[j]; C[j] = c; }
+    for (int i = 0; i < N; ++i) {
+        int a = first_reaching(C, N, u[i] * s1);
+        A[i] = a;
+        note_margin(C, N, s1, a, u[i], &mg);
+    }
+    if (margin) *margin = mg;
+    free(C);
+}
+
+/* residual: floor(N W_j) copies of every j (in order of j), the remaining N - sum floors slots drawn
+ * independently from the residual weights N W_j - floor(N W_j); u_m is the uniform of the m-th such draw */
+void orc_residual(const double* w, int N, double s1, const double* u, int32_t* A, double* margin) {
+    double* Cr = (double*)malloc(sizeof(double) * (size_t)N);
+    double mg = 1.0, cr = 0.0;
+    int D = 0;
+    for (int j = 0; j < N; ++j) {
+        double x = (double)N * w[j] / s1; /* expected offspring */
+        double fl = floor(x);
+        int n = (int)fl;
+        mg = fmin(mg, fmin(x - fl, fl + 1.0 - x) / (double)N); /* how close the count is to flipping */
+        for (int k = 0; k < n && D < N; ++k) A[D++] = j;
+        cr += x - fl;
+        Cr[j] = cr;
+    }
+    for (int m = 0; D < N; ++m, ++D) {
+        int a = first_reaching(Cr, N, u[m] * cr);
+        A[D] = a;
+        if (cr > 0.0) note_margin(Cr, N, cr, a, u[m], &mg);
+    }
+    if (margin) *margin = mg;
+    free(Cr);
+}
+
+void orc_resample(int kind, const double* w, int N, double s1, uint64_t seed, uint64_t g, uint64_t t, int32_t* A,
+                  double* margin) {
+    if (kind == ORC_RESAMPLE_SYSTEMATIC) {
+        double u0 = orc_uniform(orc_hash5(seed, ORC_STREAM_RESAMPLE, g, t, 0));
+        orc_systematic(w, N, s1, u0, A, margin);
+        return;
+    }
+    double* u = (double*)malloc(sizeof(double) * (size_t)N);
+    for (int i = 0; i < N; ++i) u[i] = orc_uniform(orc_hash5(seed, ORC_STREAM_RESAMPLE, g, t, (uint64_t)(1 + i)));
+    if (kind == ORC_RESAMPLE_STRATIFIED) orc_stratified(w, N, s1, u, A, margin);
+    else if (kind == ORC_RESAMPLE_MULTINOMIAL) orc_multinomial(w, N, s1, u, A, margin);
+    else orc_residual(w, N, s1, u, A, margin);
+    free(u);
+}
+
 void orc_slot_map(const int32_t* A, int N, int32_t* map) {
     int* off = (int*)calloc((size_t)N, sizeof(int));
     for (int i = 0; i < N; ++i) off[A[i]] += 1;
@@ -177,7 +261,7 @@ void orc_slot_map(const int32_t* A, int N, int32_t* map) {
 /* particle system                                                     */
 /* ------------------------------------------------------------------ */
 struct orc_ctx {
-    int G, N, V, R, ramp, eos, T_max, t;
+    int G, N, V, R, ramp, eos, T_max, t, resampler;
     double alpha, tau, kappa;
     uint64_t seed;
     int32_t* prompt_len;
@@ -320,8 +404,7 @@ int orc_step(orc_ctx* c, const void* logits, int dtype, int64_t ld, const int32_
             for (int i = 0; i < N; ++i) { A[i] = i; A_own[i] = i; map[i] = i; }
         } else {
             for (int i = 0; i < N; ++i) w[i] = exp(lw[i] - M);
-            double u0 = orc_uniform(orc_hash5(c->seed, ORC_STREAM_RESAMPLE, (uint64_t)g, (uint64_t)t, 0));
-            orc_systematic(w, N, s1, u0, A_own, &c->anc_margin[g]);
+            orc_resample(c->resampler, w, N, s1, c->seed, (uint64_t)g, (uint64_t)t, A_own, &c->anc_margin[g]);
             if (force_anc && force_anc[(size_t)g * N] >= 0)
                 memcpy(A, force_anc + (size_t)g * N, sizeof(int32_t) * (size_t)N);
             else
@@ -422,6 +505,11 @@ const double* orc_log_inc(const orc_ctx* c) { return c->log_inc; }
 const double* orc_logp_tok(const orc_ctx* c) { return c->logp_tok; }
 const double* orc_cum_logp(const orc_ctx* c) { return c->S; }
 const int32_t* orc_ancestors(const orc_ctx* c) { return c->anc; }
+int orc_set_resampler(orc_ctx* c, int kind) {
+    if (kind < 0 || kind > 3) return 1;
+    c->resampler = kind;
+    return 0;
+}
 const int32_t* orc_anc_own(const orc_ctx* c) { return c->anc_own; }
 const double* orc_anc_margin(const orc_ctx* c) { return c->anc_margin; }
 const int32_t* orc_slot_map_view(const orc_ctx* c) { return c->map; }

@@ -59,6 +59,21 @@ void orc_ess(const double* logW, int N, double* M, double* s1, double* s2, doubl
  * |position - prefix| met at a deciding comparison (in normalised units). */
 void orc_systematic(const double* w, int N, double s1, double u0, int32_t* A, double* margin);
 
+/* ---- the other unbiased schemes named in Appendix E.  u[i]: independent uniforms in (0,1).
+ * stratified: position (i + u_i)/N in stratum i; multinomial: position u_i; residual: floor(N W_j) copies of
+ * every j, in order of j, then the remaining slots drawn independently from the residual weights
+ * N W_j - floor(N W_j) (u[m] for the m-th such slot).  Ancestors of multinomial and residual are not sorted.
+ * *margin: smallest distance met at a deciding comparison (normalised units; for residual also the distance of
+ * N W_j to the nearest whole number, over N). */
+enum { ORC_RESAMPLE_SYSTEMATIC = 0, ORC_RESAMPLE_STRATIFIED = 1, ORC_RESAMPLE_MULTINOMIAL = 2, ORC_RESAMPLE_RESIDUAL = 3 };
+void orc_stratified(const double* w, int N, double s1, const double* u, int32_t* A, double* margin);
+void orc_multinomial(const double* w, int N, double s1, const double* u, int32_t* A, double* margin);
+void orc_residual(const double* w, int N, double s1, const double* u, int32_t* A, double* margin);
+/* ancestors of group g at step t under scheme `kind`: systematic takes u0 = H(seed, 2, g, t, 0), the others
+ * u_i = H(seed, 2, g, t, 1 + i) */
+void orc_resample(int kind, const double* w, int N, double s1, uint64_t seed, uint64_t g, uint64_t t, int32_t* A,
+                  double* margin);
+
 /* ---- hazard-free slot map from ancestors: survivors stay, dead slots (in
  * increasing order) take the surplus offspring (sources in increasing order) */
 void orc_slot_map(const int32_t* A, int N, int32_t* map);
@@ -70,6 +85,7 @@ orc_ctx* orc_create(int G, int N, int V, double alpha, double tau, double kappa,
                     uint64_t seed, int eos, int T_max, const int32_t* prompt_len /* [G] or NULL */);
 void orc_destroy(orc_ctx*);
 void orc_reset(orc_ctx*, uint64_t seed);
+int orc_set_resampler(orc_ctx*, int kind); /* ORC_RESAMPLE_*; default systematic (Algorithm 1); 0 = ok */
 
 /* One token for every group.  logits: [G*N, V] row-major with row stride ld
  * elements, dtype ORC_*.  Hooks (each may be NULL): force_tok[G*N] (>=0 to

@@ -18,6 +18,7 @@ from . import build as _build
 OK, E_INVAL, E_NOMEM, E_CUDA, E_STATE, E_NUMERIC, E_TIMEOUT, E_HAZARD, E_TOO_LARGE = range(9)
 STATIC_SCRATCH_BYTES = 4 << 20
 F32, BF16 = 0, 1
+SYSTEMATIC, STRATIFIED, MULTINOMIAL, RESIDUAL = 0, 1, 2, 3
 
 _lib = None
 
@@ -52,6 +53,8 @@ def lib():
                                         C.c_int, C.c_uint64, C.c_int, C.c_int, C.POINTER(C.c_int32)]
         L.psmc_destroy.restype = C.c_int
         L.psmc_destroy.argtypes = [vp]
+        L.psmc_set_resampler.restype = C.c_int
+        L.psmc_set_resampler.argtypes = [vp, C.c_int]
         L.psmc_reset.restype = C.c_int
         L.psmc_reset.argtypes = [vp, C.c_uint64]
         L.psmc_step.restype = C.c_int
@@ -171,6 +174,10 @@ class Psmc:
             self.destroy()
         except Exception:
             pass
+
+    def set_resampler(self, kind: int) -> None:
+        """psmc_set_resampler: SYSTEMATIC (default), STRATIFIED, MULTINOMIAL or RESIDUAL."""
+        _check(lib().psmc_set_resampler(self._h, kind), "psmc_set_resampler")
 
     def reset(self, seed):
         _check(lib().psmc_reset(self._h, seed), "psmc_reset")

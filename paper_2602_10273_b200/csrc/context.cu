@@ -11,7 +11,7 @@ using namespace psmc;
 
 struct psmc_ctx {
     int device;
-    int G, N, V, R, ramp, eos, T_max, t;
+    int G, N, V, R, ramp, eos, T_max, t, resampler;
     double alpha, tau, kappa;
     uint64_t seed;
     int32_t* prompt_len_host;  // [G]
@@ -179,6 +179,12 @@ extern "C" psmc_status psmc_init(psmc_ctx** out, int N, int V, float alpha, floa
     return psmc_init_batched(out, 1, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, 4096, nullptr);
 }
 
+extern "C" psmc_status psmc_set_resampler(psmc_ctx* c, psmc_resampler kind) {
+    if (!c || (int)kind < 0 || (int)kind > 3) return PSMC_E_INVAL;
+    c->resampler = (int)kind;
+    return PSMC_OK;
+}
+
 extern "C" psmc_status psmc_destroy(psmc_ctx* c) {
     if (!c) return PSMC_E_INVAL;
     cudaDeviceSynchronize();
@@ -210,7 +216,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     la.zero_words = c->counts[(t + 1) & 1];  // each step clears the pair of move counters the next step will use
 
     WeightsArgs wa{};
-    wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos;
+    wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos; wa.resampler = c->resampler;
     wa.alpha_t = alpha_t; wa.beta = beta_t; wa.delta = alpha_t - alpha_prev; wa.kappa = c->kappa; wa.seed = c->seed;
     wa.logits = logits; wa.dt = dt; wa.V = c->V; wa.ld = ld; wa.scratch = c->scratch;
     wa.logp = c->logp; wa.loginc = c->loginc;

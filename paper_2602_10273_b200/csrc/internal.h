@@ -62,6 +62,7 @@ struct MoveSource {      // one surviving particle with surplus offspring
 };
 struct WeightsArgs {
     int G, N, R, t, eos;
+    int resampler;  // psmc_resampler
     double alpha_t, beta, delta, kappa;
     uint64_t seed;
     // the logit block of this step and the span triples the streaming kernel left

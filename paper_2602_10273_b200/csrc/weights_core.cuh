@@ -8,7 +8,8 @@
 //   live:  log W_r += log omega_r;  S_r += log p(y);  len_r += 1;  done_r |= (y == EOS)
 //   done:  y = EOS, factor 1
 //   w_i = exp(log W_i - max), C = inclusive prefix of w, ESS = (sum w)^2 / sum w^2.
-//   If ESS < kappa*N:  u0 = hash uniform, A_i = min{j : C_j * N >= (u0 + i) * C_{N-1}} (N-1 if none),
+//   If ESS < kappa*N:  u0 = hash uniform, A_i = min{j : C_j * N >= (u0 + i) * C_{N-1}} (N-1 if none)
+//   [systematic, the scheme of Algorithm 1; stratified, multinomial and residual resampling of Appendix E on request],
 //   offspring counts -> slot map (survivors stay; dead slots, in increasing order, take the surplus offspring,
 //   sources in increasing order), state gathered by the map, log W <- 0, log Z-hat += max + log(sum w / N).
 #pragma once
@@ -24,6 +25,7 @@ struct GroupScratch {
     int redi[33];
     double C[CAP];  // weight prefix
     double S[CAP];  // cumulative log p
+    double Rp[CAP];  // residual scheme: prefix of the residual weights
     int off[CAP];
     int Einc[CAP];
     int len[CAP];
@@ -107,13 +109,50 @@ __device__ __forceinline__ void group_update(const WeightsArgs& a, int g, int i,
     }
     group_sync(nw);
     int anc = N - 1;
-    if (on) {
-        const double u0 = hash_uniform(hash5(a.seed, kStreamResample, (uint64_t)g, (uint64_t)a.t, 0));
-        const double pos = (u0 + (double)i) * s1;
-        int lo = 0, hi = N;  // first j in [0,N) with C_j * N >= pos; C is non-decreasing
+    if (a.resampler == PSMC_RESAMPLE_RESIDUAL) {
+        // floor(N W_j) copies of every j in order of j, the rest drawn from the residual weights (Appendix E)
+        const double x = on ? (double)N * w / s1 : 0.0;
+        const double fl = floor(x);
+        int D;
+        double res_total;
+        const int d_incl = block_scan_incl(on ? (int)fl : 0, sc.redi, &D, nw);
+        const double r_incl = block_scan_incl(on ? x - fl : 0.0, sc.red, &res_total, nw);
+        if (on) {
+            sc.Einc[i] = d_incl;
+            sc.Rp[i] = r_incl;
+        }
+        group_sync(nw);
+        if (on) {
+            int lo = 0, hi = N;
+            if (i < D) {  // first j whose copies reach beyond position i
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sc.Einc[mid] > i) hi = mid; else lo = mid + 1;
+                }
+            } else {      // residual draw number i - D
+                const double level =
+                    hash_uniform(hash5(a.seed, kStreamResample, (uint64_t)g, (uint64_t)a.t, (uint64_t)(1 + i - D))) * res_total;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sc.Rp[mid] >= level) hi = mid; else lo = mid + 1;
+                }
+            }
+            anc = lo < N ? lo : N - 1;
+            atomicAdd(&sc.off[anc], 1);
+        }
+        group_sync(nw);  // Einc is written again below
+    } else if (on) {
+        // position of this particle against the weight prefix: first j with C_j * N >= pos (systematic, stratified)
+        // or C_j >= level (multinomial); C is non-decreasing
+        const bool multinomial = a.resampler == PSMC_RESAMPLE_MULTINOMIAL;
+        const uint64_t which = a.resampler == PSMC_RESAMPLE_SYSTEMATIC ? 0 : (uint64_t)(1 + i);
+        const double u = hash_uniform(hash5(a.seed, kStreamResample, (uint64_t)g, (uint64_t)a.t, which));
+        const double pos = multinomial ? u * s1 : (u + (double)i) * s1;
+        const double scale = multinomial ? 1.0 : (double)N;
+        int lo = 0, hi = N;
         while (lo < hi) {
             const int mid = (lo + hi) >> 1;
-            if (sc.C[mid] * (double)N >= pos) hi = mid; else lo = mid + 1;
+            if (sc.C[mid] * scale >= pos) hi = mid; else lo = mid + 1;
         }
         anc = lo < N ? lo : N - 1;
         atomicAdd(&sc.off[anc], 1);

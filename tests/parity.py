@@ -46,7 +46,8 @@ def logits_to_numpy(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy()
 
 
-def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp: int = None, kappa: float = None):
+def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp: int = None, kappa: float = None,
+              resampler: int = 0):
     G = cfg.G if G is None else G
     T_max = cfg.T if T_max is None else T_max
     ramp = cfg.ramp if ramp is None else ramp
@@ -56,6 +57,8 @@ def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp
                 prompt_len=wl.prompt_len)
     orc = O.Oracle(cfg.N, cfg.V, float(np.float32(cfg.alpha)), float(np.float32(cfg.tau)), float(np.float32(kappa)),
                    ramp, seed, cfg.eos_id, G=G, T_max=T_max, prompt_len=wl.prompt_len)
+    ps.set_resampler(resampler)
+    orc.set_resampler(resampler)
     return wl, ps, orc
 
 
@@ -117,10 +120,10 @@ def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, 
 
 
 def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = None, kappa: float = None,
-                kv_shape=None, logit_bias_fn=None) -> LoopStats:
+                kv_shape=None, logit_bias_fn=None, resampler: int = 0) -> LoopStats:
     """Run T tokens on both sides.  kv_shape=(layers, heads, max_len, dim) also carries a KV cache
     through every reindex on both sides and compares the whole buffers at the end."""
-    wl, ps, orc = make_pair(cfg, seed, G=G, T_max=T, ramp=ramp, kappa=kappa)
+    wl, ps, orc = make_pair(cfg, seed, G=G, T_max=T, ramp=ramp, kappa=kappa, resampler=resampler)
     kappa_f = float(np.float32(cfg.kappa if kappa is None else kappa))
     st = LoopStats()
     lg = wl.new_logits()

@@ -123,13 +123,16 @@ def test_logits_pass_token_independence_on_device():
 
 
 # ------------------------------------------------------------------ weights / ESS / resampling on identical state
+@pytest.mark.parametrize("resampler", [B.SYSTEMATIC, B.STRATIFIED, B.MULTINOMIAL, B.RESIDUAL])
 @pytest.mark.parametrize("N", [1, 2, 4, 8, 32, 33, 100, 1024])
-def test_resampling_kernel_bit_exact_on_identical_log_weights(N):
+def test_resampling_kernel_bit_exact_on_identical_log_weights(N, resampler):
     rng = np.random.default_rng(N)
     V, G = 64, 3
     for trial in range(4):
         ps = B.Psmc(N, V, 2.0, 0.5, 1.0, 0, 11 + trial, V - 1, G=G, T_max=4, prompt_len=[5, 6, 7])
         orc = O.Oracle(N, V, 2.0, 0.5, 1.0, 0, 11 + trial, V - 1, G=G, T_max=4, prompt_len=[5, 6, 7])
+        ps.set_resampler(resampler)
+        orc.set_resampler(resampler)
         lw = rng.normal(0, 2.0 + trial, size=G * N)
         lw[N:2 * N] = -1.25                                # group 1: uniform weights, must not resample
         S = rng.normal(-3, 1, size=G * N)
@@ -141,7 +144,13 @@ def test_resampling_kernel_bit_exact_on_identical_log_weights(N):
         orc.step(logits.cpu().numpy(), force_tok=ps.tokens.numpy())
         assert ps.sync_status() == B.OK
         assert np.array_equal(ps.resampled.numpy(), orc.resampled) and orc.resampled[1] == 0
-        assert np.array_equal(ps.ancestors.numpy(), orc.ancestors)
+        if not np.array_equal(ps.ancestors.numpy(), orc.ancestors):
+            # only where the oracle itself reports a position within rounding of a weight prefix (the CUDA prefix
+            # is summed in another order) may the two differ
+            bad = np.nonzero((ps.ancestors.numpy() != orc.ancestors).reshape(G, N).any(axis=1))[0]
+            assert all(orc.anc_margin[g] <= 1e-12 for g in bad), (bad, orc.anc_margin)
+            ps.destroy()
+            continue                                       # a genuine tie: nothing further to compare in this trial
         assert np.array_equal(ps.slot_map.numpy(), orc.slot_map)
         assert np.array_equal(ps.lens.numpy(), orc.lens)
         assert np.allclose(ps.ess.numpy(), orc.ess, rtol=1e-12)
@@ -163,6 +172,19 @@ def test_closed_loop_tiny_full():
 def test_closed_loop_tiny_other_seeds(seed):
     c = W.CONFIGS["tiny"]
     P.closed_loop(c, seed=seed, T=c.T, kv_shape=(c.n_layers, c.n_kv_heads, c.max_len, c.head_dim))
+
+
+@pytest.mark.parametrize("resampler", [B.STRATIFIED, B.MULTINOMIAL, B.RESIDUAL])
+def test_closed_loop_other_resamplers(resampler):
+    c = W.CONFIGS["tiny"]
+    st = P.closed_loop(c, seed=4, T=c.T, kv_shape=(c.n_layers, c.n_kv_heads, c.max_len, c.head_dim), resampler=resampler)
+    assert st.resample_events > 0 and st.slots_moved > 0
+    c = W.CONFIGS["resample_stress"]
+    st = P.closed_loop(c, seed=3, T=24, ramp=8, resampler=resampler)
+    assert st.resample_events >= 5
+    c = W.CONFIGS["batched_prompts"]
+    st = P.closed_loop(c, seed=2, T=12, G=4, resampler=resampler)
+    assert st.resample_events > 0
 
 
 def test_closed_loop_llama_shape():
@@ -195,6 +217,15 @@ def test_closed_loop_batched_prompts():
     st = P.closed_loop(c, seed=1, T=24, G=8, kv_shape=(1, 2, 256 + 24 + 8, c.head_dim))
     assert st.resample_events > 0
     print("batched_prompts (8 prompts):", st)
+
+
+def test_closed_loop_batched_prompts_full_size():
+    """All 64 prompts x 8 particles x 128256 logits, i.e. the launch configuration the benchmark times (two kernels,
+    148 CTAs), every row compared with the oracle; the cache carries every head and position of one layer."""
+    c = W.CONFIGS["batched_prompts"]
+    st = P.closed_loop(c, seed=1, T=5, kv_shape=(1, c.n_kv_heads, c.max_len, c.head_dim))
+    assert st.live_rows == 5 * 512 and st.resample_events > 0 and st.slots_moved > 0
+    print("batched_prompts (64 prompts, full size):", st)
 
 
 def test_eos_rows_freeze_and_are_not_read():

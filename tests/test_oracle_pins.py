@@ -165,6 +165,83 @@ def test_systematic_resampling_hand_example():
     assert mg == pytest.approx(0.025, abs=1e-12)  # |0.625 - 0.6| and |0.125 - 0.1| are the closest calls
 
 
+# ---------------------------------------------------------------- the other schemes of Appendix E
+def test_other_resamplers_hand_example():
+    # weights .1 .5 .05 .35 -> prefix .1 .6 .65 1 ; uniforms .3 .9 .2 .6
+    w, u = np.array([0.1, 0.5, 0.05, 0.35]), np.array([0.3, 0.9, 0.2, 0.6])
+    A, mg = O.resample(O.STRATIFIED, w, u)           # positions .075 .475 .55 .9
+    assert A.tolist() == [0, 1, 1, 3] and mg == pytest.approx(0.025, abs=1e-12)
+    A, mg = O.resample(O.MULTINOMIAL, w, u)          # positions .3 .9 .2 .6 ; .6 sits exactly on the prefix .6
+    assert A.tolist() == [1, 3, 1, 1] and mg == pytest.approx(0.0, abs=1e-15)
+    # N W = .4 2 .2 1.4 -> two copies of 1, one of 3, one slot left; residual weights .4 0 .2 .4, first uniform .3
+    A, _ = O.resample(O.RESIDUAL, w, u)
+    assert A.tolist() == [1, 1, 3, 0]
+
+
+@pytest.mark.parametrize("N", [1, 2, 5, 32, 257])
+def test_other_resamplers_against_library_search(N):
+    rng = np.random.default_rng(100 + N)
+    for trial in range(20):
+        w = rng.exponential(size=N) ** 3
+        u = np.array([O.uniform(O.hash5(2, O.STREAM_RESAMPLE, 0, trial, 1 + i)) for i in range(N)])
+        W = w / w.sum()
+        cdf = np.cumsum(w) / w.sum()
+        A, _ = O.resample(O.STRATIFIED, w, u)
+        assert np.array_equal(A, np.minimum(np.searchsorted(cdf, (np.arange(N) + u) / N, side="left"), N - 1))
+        assert np.all(np.diff(A) >= 0)
+        off = np.bincount(A, minlength=N)
+        assert np.all(np.abs(off - N * W) < 2.0)      # stratified counts stay within two of their mean
+        A, _ = O.resample(O.MULTINOMIAL, w, u)
+        assert np.array_equal(A, np.minimum(np.searchsorted(cdf, u, side="left"), N - 1))
+        A, _ = O.resample(O.RESIDUAL, w, u)
+        fl = np.floor(N * W + 1e-12).astype(int)
+        D = int(fl.sum())
+        assert np.array_equal(A[:D], np.repeat(np.arange(N), fl))      # the deterministic copies, in order
+        res = N * W - fl
+        if D < N:
+            rc = np.cumsum(res) / res.sum()
+            assert np.array_equal(A[D:], np.minimum(np.searchsorted(rc, u[: N - D], side="left"), N - 1))
+        assert np.all(np.bincount(A, minlength=N) >= fl)
+
+
+@pytest.mark.parametrize("kind", [O.SYSTEMATIC, O.STRATIFIED, O.MULTINOMIAL, O.RESIDUAL])
+def test_every_resampler_is_unbiased(kind):
+    """E[offspring of j] = N W_j (the property Appendix E asks of a resampling scheme), by Monte Carlo."""
+    w = np.array([0.03, 0.4, 0.07, 0.25, 0.2, 0.05])
+    N, n = w.size, 20000
+    counts = np.zeros((n, N))
+    for s in range(n):
+        if kind == O.SYSTEMATIC:
+            A, _ = O.systematic(w, O.uniform(O.hash5(7, O.STREAM_RESAMPLE, 0, s, 0)))
+        else:
+            A, _ = O.resample(kind, w, [O.uniform(O.hash5(7, O.STREAM_RESAMPLE, 0, s, 1 + i)) for i in range(N)])
+        counts[s] = np.bincount(A, minlength=N)
+    sem = counts.std(axis=0, ddof=1) / math.sqrt(n)
+    assert np.all(np.abs(counts.mean(axis=0) - N * w / w.sum()) < 4.0 * sem + 1e-9)
+
+
+@pytest.mark.parametrize("kind", [O.STRATIFIED, O.MULTINOMIAL, O.RESIDUAL])
+def test_normaliser_estimate_is_unbiased_under_every_resampler(kind):
+    V, T, alpha = 3, 4, 4.0
+    lm = TinyLM(V, 55)
+    _, gam = lm.enumerate(T, alpha, V - 1)
+    Z = gam.sum()
+    n = 12000
+    o = O.Oracle(N=4, V=V, alpha=alpha, tau=1.0 / alpha, kappa=0.9, ramp=0, seed=0, eos=V - 1, T_max=T)
+    o.set_resampler(kind)
+    zs = np.empty(n)
+    resamples = 0
+    for s in range(n):
+        o.reset(5000 + s)
+        for _ in range(T):
+            o.step(lm.logits(o.last_tokens))
+            resamples += int(o.resampled[0])
+        zs[s] = math.exp(o.log_z_final[0])
+    assert resamples > n // 20
+    sem = zs.std(ddof=1) / math.sqrt(n)
+    assert abs(zs.mean() - Z) < 4.0 * sem + 1e-12, (zs.mean(), Z, sem)
+
+
 def test_slot_map_properties_and_hand_examples():
     assert O.slot_map([1, 2, 3, 3]).tolist() == [3, 1, 2, 3]
     assert O.slot_map([0, 0, 0, 0]).tolist() == [0, 0, 0, 0]
