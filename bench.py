@@ -108,11 +108,14 @@ def logits_to_numpy(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy()
 
 
-def moved_bytes(slot_map, lens, G, N, bytes_per_pos):
+def moved_bytes(slot_map, lens, G, N, bytes_per_pos, skip=None):
     """Algorithmic bytes of one KV reindex: each source with surplus offspring is read once, each rewritten slot
-    written once; lens are the post-step live lengths (a rewritten slot carries its source's length)."""
+    written once; lens are the post-step live lengths (a rewritten slot carries its source's length).  skip [G]:
+    positions at the start of every row of the group that stay in place (a prompt shared by the group)."""
     m = slot_map.reshape(G, N)
     ln = lens.reshape(G, N)
+    if skip is not None:
+        ln = np.maximum(ln - np.asarray(skip).reshape(G, 1), 0)
     moved = m != np.arange(N)[None, :]
     wr = int(ln[moved].sum())
     rd = 0
@@ -155,7 +158,8 @@ def run_ours(args):
     ks, vs = wl.new_kv()
     ps = B.Psmc(N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=G, T_max=T_total,
                 prompt_len=wl.prompt_len)
-    desc = ps.make_kv_desc(ks, vs)
+    desc = ps.make_kv_desc(ks, vs, skip_shared_prompt=args.skip_shared_prompt)
+    skip = wl.prompt_len if args.skip_shared_prompt else None
     last = ps.device_view("psmc_last_tokens", R)
 
     # logit blocks: generated along a short closed loop, then reused cyclically by every pass below
@@ -178,7 +182,7 @@ def run_ours(args):
     for t in range(1, T_total + 1):
         live_rows.append(R - int(ps.done.numpy().sum()))  # rows that are live when step t starts
         one_pass(1, t)
-        b, mv = moved_bytes(ps.slot_map.numpy(), ps.lens.numpy(), G, N, cfg.kv_bytes_per_pos_per_row)
+        b, mv = moved_bytes(ps.slot_map.numpy(), ps.lens.numpy(), G, N, cfg.kv_bytes_per_pos_per_row, skip)
         kv_bytes.append(b)
         moved_slots.append(mv)
     assert ps.sync_status() == B.OK
@@ -275,6 +279,7 @@ def run_ours(args):
                    "prompts_per_gpu": G, "rows_per_gpu": R, "alpha": cfg.alpha, "tau": cfg.tau, "kappa": cfg.kappa,
                    "ramp": cfg.ramp, "l2": "inputs larger than L2: %d logit blocks of %.0f MB rotated, KV %.1f GB" % (
                        N_BLOCKS, R * cfg.logit_bytes_per_row / 1e6, G * per_group / 1e9),
+                   "kv_reindex": "prompt positions left in place" if args.skip_shared_prompt else "whole live prefix copied",
                    "parallelism": "replicas only (prompts sharded, no collective)"},
         "clocks": clk.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": R * cfg.logit_bytes_per_row,
@@ -397,6 +402,9 @@ def main():
     ap.add_argument("--groups", type=int, default=None, help="override the number of prompts (default: the workload's)")
     ap.add_argument("--e2e-steps", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-shared-prompt", action="store_true",
+                    help="supplementary run: the KV reindex leaves each group's prompt positions in place (not the "
+                         "headline configuration, which copies whole live prefixes)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps

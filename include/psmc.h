@@ -176,6 +176,7 @@ typedef struct {
     psmc_dtype dt;
     int64_t stride_row;    /* elements between rows (particles)                    */
     int64_t stride_head;   /* elements between heads; (position, dim) is contiguous */
+    int skip_shared_prompt; /* src only, step maps only: nonzero = leave positions below the group's prompt length alone */
 } psmc_kv_desc;
 
 /* Applies the slot map of the most recent step to caller-owned caches: for
@@ -191,6 +192,10 @@ typedef struct {
  *     PSMC_E_HAZARD is raised in the status word and nothing is written.
  *   dst != NULL: out-of-place gather dst[k] = src[idx[k]] for every k (also
  *     idx[k]==k), i.e. index_select on the particle dimension.
+ * src->skip_shared_prompt: all particles of a group start from the same prompt, so the first prompt_len positions
+ *   of their rows hold the same keys and values; when the caller vouches for that (the rows were prefilled with one
+ *   prompt per group) the copy of a row starts at the group's prompt length given to psmc_init_batched and only
+ *   generated positions move.  Ignored with idx_override.
  * The bulk-copy (TMA) path needs 16-byte aligned row/head starts and
  * head_dim*sizeof(elem) a multiple of 16; otherwise a plain-load path runs. */
 psmc_status psmc_reindex_kv(psmc_ctx*, const psmc_kv_desc* src, const psmc_kv_desc* dst,

@@ -82,7 +82,7 @@ def lib():
         L.orc_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, _i32p, _i32p, _i32p]
         L.orc_reindex_tensor.restype = None
         L.orc_reindex_tensor.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
-                                         C.c_int, C.c_int64, C.c_int64, _i32p, _i32p]
+                                         C.c_int, C.c_int64, C.c_int64, _i32p, _i32p, _i32p]
         L.orc_select.restype = None
         L.orc_select.argtypes = [C.c_void_p, _i32p, _i32p, _i32p]
         L.orc_t.restype = C.c_int
@@ -190,14 +190,16 @@ def slot_map(A):
     return m
 
 
-def reindex_tensor(dst, src, idx, copy_len=None):
-    """dst/src: C-contiguous numpy arrays [R, H, max_len, D]; in place when they are the same array."""
+def reindex_tensor(dst, src, idx, copy_len=None, copy_from=None):
+    """dst/src: C-contiguous numpy arrays [R, H, max_len, D]; in place when they are the same array.
+    Row k receives positions [copy_from[k], copy_len[k]) of row idx[k] (defaults 0 and max_len)."""
     R, H, max_len, D = src.shape
     assert src.flags.c_contiguous and dst.flags.c_contiguous and dst.shape == src.shape
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     cl = None if copy_len is None else np.ascontiguousarray(copy_len, dtype=np.int32)
+    cf = None if copy_from is None else np.ascontiguousarray(copy_from, dtype=np.int32)
     lib().orc_reindex_tensor(dst.ctypes.data, src.ctypes.data, R, H, max_len, D, src.itemsize,
-                             H * max_len * D, max_len * D, _ptr(idx, _i32p), _ptr(cl, _i32p))
+                             H * max_len * D, max_len * D, _ptr(idx, _i32p), _ptr(cl, _i32p), _ptr(cf, _i32p))
 
 
 class Oracle:

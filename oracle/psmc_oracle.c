@@ -435,17 +435,19 @@ int orc_step(orc_ctx* c, const void* logits, int dtype, int64_t ld, const int32_
 
 void orc_reindex_tensor(void* dst, const void* src, int R, int H, int max_len, int D, int elem_size,
                         int64_t stride_row, int64_t stride_head, const int32_t* idx,
-                        const int32_t* copy_len) {
+                        const int32_t* copy_len, const int32_t* copy_from) {
     const int in_place = (dst == src);
     for (int k = 0; k < R; ++k) {
         if (in_place && idx[k] == k) continue;
         int n = copy_len ? copy_len[k] : max_len;
         if (n > max_len) n = max_len;
-        if (n <= 0) continue;
+        int f = copy_from ? copy_from[k] : 0; /* positions below f are left alone */
+        if (f < 0) f = 0;
+        if (n <= f) continue;
         for (int h = 0; h < H; ++h) {
-            const char* s = (const char*)src + ((int64_t)idx[k] * stride_row + (int64_t)h * stride_head) * elem_size;
-            char* d = (char*)dst + ((int64_t)k * stride_row + (int64_t)h * stride_head) * elem_size;
-            memcpy(d, s, (size_t)n * (size_t)D * (size_t)elem_size);
+            const char* s = (const char*)src + ((int64_t)idx[k] * stride_row + (int64_t)h * stride_head + (int64_t)f * D) * elem_size;
+            char* d = (char*)dst + ((int64_t)k * stride_row + (int64_t)h * stride_head + (int64_t)f * D) * elem_size;
+            memcpy(d, s, (size_t)(n - f) * (size_t)D * (size_t)elem_size);
         }
     }
 }

@@ -99,11 +99,12 @@ int orc_step(orc_ctx*, const void* logits, int dtype, int64_t ld, const int32_t*
  * element, strides in elements; row k receives row idx[k] over positions
  * [0, copy_len[k]) (copy_len[k] = live length of the SOURCE row, which after
  * orc_step is the length recorded for slot k; NULL = max_len everywhere); the
- * rest of row k is left alone.  In place when dst == src: rows with idx[k]==k
+ * rest of row k is left alone.  copy_from[k] (NULL = 0): positions below it are left alone too -- the form for
+ * caches whose first positions (a prompt shared by the whole group) are the same in every row.  In place when dst == src: rows with idx[k]==k
  * are skipped and idx must be hazard-free (no row both read and written). */
 void orc_reindex_tensor(void* dst, const void* src, int R, int H, int max_len, int D,
                         int elem_size, int64_t stride_row, int64_t stride_head,
-                        const int32_t* idx, const int32_t* copy_len);
+                        const int32_t* idx, const int32_t* copy_len, const int32_t* copy_from);
 
 /* Final draw I ~ Categorical(W_T) per group and back-trace of its tokens. */
 void orc_select(orc_ctx*, int32_t* out_tokens /* [G, T_max] */, int32_t* out_len /* [G] */,

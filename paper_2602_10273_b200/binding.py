@@ -33,7 +33,7 @@ class PsmcError(RuntimeError):
 class KvDesc(C.Structure):
     _fields_ = [("n_layers", C.c_int), ("k", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)),
                 ("n_kv_heads", C.c_int), ("head_dim", C.c_int), ("max_len", C.c_int), ("dt", C.c_int),
-                ("stride_row", C.c_int64), ("stride_head", C.c_int64)]
+                ("stride_row", C.c_int64), ("stride_head", C.c_int64), ("skip_shared_prompt", C.c_int)]
 
 
 def lib():
@@ -195,8 +195,9 @@ class Psmc:
         _check(lib().psmc_step_host(self._h, logits.data_ptr(), _dtype_code(logits), logits.stride(0),
                                     tokens_out.data_ptr(), _stream(stream)), "psmc_step_host")
 
-    def make_kv_desc(self, k_layers, v_layers):
-        """k_layers / v_layers: lists of CUDA tensors [R, H, max_len, D] with (max_len, D) contiguous."""
+    def make_kv_desc(self, k_layers, v_layers, skip_shared_prompt: bool = False):
+        """k_layers / v_layers: lists of CUDA tensors [R, H, max_len, D] with (max_len, D) contiguous.
+        skip_shared_prompt: the rows of a group hold the same prompt positions, which then stay where they are."""
         k0 = k_layers[0]
         R, H, L, D = k0.shape
         assert R == self.R and k0.stride(3) == 1 and k0.stride(2) == D
@@ -206,7 +207,7 @@ class Psmc:
         for t in list(k_layers) + list(v_layers):
             assert t.shape == k0.shape and t.stride() == k0.stride() and t.dtype == k0.dtype and t.is_cuda
         d = KvDesc(n, C.cast(ka, C.POINTER(C.c_void_p)), C.cast(va, C.POINTER(C.c_void_p)), H, D, L,
-                   _dtype_code(k0), k0.stride(0), k0.stride(1))
+                   _dtype_code(k0), k0.stride(0), k0.stride(1), 1 if skip_shared_prompt else 0)
         d._keep = (ka, va, list(k_layers), list(v_layers))
         return d
 

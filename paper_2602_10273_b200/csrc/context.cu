@@ -15,6 +15,7 @@ struct psmc_ctx {
     double alpha, tau, kappa;
     uint64_t seed;
     int32_t* prompt_len_host;  // [G]
+    int32_t* prompt_len_dev;   // [G] the same on the device (for the shared-prompt form of the KV reindex)
     // particle state
     double *logW, *S;
     uint8_t* done;
@@ -120,7 +121,7 @@ void free_ctx(psmc_ctx* c) {
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
-                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging};
+                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete[] c->prompt_len_host;
@@ -163,6 +164,8 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     }
     for (int s = 0; s < 3; ++s) ok(dev_alloc(&c->counts[s], 2));
     ok(dev_alloc(&c->row_arrivals, R)); ok(dev_alloc(&c->group_arrivals, (size_t)G));
+    ok(dev_alloc(&c->prompt_len_dev, (size_t)G));
+    if (e == cudaSuccess) e = cudaMemcpy(c->prompt_len_dev, c->prompt_len_host, 4 * (size_t)G, cudaMemcpyHostToDevice);
     ok(dev_alloc(&c->status, 1));
     ok(dev_alloc(&c->kv_work, 2));
     ok(cudaMalloc(&c->scratch, logits_pass_scratch_bytes(c->R, c->V)));
@@ -306,6 +309,8 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
     k.n_sources = idx_override ? c->counts[2] : c->counts[c->t & 1];
     k.status = c->status;
     k.work = c->kv_work;
+    k.skip_pos = (!idx_override && src->skip_shared_prompt) ? c->prompt_len_dev : nullptr;
+    k.N = c->N;
     uint64_t bits = (uint64_t)k.row_bytes_stride | (uint64_t)k.head_bytes_stride | (uint64_t)k.dst_row_bytes_stride |
                     (uint64_t)k.dst_head_bytes_stride | (uint64_t)k.pos_bytes;
     for (int l = 0; l < src->n_layers; ++l) {

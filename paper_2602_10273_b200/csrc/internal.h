@@ -118,6 +118,8 @@ struct KvLaunch {
     const int32_t* dst_rows;
     const int32_t* n_sources;
     int32_t* status;
+    const int32_t* skip_pos;  // [G] positions at the start of every row of group g that are not copied, or NULL
+    int N;                    // particles per group (rows per entry of skip_pos)
     int32_t* work;   // [2] unit queue of the copy kernels: next unit, CTAs that have left; both zero between launches
     int bulk_ok;     // 16-byte alignment holds everywhere
 };

@@ -44,13 +44,15 @@ __device__ __forceinline__ void open_unit(const KvLaunch& k, int u, int n_seg, U
     const int s = u / n_seg, seg = u - s * n_seg;
     const MoveSource ms = k.sources[s];
     const int len = ms.len < k.max_len ? ms.len : k.max_len;
+    int skip = k.skip_pos ? k.skip_pos[ms.src_row / k.N] : 0;  // a prompt shared by the group stays where it is
+    skip = skip < 0 ? 0 : (skip > len ? len : skip);
     c.seg_ptr = seg / k.H;
     c.seg_head = seg - c.seg_ptr * k.H;
     c.dst_begin = ms.dst_begin;
     c.n_dst = ms.n_dst;
     c.src = k.src[c.seg_ptr] + (int64_t)ms.src_row * k.row_bytes_stride + (int64_t)c.seg_head * k.head_bytes_stride;
     c.seg_bytes = (int64_t)(len > 0 ? len : 0) * k.pos_bytes;
-    c.off = 0;
+    c.off = (int64_t)skip * k.pos_bytes;
 }
 __device__ __forceinline__ void take_chunk(UnitCursor& c, Item& it) {
     it.src = c.src + c.off;
@@ -170,7 +172,7 @@ __global__ void __launch_bounds__(256) reindex_plain_kernel(const __grid_constan
         it.seg_ptr = c.seg_ptr; it.seg_head = c.seg_head; it.dst_begin = c.dst_begin; it.n_dst = c.n_dst; it.dst_off = 0;
         const int64_t n_units_u = c.seg_bytes / (int64_t)sizeof(U);
         const U* s = reinterpret_cast<const U*>(c.src);
-        for (int64_t e = threadIdx.x; e < n_units_u; e += blockDim.x) {
+        for (int64_t e = c.off / (int64_t)sizeof(U) + threadIdx.x; e < n_units_u; e += blockDim.x) {
             const U v = s[e];
             for (int d = 0; d < it.n_dst; ++d) reinterpret_cast<U*>(dst_addr(k, it, d))[e] = v;
         }

@@ -120,7 +120,7 @@ def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, 
 
 
 def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = None, kappa: float = None,
-                kv_shape=None, logit_bias_fn=None, resampler: int = 0) -> LoopStats:
+                kv_shape=None, logit_bias_fn=None, resampler: int = 0, skip_shared_prompt: bool = False) -> LoopStats:
     """Run T tokens on both sides.  kv_shape=(layers, heads, max_len, dim) also carries a KV cache
     through every reindex on both sides and compares the whole buffers at the end."""
     wl, ps, orc = make_pair(cfg, seed, G=G, T_max=T, ramp=ramp, kappa=kappa, resampler=resampler)
@@ -137,9 +137,18 @@ def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = N
         for l in range(L):
             WC.fill_kv(ks[l], seed, l, 0)
             WC.fill_kv(vs[l], seed, l, 1)
-        desc = ps.make_kv_desc(ks, vs)
+        copy_from = None
+        if skip_shared_prompt:  # a group's rows were prefilled with one prompt: the same keys and values below its length
+            for g in range(ps.G):
+                pl = int(wl.prompt_len[g])
+                for t_ in ks + vs:
+                    t_[g * ps.N:(g + 1) * ps.N, :, :pl, :] = t_[g * ps.N, :, :pl, :].clone()
+            copy_from = np.repeat(wl.prompt_len, ps.N).astype(np.int32)
+        desc = ps.make_kv_desc(ks, vs, skip_shared_prompt=skip_shared_prompt)
         as_np = lambda t: (t.view(torch.int16) if t.dtype == torch.bfloat16 else t).cpu().numpy()
-        kv = dict(desc=desc, ks=ks, vs=vs, host=[as_np(t).copy() for t in ks + vs], as_np=as_np)
+        kv = dict(desc=desc, ks=ks, vs=vs, host=[as_np(t).copy() for t in ks + vs], as_np=as_np, copy_from=copy_from)
+        if skip_shared_prompt:  # second mirror moved in full: with shared prompts both forms give the same cache
+            kv["host_full"] = [h.copy() for h in kv["host"]]
     last_view = ps.device_view("psmc_last_tokens", ps.R)
     for t in range(1, T + 1):
         wl.fill(lg, t, prev)
@@ -153,11 +162,15 @@ def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = N
             m = orc.slot_map.reshape(ps.G, ps.N) + (np.arange(ps.G) * ps.N)[:, None]
             idx, ln = m.reshape(-1).astype(np.int32), orc.lens
             for h in kv["host"]:
+                O.reindex_tensor(h, h, idx, ln, kv["copy_from"])
+            for h in kv.get("host_full", []):
                 O.reindex_tensor(h, h, idx, ln)
         prev.copy_(last_view)
     if kv is not None:
         for dev, host in zip(kv["ks"] + kv["vs"], kv["host"]):
             assert np.array_equal(kv["as_np"](dev), host), "KV cache differs after the reindexes"
+        for full, host in zip(kv.get("host_full", []), kv["host"]):
+            assert np.array_equal(full, host), "leaving the shared prompt in place changed the cache"
     # final draw and back-trace
     toks, ln, ix = ps.select()
     o_toks, o_ln, o_ix = orc.select()

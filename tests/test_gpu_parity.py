@@ -228,6 +228,15 @@ def test_closed_loop_batched_prompts_full_size():
     print("batched_prompts (64 prompts, full size):", st)
 
 
+@pytest.mark.parametrize("name,G,T", [("batched_prompts", 6, 16), ("tiny", None, 48)])
+def test_reindex_leaves_a_shared_prompt_in_place(name, G, T):
+    """Rows of a group prefilled with one prompt: only generated positions move, and the cache ends up as if whole
+    live prefixes had been copied."""
+    c = W.CONFIGS[name]
+    st = P.closed_loop(c, seed=2, T=T, G=G, kv_shape=(2, 2, c.prompt_hi + T + 8, c.head_dim), skip_shared_prompt=True)
+    assert st.slots_moved > 0
+
+
 def test_eos_rows_freeze_and_are_not_read():
     c = W.CONFIGS["tiny"]
 

@@ -525,3 +525,13 @@ def test_reindex_is_index_select_on_the_particle_dimension():
             want[k, :, : lens[k]] = src[m[k], :, : lens[k]]
     assert np.array_equal(buf, want)
     assert np.array_equal(buf[0, :, 7:], src[0, :, 7:]) and not np.array_equal(buf[0], src[0])
+    # positions below copy_from stay as well: the form for rows that share a prompt
+    start = np.array([3, 3, 3, 2, 2, 0], dtype=np.int32)
+    buf = src.copy()
+    O.reindex_tensor(buf, buf, m, lens, start)
+    want = src.copy()
+    for k in range(R):
+        if m[k] != k:
+            want[k, :, start[k]: lens[k]] = src[m[k], :, start[k]: lens[k]]
+    assert np.array_equal(buf, want)
+    assert np.array_equal(buf[0, :, :3], src[0, :, :3]) and np.array_equal(buf[0, :, 3:7], src[1, :, 3:7])
