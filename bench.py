@@ -2,7 +2,7 @@
 """Benchmark of the Power-SMC hot path on B200: one "step" = one decoded token for every particle =
 logit pass + weights/ESS/resampling + KV-cache reindex, on synthetic inputs shaped like the paper's.
 
-  python bench.py --gpus 1 --steps 256 --warmup 8            # this repository's CUDA path
+  python bench.py --gpus 1 --steps 1016 --warmup 8           # this repository's CUDA path (the defaults)
   python bench.py --impl reference --steps 3 --warmup 1      # the CPU oracle as the reference arm
 
 Prints ONE JSON line.  `value` is particle-tokens/s with every input resident in HBM; `e2e` is the
@@ -411,7 +411,7 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
     else:
-        args.steps = 256 if args.steps is None else args.steps
+        args.steps = 1016 if args.steps is None else args.steps  # with the warm-up: all 1024 tokens of the workload
         args.warmup = 8 if args.warmup is None else args.warmup
         if args.warmup < 3:
             args.warmup = 3
