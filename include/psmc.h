@@ -241,10 +241,12 @@ int psmc_rows(const psmc_ctx*);              /* R                               
 psmc_status psmc_set_state(psmc_ctx*, const double* log_w, const double* cum_logp,
                            const uint8_t* done, const int32_t* lens);
 
-/* Profiling aid.  While enabled, every kernel launched by psmc_step / psmc_step_host /
- * psmc_reindex_kv is bracketed by CUDA events on the caller's stream.  psmc_timing_read waits for
- * the recorded events, adds up the device time per kernel (HOST arrays of 3: [0] logit pass,
- * [1] weights/ESS/resampling, [2] KV reindex; milliseconds and launch counts) and clears the record. */
+/* Profiling aid.  on = 1: every kernel launched by psmc_step / psmc_step_host / psmc_reindex_kv is bracketed by
+ * CUDA events on the caller's stream.  on = 2: one bracket around the kernels of a psmc_step (they then keep
+ * their chained launches) and one around every reindex kernel.  on = 0: off.  psmc_timing_read waits for the
+ * recorded events, adds up the device time per bracket kind (HOST arrays of 3: [0] logit pass, or with on = 2 the
+ * whole step; [1] weights/ESS/resampling when it is a kernel of its own; [2] KV reindex; milliseconds and
+ * bracket counts) and clears the record. */
 psmc_status psmc_timing_enable(psmc_ctx*, int on);
 psmc_status psmc_timing_read(psmc_ctx*, double* ms_out, int64_t* launches_out);
 

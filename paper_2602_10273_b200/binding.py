@@ -236,8 +236,9 @@ class Psmc:
         d = None if lens is None else np.ascontiguousarray(lens, dtype=np.int32)
         _check(lib().psmc_set_state(self._h, _ptr(a), _ptr(b), _ptr(c), _ptr(d)), "psmc_set_state")
 
-    def timing_enable(self, on: bool):
-        _check(lib().psmc_timing_enable(self._h, 1 if on else 0), "psmc_timing_enable")
+    def timing_enable(self, on):
+        """False/0: off; True/1: one event bracket per kernel; 2: one per psmc_step call and one per reindex kernel."""
+        _check(lib().psmc_timing_enable(self._h, int(on)), "psmc_timing_enable")
 
     def timing_read(self):
         """(ms[3], launches[3]) for the logit pass, the weights/resampling kernel and the KV reindex."""

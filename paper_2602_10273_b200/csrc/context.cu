@@ -92,7 +92,9 @@ struct LaunchTimer {
     cudaStream_t s;
     psmc_ctx::Timed t;
     bool on;
-    LaunchTimer(psmc_ctx* ctx, cudaStream_t stream, int kind) : c(ctx), s(stream), on(ctx->timing_on != 0) {
+    // level: 1 = a single kernel, 2 = a whole call; the bracket is taken when it matches the mode that is switched on
+    LaunchTimer(psmc_ctx* ctx, cudaStream_t stream, int kind, int level = 1)
+        : c(ctx), s(stream), on(ctx->timing_on == level) {
         if (!on) return;
         cudaEvent_t ev[2];
         for (int i = 0; i < 2; ++i) {
@@ -231,6 +233,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     wa.sources = c->sources[0]; wa.dst_rows = c->dst_rows[0];
     wa.n_sources = c->counts[t & 1]; wa.n_moves = c->counts[t & 1] + 1;
     wa.status = c->status;
+    LaunchTimer whole(c, s, 0, 2);
     if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
         LaunchTimer lt(c, s, 0);
         if (launch_step_fused(la, wa, c->row_arrivals, c->group_arrivals, s) != cudaSuccess) return PSMC_E_CUDA;
@@ -328,7 +331,7 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
             k.dst[2 * l + 1] = static_cast<char*>(d->v[l0 + l]);
         }
         k.n_ptrs = 2 * nl;
-        LaunchTimer lt(c, s, 2);
+        LaunchTimer lt(c, s, 2, c->timing_on ? c->timing_on : 1);  // bracketed in either mode
         if (launch_reindex_kv(k, s) != cudaSuccess) return PSMC_E_CUDA;
     }
     return PSMC_OK;
@@ -368,7 +371,7 @@ extern "C" psmc_status psmc_sync_status(psmc_ctx* c, void* stream) {
 
 extern "C" psmc_status psmc_timing_enable(psmc_ctx* c, int on) {
     if (!c) return PSMC_E_INVAL;
-    c->timing_on = on ? 1 : 0;
+    c->timing_on = on == 2 ? 2 : (on ? 1 : 0);
     return PSMC_OK;
 }
 

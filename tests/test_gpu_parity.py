@@ -78,6 +78,19 @@ def test_logits_pass_matches_oracle(dtype, beta, V):
     assert abs(loginc[4] - (1.0 - beta) * math.log(V)) < 1e-5
 
 
+def test_logits_pass_very_long_rows():
+    """More spans per row than a lane keeps in registers (300001 logits = 293 spans of 1024), ragged end included."""
+    torch.manual_seed(7)
+    R, V = 3, 300001
+    for dtype, beta in ((torch.bfloat16, 4.0), (torch.float32, 2.71875)):
+        logits = (torch.randn(R, V, device="cuda") * 3.0).to(dtype)
+        u = np.array([O.uniform(O.hash5(13, 1, 0, V, r)) for r in range(R)])
+        u[1] = 1.0 - 2.0**-53                               # lands in the last spans
+        tok, logp, loginc, status = run_logits_pass(logits, beta, 4.0, u)
+        assert status == B.OK
+        check_rows_against_oracle(logits, beta, 4.0, u, tok, logp, loginc)
+
+
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 def test_logits_pass_unaligned_rows_and_non_optimal_proposal(dtype):
     torch.manual_seed(3)
