@@ -202,6 +202,49 @@ psmc_status psmc_reindex_kv(psmc_ctx*, const psmc_kv_desc* src, const psmc_kv_de
                             const int32_t* idx_override, void* stream);
 
 /* ------------------------------------------------------------------------- */
+/* Paged KV cache with copy-on-write resampling (Appendix C on a block table)  */
+/* ------------------------------------------------------------------------- */
+/* The reorder of Algorithm 1 row 14 asks that slot k hold the cache of its ancestor.  With the cache cut into
+ * blocks of block_len positions that are reached through a per-row block table, a duplicated particle can SHARE
+ * its ancestor's full blocks (a table entry and a reference count instead of a copy); only the last, partly
+ * filled block is copied, because both particles go on appending to it.  The bytes moved per rewritten slot drop
+ * from len to less than block_len positions.  The result is the same cache, read through the table:
+ * position p of row r lives in block table[r][p / block_len] at offset p % block_len.
+ *
+ * The context owns the table [R, max_blocks_per_row] (-1 = no block), the reference counts [n_blocks] and the
+ * free list; the caller owns the pools.  psmc_kv_paged_create sizes them and gives every row the blocks of its
+ * prompt (lengths of psmc_init_batched): with share_prompt != 0 the full blocks of a prompt are shared by the N
+ * rows of its group and only a partly filled last block is private; the caller then writes the prompt's keys and
+ * values through the table (once per group for shared blocks).  Invariant kept by every call: a partly filled
+ * block has exactly one owner.  Running out of blocks raises PSMC_E_NOMEM in the status word.  Synchronises. */
+psmc_status psmc_kv_paged_create(psmc_ctx*, int n_blocks, int block_len, int max_blocks_per_row, int share_prompt);
+
+/* Before the language model writes position len[r] of every live row: rows whose next position starts a new block
+ * get one from the free list.  Stream-ordered. */
+psmc_status psmc_kv_paged_append(psmc_ctx*, void* stream);
+
+/* At most 64 layers per call; pools 16-byte aligned with head_dim*sizeof(elem) a multiple of 16. */
+typedef struct {
+    int n_layers;
+    void* const* k;      /* HOST array [n_layers] of DEVICE pointers, each pool [n_blocks, H, block_len, D] contiguous */
+    void* const* v;
+    int n_kv_heads;      /* H */
+    int head_dim;        /* D */
+    psmc_dtype dt;
+} psmc_kv_pools;
+
+/* Applies the slot map of the most recent step: every rewritten slot gives its blocks back, takes a reference to
+ * each full block of its ancestor and a private copy of the ancestor's partly filled last block (all layers, K and
+ * V, all heads).  Groups that did not resample change nothing; without any resampling the kernels return after
+ * reading one counter.  Stream-ordered, no host synchronisation. */
+psmc_status psmc_reindex_kv_paged(psmc_ctx*, const psmc_kv_pools* pools, void* stream);
+
+/* DEVICE views of the paging state (valid until psmc_destroy or the next psmc_kv_paged_create). */
+const int32_t* psmc_kv_paged_table(psmc_ctx*);      /* [R, max_blocks_per_row] */
+const int32_t* psmc_kv_paged_refcount(psmc_ctx*);   /* [n_blocks]              */
+const int32_t* psmc_kv_paged_free_count(psmc_ctx*); /* [1] blocks on the free list */
+
+/* ------------------------------------------------------------------------- */
 /* Output (Algorithm 1 row 18)                                                */
 /* ------------------------------------------------------------------------- */
 

@@ -36,6 +36,11 @@ class KvDesc(C.Structure):
                 ("stride_row", C.c_int64), ("stride_head", C.c_int64), ("skip_shared_prompt", C.c_int)]
 
 
+class KvPools(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("k", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)),
+                ("n_kv_heads", C.c_int), ("head_dim", C.c_int), ("dt", C.c_int)]
+
+
 def lib():
     """Load libpsmc.so (once).  Raises if it has not been built: there is no other code path."""
     global _lib
@@ -87,6 +92,15 @@ def lib():
         L.psmc_set_state.argtypes = [vp, vp, vp, vp, vp]
         L.psmc_sync_status.restype = C.c_int
         L.psmc_sync_status.argtypes = [vp, vp]
+        L.psmc_kv_paged_create.restype = C.c_int
+        L.psmc_kv_paged_create.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int]
+        L.psmc_kv_paged_append.restype = C.c_int
+        L.psmc_kv_paged_append.argtypes = [vp, vp]
+        L.psmc_reindex_kv_paged.restype = C.c_int
+        L.psmc_reindex_kv_paged.argtypes = [vp, C.POINTER(KvPools), vp]
+        for name in ("psmc_kv_paged_table", "psmc_kv_paged_refcount", "psmc_kv_paged_free_count"):
+            getattr(L, name).restype = C.c_void_p
+            getattr(L, name).argtypes = [vp]
         L.psmc_timing_enable.restype = C.c_int
         L.psmc_timing_enable.argtypes = [vp, C.c_int]
         L.psmc_timing_read.restype = C.c_int
@@ -135,7 +149,8 @@ _VIEW_DTYPES = {"psmc_tokens": torch.int32, "psmc_last_tokens": torch.int32, "ps
                 "psmc_log_inc": torch.float64, "psmc_logp_tok": torch.float64, "psmc_cum_logp": torch.float64,
                 "psmc_ancestors": torch.int32, "psmc_slot_map": torch.int32, "psmc_resampled": torch.int32,
                 "psmc_ess": torch.float64, "psmc_log_z": torch.float64, "psmc_lens": torch.int32,
-                "psmc_done": torch.uint8, "psmc_move_count": torch.int32}
+                "psmc_done": torch.uint8, "psmc_move_count": torch.int32, "psmc_kv_paged_table": torch.int32,
+                "psmc_kv_paged_refcount": torch.int32, "psmc_kv_paged_free_count": torch.int32}
 
 
 _TYPESTR = {torch.int32: "<i4", torch.float64: "<f8", torch.uint8: "|u1"}
@@ -216,6 +231,36 @@ class Psmc:
             assert idx_override.is_cuda and idx_override.dtype == torch.int32 and idx_override.numel() == self.R
         _check(lib().psmc_reindex_kv(self._h, C.byref(src), None if dst is None else C.byref(dst),
                                      _ptr(idx_override), _stream(stream)), "psmc_reindex_kv")
+
+    # ---- paged KV cache (block table, copy on write)
+    def kv_paged_create(self, n_blocks: int, block_len: int, max_blocks_per_row: int, share_prompt: bool = True):
+        _check(lib().psmc_kv_paged_create(self._h, n_blocks, block_len, max_blocks_per_row, 1 if share_prompt else 0),
+               "psmc_kv_paged_create")
+        self._paged = (n_blocks, block_len, max_blocks_per_row)
+
+    def kv_paged_append(self, stream=None):
+        _check(lib().psmc_kv_paged_append(self._h, _stream(stream)), "psmc_kv_paged_append")
+
+    def make_kv_pools(self, k_pools, v_pools):
+        """k_pools / v_pools: lists (one per layer) of contiguous CUDA tensors [n_blocks, H, block_len, D]."""
+        p0 = k_pools[0]
+        nb, H, Bl, D = p0.shape
+        assert (nb, Bl) == self._paged[:2]
+        n = len(k_pools)
+        for t in list(k_pools) + list(v_pools):
+            assert t.shape == p0.shape and t.is_contiguous() and t.dtype == p0.dtype and t.is_cuda
+        ka = (C.c_void_p * n)(*[t.data_ptr() for t in k_pools])
+        va = (C.c_void_p * n)(*[t.data_ptr() for t in v_pools])
+        d = KvPools(n, C.cast(ka, C.POINTER(C.c_void_p)), C.cast(va, C.POINTER(C.c_void_p)), H, D, _dtype_code(p0))
+        d._keep = (ka, va, list(k_pools), list(v_pools))
+        return d
+
+    def reindex_kv_paged(self, pools: KvPools, stream=None):
+        _check(lib().psmc_reindex_kv_paged(self._h, C.byref(pools), _stream(stream)), "psmc_reindex_kv_paged")
+
+    kv_paged_table = property(lambda s: s.device_view("psmc_kv_paged_table", s.R * s._paged[2]).view(s.R, s._paged[2]))
+    kv_paged_refcount = property(lambda s: s.device_view("psmc_kv_paged_refcount", s._paged[0]))
+    kv_paged_free_count = property(lambda s: int(s._view("psmc_kv_paged_free_count", 1)[0]))
 
     def select(self, out_tokens=None, out_len=None, out_index=None, stream=None):
         dev = torch.device("cuda", torch.cuda.current_device())

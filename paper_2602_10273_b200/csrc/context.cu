@@ -16,6 +16,7 @@ struct psmc_ctx {
     uint64_t seed;
     int32_t* prompt_len_host;  // [G]
     int32_t* prompt_len_dev;   // [G] the same on the device (for the shared-prompt form of the KV reindex)
+    PagedState paged;          // block table, reference counts and free list of the paged cache (zero until created)
     // particle state
     double *logW, *S;
     uint8_t* done;
@@ -125,6 +126,9 @@ void free_ctx(psmc_ctx* c) {
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
                     c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev};
     for (void* p : ptrs)
+        if (p) cudaFree(p);
+    void* paged_ptrs[] = {c->paged.table, c->paged.refc, c->paged.free_list, c->paged.free_top};
+    for (void* p : paged_ptrs)
         if (p) cudaFree(p);
     delete[] c->prompt_len_host;
     delete c;
@@ -336,6 +340,61 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
     }
     return PSMC_OK;
 }
+
+extern "C" psmc_status psmc_kv_paged_create(psmc_ctx* c, int n_blocks, int block_len, int max_blocks_per_row,
+                                            int share_prompt) {
+    if (!c || n_blocks < 1 || block_len < 1 || max_blocks_per_row < 1) return PSMC_E_INVAL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    PagedState& ps = c->paged;
+    void* old[] = {ps.table, ps.refc, ps.free_list, ps.free_top};
+    for (void* p : old)
+        if (p) cudaFree(p);
+    ps = PagedState{};
+    ps.n_blocks = n_blocks; ps.block_len = block_len; ps.max_blocks = max_blocks_per_row; ps.R = c->R; ps.N = c->N;
+    cudaError_t e = cudaSuccess;
+    auto ok = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
+    ok(dev_alloc(&ps.table, (size_t)c->R * max_blocks_per_row));
+    ok(dev_alloc(&ps.refc, (size_t)n_blocks));
+    ok(dev_alloc(&ps.free_list, paged_free_list_words(n_blocks, c->R)));
+    ok(dev_alloc(&ps.free_top, 1));
+    if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? PSMC_E_NOMEM : PSMC_E_CUDA;
+    if (launch_paged_init(ps, c->prompt_len_dev, c->G, share_prompt, c->status, nullptr) != cudaSuccess) return PSMC_E_CUDA;
+    return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_kv_paged_append(psmc_ctx* c, void* stream) {
+    if (!c) return PSMC_E_INVAL;
+    if (!c->paged.table) return PSMC_E_STATE;
+    return launch_paged_append(c->paged, c->len, c->done, c->status, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" psmc_status psmc_reindex_kv_paged(psmc_ctx* c, const psmc_kv_pools* pools, void* stream) {
+    if (!c || !pools || !pools->k || !pools->v) return PSMC_E_INVAL;
+    if (!c->paged.table) return PSMC_E_STATE;
+    if (pools->n_layers < 1 || pools->n_layers > kMaxKvPtrs / 2 || pools->n_kv_heads < 1 || pools->head_dim < 1)
+        return PSMC_E_INVAL;
+    if (pools->dt != PSMC_F32 && pools->dt != PSMC_BF16) return PSMC_E_INVAL;
+    PagedPools pp;
+    pp.n_layers = pools->n_layers; pp.H = pools->n_kv_heads;
+    pp.pos_bytes = pools->head_dim * (pools->dt == PSMC_F32 ? 4 : 2);
+    uint64_t bits = (uint64_t)pp.pos_bytes;
+    for (int l = 0; l < pools->n_layers; ++l) {
+        if (!pools->k[l] || !pools->v[l]) return PSMC_E_INVAL;
+        pp.k[l] = static_cast<char*>(pools->k[l]);
+        pp.v[l] = static_cast<char*>(pools->v[l]);
+        bits |= (uint64_t)(uintptr_t)pools->k[l] | (uint64_t)(uintptr_t)pools->v[l];
+    }
+    if (bits % 16 != 0) return PSMC_E_INVAL;  // the block copy moves 16 bytes at a time
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LaunchTimer lt(c, s, 2, c->timing_on ? c->timing_on : 1);
+    return launch_paged_reindex(c->paged, pp, c->sources[0], c->dst_rows[0], c->counts[c->t & 1], c->counts[c->t & 1] + 1,
+                                c->status, s) == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
+extern "C" const int32_t* psmc_kv_paged_table(psmc_ctx* c) { return c ? c->paged.table : nullptr; }
+extern "C" const int32_t* psmc_kv_paged_refcount(psmc_ctx* c) { return c ? c->paged.refc : nullptr; }
+extern "C" const int32_t* psmc_kv_paged_free_count(psmc_ctx* c) { return c ? c->paged.free_top : nullptr; }
 
 extern "C" psmc_status psmc_select(psmc_ctx* c, int32_t* out_tokens, int32_t* out_len, int32_t* out_index,
                                    void* stream) {

@@ -129,6 +129,29 @@ cudaError_t launch_build_moves(const int32_t* idx, int R, int max_len, int in_pl
                                int32_t* dst_rows, int32_t* n_sources, int32_t* n_moves, int32_t* status,
                                cudaStream_t stream);
 
+// ---------------------------------------------------------------- paged KV cache (block table, copy on write)
+struct PagedState {
+    int32_t* table;      // [R][max_blocks]
+    int32_t* refc;       // [n_blocks]
+    int32_t* free_list;  // [n_blocks] stack; entries [0, *free_top) are free
+    int32_t* free_top;   // [1]
+    int n_blocks, block_len, max_blocks, R, N;
+};
+struct PagedPools {
+    char* k[kMaxKvPtrs / 2];
+    char* v[kMaxKvPtrs / 2];
+    int n_layers, H;
+    int pos_bytes;       // head_dim * sizeof(elem)
+};
+size_t paged_free_list_words(int n_blocks, int R);  // words to allocate for PagedState::free_list
+cudaError_t launch_paged_init(const PagedState& ps, const int32_t* prompt_len_dev, int G, int share_prompt,
+                              int32_t* status, cudaStream_t stream);
+cudaError_t launch_paged_append(const PagedState& ps, const int32_t* len, const uint8_t* done, int32_t* status,
+                                cudaStream_t stream);
+cudaError_t launch_paged_reindex(const PagedState& ps, const PagedPools& pools, const MoveSource* sources,
+                                 const int32_t* dst_rows, const int32_t* n_sources, const int32_t* n_moves,
+                                 int32_t* status, cudaStream_t stream);
+
 // ---------------------------------------------------------------- final draw and back-trace
 struct SelectArgs {
     int G, N, R, t, T_max, eos;
