@@ -155,11 +155,40 @@ def run_ours(args):
     seed = plan.seed
     wl = WC.DeviceWorkload(cfg, seed, G=G, device=dev)
     R, N = wl.R, cfg.N
-    ks, vs = wl.new_kv()
     ps = B.Psmc(N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=G, T_max=T_total,
                 prompt_len=wl.prompt_len)
-    desc = ps.make_kv_desc(ks, vs, skip_shared_prompt=args.skip_shared_prompt)
     skip = wl.prompt_len if args.skip_shared_prompt else None
+    PAGE = 16  # positions per block in the supplementary paged run
+    if args.paged_kv:  # same capacity as the dense cache, cut into blocks reached through a table
+        max_blocks = -(-cfg.max_len // PAGE)
+        n_blocks = R * max_blocks
+        shape = (n_blocks, cfg.n_kv_heads, PAGE, cfg.head_dim)
+        kpools = [torch.empty(shape, dtype=wl.tdtype, device=dev) for _ in range(cfg.n_layers)]
+        vpools = [torch.empty(shape, dtype=wl.tdtype, device=dev) for _ in range(cfg.n_layers)]
+        ps.kv_paged_create(n_blocks, PAGE, max_blocks, share_prompt=True)
+        pdesc = ps.make_kv_pools(kpools, vpools)
+
+        def reset_all():
+            ps.reset(seed)
+            ps.kv_paged_create(n_blocks, PAGE, max_blocks, share_prompt=True)
+
+        def before_step():
+            ps.kv_paged_append()
+
+        def move_cache():
+            ps.reindex_kv_paged(pdesc)
+    else:
+        ks, vs = wl.new_kv()
+        desc = ps.make_kv_desc(ks, vs, skip_shared_prompt=args.skip_shared_prompt)
+
+        def reset_all():
+            ps.reset(seed)
+
+        def before_step():
+            pass
+
+        def move_cache():
+            ps.reindex_kv(desc)
     last = ps.device_view("psmc_last_tokens", R)
 
     # logit blocks: generated along a short closed loop, then reused cyclically by every pass below
@@ -170,19 +199,25 @@ def run_ours(args):
         ps.step(blocks[t - 1])
         prev.copy_(last)
     assert ps.sync_status() == B.OK
-    ps.reset(seed)
+    reset_all()
 
     def one_pass(n_steps, first_t=1):
         for t in range(first_t, first_t + n_steps):
+            before_step()
             ps.step(blocks[(t - 1) % N_BLOCKS])
-            ps.reindex_kv(desc)
+            move_cache()
 
     # recording pass: per-step algorithmic KV bytes and live rows (deterministic, so the timed passes repeat it)
     kv_bytes, moved_slots, live_rows = [], [], []
     for t in range(1, T_total + 1):
         live_rows.append(R - int(ps.done.numpy().sum()))  # rows that are live when step t starts
         one_pass(1, t)
-        b, mv = moved_bytes(ps.slot_map.numpy(), ps.lens.numpy(), G, N, cfg.kv_bytes_per_pos_per_row, skip)
+        if args.paged_kv:  # one partly filled block per rewritten slot, read and written once
+            sm, ln = ps.slot_map.numpy().reshape(G, N), ps.lens.numpy().reshape(G, N)
+            mvd = sm != np.arange(N)[None, :]
+            b, mv = 2 * int((ln[mvd] % PAGE).sum()) * cfg.kv_bytes_per_pos_per_row, int(mvd.sum())
+        else:
+            b, mv = moved_bytes(ps.slot_map.numpy(), ps.lens.numpy(), G, N, cfg.kv_bytes_per_pos_per_row, skip)
         kv_bytes.append(b)
         moved_slots.append(mv)
     assert ps.sync_status() == B.OK
@@ -199,7 +234,7 @@ def run_ours(args):
         return replicas.sum_over_ranks(x, dev)
 
     # ---- pass A: the headline. K steps, device-resident inputs, one pair of events around all of them ----
-    ps.reset(seed)
+    reset_all()
     one_pass(Wm, 1)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -214,7 +249,7 @@ def run_ours(args):
     value = sum_over_ranks(live_timed) / (ms_total * 1e-3)
 
     # ---- pass B: same K steps with every kernel bracketed by events, for the roofline of each kernel ----
-    ps.reset(seed)
+    reset_all()
     one_pass(Wm, 1)
     torch.cuda.synchronize(dev)
     ps.timing_enable(True)
@@ -232,26 +267,27 @@ def run_ours(args):
         return None if r is None or launches < 1 else r * algorithmic_bytes / launches
 
     dominant = int(np.argmax(kms))
-    names = ["logits_stream_kernel", "finish_weights_resample_kernel", "reindex_bulk_kernel"]
+    kv_name = "paged_release_acquire_copy_kernels" if args.paged_kv else "reindex_bulk_kernel"
+    names = ["logits_stream_kernel", "finish_weights_resample_kernel", kv_name]
     roofs = {
         "logits_stream_kernel": {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
                                "frac": k1_gbs / hbm_peak, "traffic": traffic("logits_stream_kernel", k1_bytes, kn[0]),
                                "peak_kind": peak_kind,
                                "avg_launch_us": 1e3 * kms[0] / max(kn[0], 1), "time_share": shares[0],
                                "bytes_per_launch": k1_bytes / max(kn[0], 1)},
-        "reindex_bulk_kernel": {"bound": "hbm", "achieved": k3_gbs, "peak": hbm_peak, "unit": "GB/s",
-                                "frac": k3_gbs / hbm_peak, "traffic": traffic("reindex_bulk_kernel", k3_bytes, kn[2]),
+        kv_name: {"bound": "hbm", "achieved": k3_gbs, "peak": hbm_peak, "unit": "GB/s",
+                                "frac": k3_gbs / hbm_peak, "traffic": traffic(kv_name, k3_bytes, kn[2]),
                                 "peak_kind": peak_kind,
                                 "avg_launch_us": 1e3 * kms[2] / max(kn[2], 1), "time_share": shares[2],
                                 "bytes_per_launch": k3_bytes / max(kn[2], 1)},
         "finish_weights_resample_kernel": {"bound": "latency", "avg_launch_us": 1e3 * kms[1] / max(kn[1], 1),
                                     "time_share": shares[1]},
     }
-    roofline = dict(roofs[names[dominant]] if dominant != 1 else roofs["reindex_bulk_kernel"])
-    roofline["kernel"] = names[dominant] if dominant != 1 else "reindex_bulk_kernel"
+    roofline = dict(roofs[names[dominant]] if dominant != 1 else roofs[kv_name])
+    roofline["kernel"] = names[dominant] if dominant != 1 else kv_name
 
     # ---- pass C: the same K steps with one bracket around each psmc_step (its kernels keep their chained launches) ----
-    ps.reset(seed)
+    reset_all()
     one_pass(Wm, 1)
     torch.cuda.synchronize(dev)
     ps.timing_enable(2)
@@ -265,15 +301,17 @@ def run_ours(args):
     Ke = min(K, args.e2e_steps)
     host_blocks = [b.cpu().pin_memory() for b in blocks]
     tok_host = torch.empty(R, dtype=torch.int32).pin_memory()
-    ps.reset(seed)
+    reset_all()
     for t in range(1, Wm + 1):
+        before_step()
         ps.step_host(host_blocks[(t - 1) % N_BLOCKS], tok_host)
-        ps.reindex_kv(desc)
+        move_cache()
     barrier()
     e0.record()
     for t in range(Wm + 1, Wm + Ke + 1):
+        before_step()
         ps.step_host(host_blocks[(t - 1) % N_BLOCKS], tok_host)
-        ps.reindex_kv(desc)
+        move_cache()
     e1.record()
     torch.cuda.synchronize(dev)
     barrier()
@@ -290,12 +328,15 @@ def run_ours(args):
                    "prompts_per_gpu": G, "rows_per_gpu": R, "alpha": cfg.alpha, "tau": cfg.tau, "kappa": cfg.kappa,
                    "ramp": cfg.ramp, "l2": "inputs larger than L2: %d logit blocks of %.0f MB rotated, KV %.1f GB" % (
                        N_BLOCKS, R * cfg.logit_bytes_per_row / 1e6, G * per_group / 1e9),
-                   "kv_reindex": "prompt positions left in place" if args.skip_shared_prompt else "whole live prefix copied",
+                   "kv_reindex": ("paged cache, blocks of %d positions, copy on write" % PAGE) if args.paged_kv else
+                                 ("prompt positions left in place" if args.skip_shared_prompt else "whole live prefix copied"),
                    "parallelism": "replicas only (prompts sharded, no collective)"},
         "clocks": clk.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": R * cfg.logit_bytes_per_row,
                 "d2h_bytes_per_step": R * 4, "steps": Ke, "ms_per_step": ms_e2e / Ke},
-        "gpu_launches": int(K * (2 + (cfg.n_layers + 63) // 64)),
+        # per step: logit pass + finish/weights/resampling (two kernels on this workload) + the cache move (one bulk
+        # reindex kernel per 64 layers, or append + release + acquire + copy for the paged cache)
+        "gpu_launches": int(K * (2 + (4 if args.paged_kv else (cfg.n_layers + 63) // 64))),
         "roofline": roofline,
         "kernels": roofs,
         "kv_reindex": {"gb_per_s": k3_gbs, "frac_of_hbm_peak": k3_gbs / hbm_peak,
@@ -414,6 +455,8 @@ def main():
     ap.add_argument("--groups", type=int, default=None, help="override the number of prompts (default: the workload's)")
     ap.add_argument("--e2e-steps", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--paged-kv", action="store_true",
+                    help="supplementary run: paged cache with copy-on-write resampling instead of the dense cache")
     ap.add_argument("--skip-shared-prompt", action="store_true",
                     help="supplementary run: the KV reindex leaves each group's prompt positions in place (not the "
                          "headline configuration, which copies whole live prefixes)")
