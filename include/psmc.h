@@ -284,6 +284,18 @@ int psmc_rows(const psmc_ctx*);              /* R                               
 psmc_status psmc_set_state(psmc_ctx*, const double* log_w, const double* cum_logp,
                            const uint8_t* done, const int32_t* lens);
 
+/* Snapshot of a run, for checkpointing and for moving a run to another context.  Because all randomness is a
+ * counter hash of (seed, group, step, slot), a context that loads a snapshot continues bit for bit as the one that
+ * saved it would have.  The snapshot holds the particle state, the results of the last step and the ancestry log
+ * up to the current step; caches (dense or paged, with their tables) are the caller's to save, and the move list
+ * of a step does not travel: take the snapshot after the step's cache move.  psmc_state_save
+ * writes psmc_state_bytes() bytes to HOST memory; psmc_state_load needs a context created with the same G, N, V,
+ * T_max (PSMC_E_INVAL otherwise, nothing loaded) and takes over alpha, tau, kappa, ramp, eos, seed, resampler and
+ * the step counter from the snapshot.  Both synchronise the device. */
+size_t psmc_state_bytes(const psmc_ctx*);
+psmc_status psmc_state_save(psmc_ctx*, void* host_buf, size_t bytes);
+psmc_status psmc_state_load(psmc_ctx*, const void* host_buf, size_t bytes);
+
 /* Profiling aid.  on = 1: every kernel launched by psmc_step / psmc_step_host / psmc_reindex_kv is bracketed by
  * CUDA events on the caller's stream.  on = 2: one bracket around the kernels of a psmc_step (they then keep
  * their chained launches) and one around every reindex kernel.  on = 0: off.  psmc_timing_read waits for the

@@ -101,6 +101,12 @@ def lib():
         for name in ("psmc_kv_paged_table", "psmc_kv_paged_refcount", "psmc_kv_paged_free_count"):
             getattr(L, name).restype = C.c_void_p
             getattr(L, name).argtypes = [vp]
+        L.psmc_state_bytes.restype = C.c_size_t
+        L.psmc_state_bytes.argtypes = [vp]
+        L.psmc_state_save.restype = C.c_int
+        L.psmc_state_save.argtypes = [vp, vp, C.c_size_t]
+        L.psmc_state_load.restype = C.c_int
+        L.psmc_state_load.argtypes = [vp, vp, C.c_size_t]
         L.psmc_timing_enable.restype = C.c_int
         L.psmc_timing_enable.argtypes = [vp, C.c_int]
         L.psmc_timing_read.restype = C.c_int
@@ -231,6 +237,17 @@ class Psmc:
             assert idx_override.is_cuda and idx_override.dtype == torch.int32 and idx_override.numel() == self.R
         _check(lib().psmc_reindex_kv(self._h, C.byref(src), None if dst is None else C.byref(dst),
                                      _ptr(idx_override), _stream(stream)), "psmc_reindex_kv")
+
+    def state_save(self) -> bytes:
+        """psmc_state_save: snapshot of the run (particle state, last results, ancestry log) as bytes."""
+        n = lib().psmc_state_bytes(self._h)
+        buf = C.create_string_buffer(n)
+        _check(lib().psmc_state_save(self._h, buf, n), "psmc_state_save")
+        return buf.raw
+
+    def state_load(self, blob: bytes) -> None:
+        """psmc_state_load: continue the run a snapshot was taken from (same G, N, V, T_max)."""
+        _check(lib().psmc_state_load(self._h, blob, len(blob)), "psmc_state_load")
 
     # ---- paged KV cache (block table, copy on write)
     def kv_paged_create(self, n_blocks: int, block_len: int, max_blocks_per_row: int, share_prompt: bool = True):

@@ -420,6 +420,89 @@ extern "C" psmc_status psmc_set_state(psmc_ctx* c, const double* log_w, const do
     return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
+namespace {
+
+struct SnapshotHeader {
+    uint64_t magic;
+    int32_t G, N, V, T_max, t, ramp, eos, resampler;
+    double alpha, tau, kappa;
+    uint64_t seed;
+};
+constexpr uint64_t kSnapshotMagic = 0x31434d5350ull;  // "PSMC1"
+
+// the device arrays of a snapshot, in file order; hist arrays only up to step t
+struct Piece {
+    void* dev;
+    size_t bytes;
+};
+int snapshot_pieces(psmc_ctx* c, int t, Piece* out) {
+    const size_t R = (size_t)c->R, G = (size_t)c->G;
+    int n = 0;
+    auto add = [&](void* p, size_t b) { out[n].dev = p; out[n].bytes = b; ++n; };
+    add(c->logW, 8 * R); add(c->S, 8 * R); add(c->logp, 8 * R); add(c->loginc, 8 * R);
+    add(c->ess, 8 * G); add(c->logZ, 8 * G);
+    add(c->len, 4 * R); add(c->tok, 4 * R); add(c->last_tok, 4 * R); add(c->anc, 4 * R); add(c->map, 4 * R);
+    add(c->resampled, 4 * G); add(c->status, 4);
+    add(c->hist_tok, 4 * R * (size_t)t); add(c->hist_map, 4 * R * (size_t)t);
+    add(c->done, R);
+    return n;
+}
+size_t snapshot_bytes(psmc_ctx* c, int t) {
+    Piece ps[20];
+    const int n = snapshot_pieces(c, t, ps);
+    size_t total = sizeof(SnapshotHeader);
+    for (int i = 0; i < n; ++i) total += ps[i].bytes;
+    return total;
+}
+
+}  // namespace
+
+extern "C" size_t psmc_state_bytes(const psmc_ctx* c) {
+    return c ? snapshot_bytes(const_cast<psmc_ctx*>(c), c->t) : 0;
+}
+
+extern "C" psmc_status psmc_state_save(psmc_ctx* c, void* host_buf, size_t bytes) {
+    if (!c || !host_buf || bytes < snapshot_bytes(c, c->t)) return PSMC_E_INVAL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    SnapshotHeader h{};
+    h.magic = kSnapshotMagic;
+    h.G = c->G; h.N = c->N; h.V = c->V; h.T_max = c->T_max; h.t = c->t; h.ramp = c->ramp; h.eos = c->eos;
+    h.resampler = c->resampler; h.alpha = c->alpha; h.tau = c->tau; h.kappa = c->kappa; h.seed = c->seed;
+    char* out = static_cast<char*>(host_buf);
+    memcpy(out, &h, sizeof(h));
+    out += sizeof(h);
+    Piece ps[20];
+    const int n = snapshot_pieces(c, c->t, ps);
+    for (int i = 0; i < n; ++i) {
+        if (ps[i].bytes && cudaMemcpy(out, ps[i].dev, ps[i].bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return PSMC_E_CUDA;
+        out += ps[i].bytes;
+    }
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_state_load(psmc_ctx* c, const void* host_buf, size_t bytes) {
+    if (!c || !host_buf || bytes < sizeof(SnapshotHeader)) return PSMC_E_INVAL;
+    SnapshotHeader h;
+    memcpy(&h, host_buf, sizeof(h));
+    if (h.magic != kSnapshotMagic || h.G != c->G || h.N != c->N || h.V != c->V || h.T_max != c->T_max || h.t < 0 ||
+        h.t > c->T_max || h.resampler < 0 || h.resampler > 3)
+        return PSMC_E_INVAL;
+    if (bytes < snapshot_bytes(c, h.t)) return PSMC_E_INVAL;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    psmc_status st = reset_device_state(c);  // counters, arrival words and the rest of the scratch state start clean
+    if (st != PSMC_OK) return st;
+    const char* in = static_cast<const char*>(host_buf) + sizeof(h);
+    Piece ps[20];
+    const int n = snapshot_pieces(c, h.t, ps);
+    for (int i = 0; i < n; ++i) {
+        if (ps[i].bytes && cudaMemcpy(ps[i].dev, in, ps[i].bytes, cudaMemcpyHostToDevice) != cudaSuccess) return PSMC_E_CUDA;
+        in += ps[i].bytes;
+    }
+    c->t = h.t; c->ramp = h.ramp; c->eos = h.eos; c->resampler = h.resampler;
+    c->alpha = h.alpha; c->tau = h.tau; c->kappa = h.kappa; c->seed = h.seed;
+    return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+}
+
 extern "C" psmc_status psmc_sync_status(psmc_ctx* c, void* stream) {
     if (!c) return PSMC_E_INVAL;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PSMC_E_CUDA;

@@ -250,6 +250,39 @@ def test_reindex_leaves_a_shared_prompt_in_place(name, G, T):
     assert st.slots_moved > 0
 
 
+def test_snapshot_resumes_bit_for_bit():
+    """Save after 10 tokens, load into a fresh context, go on: the oracle, which never stopped, still agrees at every
+    step, and the final draw walks an ancestry log that spans the snapshot."""
+    c = W.CONFIGS["tiny"]
+    T = 40
+    wl, ps, orc = P.make_pair(c, seed=6, T_max=T, resampler=B.RESIDUAL)
+    st = P.LoopStats()
+    kappa_f = float(np.float32(c.kappa))
+    lg = wl.new_logits()
+    prev = wl.first_prev.clone()
+    for t in range(1, T + 1):
+        wl.fill(lg, t, prev)
+        ps.step(lg)
+        P.compare_step(ps, orc, P.logits_to_numpy(lg), st, kappa_f)
+        prev.copy_(ps.device_view("psmc_last_tokens", ps.R))
+        if t == 10:
+            blob = ps.state_save()
+            assert len(blob) == B.lib().psmc_state_bytes(ps._h)
+            ps.destroy()
+            ps = B.Psmc(c.N, c.V, 2.0, 1.0, 0.3, 0, 999, 0, G=1, T_max=T, prompt_len=wl.prompt_len)  # other settings
+            ps.state_load(blob)
+            other = B.Psmc(c.N, c.V + 1, c.alpha, c.tau, c.kappa, 0, 6, c.eos_id, G=1, T_max=T)
+            with pytest.raises(B.PsmcError):
+                other.state_load(blob)                       # a different vocabulary: refused, nothing loaded
+            other.destroy()
+    assert st.resample_events > 0
+    toks, ln, ix = ps.select()
+    o_toks, o_ln, o_ix = orc.select()
+    assert np.array_equal(ix.cpu().numpy(), o_ix) and np.array_equal(toks.cpu().numpy(), o_toks)
+    assert np.array_equal(ln.cpu().numpy(), o_ln)
+    ps.destroy()
+
+
 def test_eos_rows_freeze_and_are_not_read():
     c = W.CONFIGS["tiny"]
 
