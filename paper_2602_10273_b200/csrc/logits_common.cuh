@@ -194,13 +194,11 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
 }
 
 // One lane's share of the selected span: `E` consecutive logits from e0 (clipped to b0).  Returns their mass
-// (eight logits summed in fp32 at a time, then in fp64) and the last position with mass (-1 if none).
+// (eight logits summed in fp32 at a time, then in fp64).
 template <int DT, int MODE>
-__device__ __forceinline__ double lane_share(const FinishParams& p, const void* rowp, int e0, int E, int b0, float neg_C,
-                                            int& lane_last) {
+__device__ __forceinline__ double lane_share(const FinishParams& p, const void* rowp, int e0, int E, int b0, float neg_C) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;  // logits per 16 bytes
     double lm = 0.0;
-    lane_last = -1;
     if (e0 >= b0) return lm;
     if (p.vec && e0 + E <= b0) {
         const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)e0 * (16 / kPer));
@@ -214,33 +212,33 @@ __device__ __forceinline__ double lane_share(const FinishParams& p, const void* 
             for (int i = 0; i < 4; ++i) {
                 if (q0 + i >= Q) break;
                 const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-                const int at = e0 + (q0 + i) * kPer;
                 float g[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    if (DT == PSMC_BF16) {
-                        const float m0 = logit_mass<MODE>(__uint_as_float(w[j] << 16), neg_C, p.bf);
-                        const float m1 = logit_mass<MODE>(__uint_as_float(w[j] & 0xffff0000u), neg_C, p.bf);
-                        if (m0 > 0.f) lane_last = at + 2 * j;
-                        if (m1 > 0.f) lane_last = at + 2 * j + 1;
-                        g[j] = m0 + m1;
-                    } else {
+                    if (DT == PSMC_BF16)
+                        g[j] = logit_mass<MODE>(__uint_as_float(w[j] << 16), neg_C, p.bf) +
+                               logit_mass<MODE>(__uint_as_float(w[j] & 0xffff0000u), neg_C, p.bf);
+                    else
                         g[j] = logit_mass<MODE>(__uint_as_float(w[j]), neg_C, p.bf);
-                        if (g[j] > 0.f) lane_last = at + j;
-                    }
                 }
                 lm += (double)((g[0] + g[1]) + (g[2] + g[3]));
             }
         }
     } else {
         const int e1 = min(b0, e0 + E);
-        for (int i = e0; i < e1; ++i) {
-            const float e = logit_mass<MODE>(load_elem<DT>(rowp, i), neg_C, p.bf);
-            if (e > 0.f) lane_last = i;
-            lm += (double)e;
-        }
+        for (int i = e0; i < e1; ++i) lm += (double)logit_mass<MODE>(load_elem<DT>(rowp, i), neg_C, p.bf);
     }
     return lm;
+}
+
+// Last position of [a0, b0) whose logit has mass, -1 if none (one warp; the rare case in which the re-read sums fall
+// a rounding error short of the target).
+template <int DT, int MODE>
+__device__ __forceinline__ int last_with_mass(const FinishParams& p, const void* rowp, int a0, int b0, float neg_C, int lane) {
+    int last = -1;
+    for (int i = a0 + lane; i < b0; i += 32)
+        if (logit_mass<MODE>(load_elem<DT>(rowp, i), neg_C, p.bf) > 0.f) last = i;
+    return warp_max(last);
 }
 
 // Token inside the owner lane's logits [o0, o1): 32 at a time across the warp, in vocabulary order, the loads of
@@ -271,12 +269,15 @@ __device__ __forceinline__ int locate_in_lane(const FinishParams& p, const void*
     return y >= 0 ? y : last_with_mass;  // the finer sums may fall a rounding error short of the lane's total
 }
 
+// Called by all 32 lanes; every lane returns the same RowResult.  The two logarithms are taken side by side
+// (lane 0 and lane 1 of one call) rather than one after the other.
 template <int DT>
-__device__ __forceinline__ RowResult row_result(const FinishParams& p, const void* rowp, const RowTotals& t, int y) {
+__device__ __forceinline__ RowResult row_result(const FinishParams& p, const void* rowp, const RowTotals& t, int y, int lane) {
     RowResult r;
     // l_y - C ln 2: the token's logit relative to the row's reference, in natural units
     const double dl = (double)load_elem<DT>(rowp, y) - (double)t.C * kLn2;
-    const double ln_s1 = log(t.S1), ln_sb = log(t.Sb);
+    const double lg = log((lane & 1) ? t.Sb : t.S1);
+    const double ln_s1 = __shfl_sync(kFull, lg, 0), ln_sb = __shfl_sync(kFull, lg, 1);
     r.tok = y;
     r.logp = dl - ln_s1;  // log p(y) = l_y - L1
     // alpha_t log p(y) - log q(y), log q(y) = beta l_y - Lb, grouped so that the token's own logit drops out
@@ -296,8 +297,7 @@ __device__ __forceinline__ RowResult finish_row_warp(const FinishParams& p, int 
     const float neg_C = -t.C;
     const int a0 = t.jsel * p.span, b0 = min(p.V, a0 + p.span);
     const int E = p.span >> 5;
-    int lane_last;
-    const double lm = lane_share<DT, MODE>(p, rowp, a0 + lane * E, E, b0, neg_C, lane_last);
+    const double lm = lane_share<DT, MODE>(p, rowp, a0 + lane * E, E, b0, neg_C);
     const double r_incl = t.base + warp_scan_incl(lm, lane);
     const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
     int y;
@@ -307,10 +307,10 @@ __device__ __forceinline__ RowResult finish_row_warp(const FinishParams& p, int 
         const int o0 = a0 + owner * E;
         y = locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
     } else {
-        y = warp_max(lane_last);  // the re-read sums fall short of the target: last token with mass in the span
+        y = last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);  // the re-read sums fall short of the target
     }
     if (y < 0) return bad;
-    return row_result<DT>(p, rowp, t, y);
+    return row_result<DT>(p, rowp, t, y, lane);
 }
 
 // ---- the finish at CTA level: several warps share a row ----
@@ -319,7 +319,6 @@ struct FinishShared {
     RowTotals row[kFinishMaxWarps];  // per row of the current pass: what its first warp learnt from the triples
     bool live[kFinishMaxWarps];      // does the row need finishing at all
     double tot[kFinishMaxWarps];     // mass of the part of the selected span each warp re-read
-    int last[kFinishMaxWarps];       // last position with mass in that part (-1 if none)
 };
 
 // warps per row: as many as the CTA can spare, each part of the span at least 256 logits (8 per lane)
@@ -343,10 +342,11 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
         // ---- one warp per row: totals, target, span ----
         if (warp < rows_per_pass) {
             const int k = k0 + warp;
-            const bool lv = k < n_rows && live(k);
+            // the triples are fetched whether or not the row turns out to be live: the two loads overlap
             RowTotals t;
             t.ok = false;
-            if (lv) t = combine_spans<MODE>(p, row0 + k, uniform(k), lane);
+            if (k < n_rows) t = combine_spans<MODE>(p, row0 + k, uniform(k), lane);
+            const bool lv = k < n_rows && live(k);
             if (lane == 0) {
                 sh.live[warp] = lv;
                 sh.row[warp] = t;
@@ -364,20 +364,16 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
         float neg_C = 0.f;
         if (active) {
             t = sh.row[kk];
-            int wl = -1;
             if (t.ok) {
                 neg_C = -t.C;
                 a0 = t.jsel * p.span;
                 b0 = min(p.V, a0 + p.span);
                 sub = p.span / wpr;
                 E = sub >> 5;
-                int lane_last;
-                lm = lane_share<DT, MODE>(p, rowp, a0 + q * sub + lane * E, E, b0, neg_C, lane_last);
+                lm = lane_share<DT, MODE>(p, rowp, a0 + q * sub + lane * E, E, b0, neg_C);
                 incl = warp_scan_incl(lm, lane);
-                wl = warp_max(lane_last);
             }
             if (lane == 31) sh.tot[warp] = incl;
-            if (lane == 0) sh.last[warp] = wl;
         }
         __syncthreads();
         // ---- the warp whose part reaches the target: the token ----
@@ -407,9 +403,13 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
                     y = locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
                 } else if (first_hit < 0 && q == 0) {
                     mine = true;  // the re-read sums fall short of the target: last token with mass in the span
-                    for (int i = 0; i < wpr; ++i) y = max(y, sh.last[w0 + i]);
+                    y = last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);
                 }
-                if (mine && lane == 0) emit(k, y >= 0 ? row_result<DT>(p, rowp, t, y) : RowResult{-1, 0.0, 0.0});
+                if (mine) {
+                    RowResult rr{-1, 0.0, 0.0};
+                    if (y >= 0) rr = row_result<DT>(p, rowp, t, y, lane);
+                    if (lane == 0) emit(k, rr);
+                }
             }
         }
         __syncthreads();  // sh is reused by the next pass; the emitted results are visible to the CTA

@@ -80,13 +80,15 @@ __device__ __forceinline__ void finishing_warp(const FusedParams& fp, int fin_id
             __threadfence();
             int tk = -1;
             double lp = 0.0, inc = 0.0;
+            ParticleState st{};
             if (lane < N) {
                 const int r = g * N + lane;
+                st = load_particle(a, r);
                 tk = __ldcg(const_cast<const int32_t*>(a.tok) + r);
                 lp = __ldcg(const_cast<const double*>(a.logp) + r);
                 inc = __ldcg(const_cast<const double*>(a.loginc) + r);
             }
-            group_update(a, g, lane, 1, sc, tk, lp, inc);
+            group_update(a, g, lane, 1, sc, tk, lp, inc, st);
             __syncwarp();  // sc is reused by the next group this warp closes
         }
     }

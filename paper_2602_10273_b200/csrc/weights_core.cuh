@@ -34,11 +34,26 @@ struct GroupScratch {
     int base[2];
 };
 
+// A particle's state as the step finds it; a kernel can fetch it early, while the row finishes are still running.
+struct ParticleState {
+    double logW, S;
+    int len;
+    unsigned char done;
+};
+__device__ __forceinline__ ParticleState load_particle(const WeightsArgs& a, int r) {
+    ParticleState s;
+    s.done = a.done[r];
+    s.S = a.S[r];
+    s.len = a.len[r];
+    s.logW = a.logW[r];
+    return s;
+}
+
 // i: this thread's index in the team (particle i when i < N).  tk_in / lp_in / inc_in: the row's drawn token
-// (-1 when the row was flagged), log p(y) and log omega; ignored for finished rows.
+// (-1 when the row was flagged), log p(y) and log omega; ignored for finished rows.  st: the particle's state.
 template <class Scratch>
 __device__ __forceinline__ void group_update(const WeightsArgs& a, int g, int i, int nw, Scratch& sc, int tk_in, double lp_in,
-                                             double inc_in) {
+                                             double inc_in, const ParticleState& st) {
     const int N = a.N;
     const bool on = i < N;
     const int r = g * N + (on ? i : 0);
@@ -46,10 +61,10 @@ __device__ __forceinline__ void group_update(const WeightsArgs& a, int g, int i,
     int tk = a.eos, ln = 0;
     unsigned char dn = 1;
     if (on) {
-        dn = a.done[r];
-        S = a.S[r];
-        ln = a.len[r];
-        lw = a.logW[r] + a.delta * S;
+        dn = st.done;
+        S = st.S;
+        ln = st.len;
+        lw = st.logW + a.delta * S;
         double lp = 0.0, inc = 0.0;
         if (!dn) {
             tk = tk_in;

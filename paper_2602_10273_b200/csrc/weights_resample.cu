@@ -26,6 +26,9 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     const int g = blockIdx.x, i = threadIdx.x, N = a.N;
 
     chain_begin();
+    // the particles' state is asked for now and used after phase 1: its latency hides behind the row finishes
+    ParticleState st{};
+    if (i < N) st = load_particle(a, g * N + i);
     // ---- phase 1: the CTA's warps finish the rows of the group's live particles ----
     finish_rows<DT, MODE>(
         ka.f, sh_fin, g * N, N, ka.wpr, [&](int k) { return a.done[g * N + k] == 0; },
@@ -42,7 +45,7 @@ __global__ void __launch_bounds__(1024) finish_weights_resample_kernel(const __g
     const int nw = (N + 31) >> 5;  // warps that hold particles
     if (nw == 1 && i >= 32) return;  // up to 32 particles: warp 0 finishes alone, on warp collectives only
     const bool on = i < N;
-    group_update(a, g, i, nw, sc, on ? sc.tok[i] : -1, on ? sc.S[i] : 0.0, on ? sc.C[i] : 0.0);
+    group_update(a, g, i, nw, sc, on ? sc.tok[i] : -1, on ? sc.S[i] : 0.0, on ? sc.C[i] : 0.0, st);
 }
 
 typedef void (*Fn)(const KernelArgs);
