@@ -4,10 +4,10 @@
  * Everything here runs in hand-written CUDA kernels; there is no CPU fallback.
  * The calls follow Algorithm 1 of the paper: N particles per prompt ("group"),
  * G independent groups, R = G*N rows.  One decoded token is one psmc_step()
- * (rows 5-11 of Algorithm 1: proposal, draw, weight update of Eq. 7, EOS
+ * (the loop body of Algorithm 1: proposal, draw, weight update of Eq. 7, EOS
  * handling, normalisation and ESS of Eq. 5, ESS-triggered systematic
- * resampling) followed by psmc_reindex_kv() (row 14, Appendix C) and, after the
- * last token, psmc_select() (row 18).
+ * resampling) followed by psmc_reindex_kv() (its cache reorder, Appendix C) and, after the
+ * last token, psmc_select() (its output step).
  *
  * Conventions
  *   - Every call returns a psmc_status; nothing throws or aborts.
@@ -57,7 +57,7 @@ typedef enum { PSMC_F32 = 0, PSMC_BF16 = 1 } psmc_dtype;
 
 /* Resampling schemes (Appendix E, "Resampling Choices": any unbiased scheme preserves the target). */
 typedef enum {
-    PSMC_RESAMPLE_SYSTEMATIC = 0,  /* Algorithm 1 row 13: positions (u0 + i)/N, one uniform per group and step */
+    PSMC_RESAMPLE_SYSTEMATIC = 0,  /* Algorithm 1, Section 6: positions (u0 + i)/N, one uniform per group and step */
     PSMC_RESAMPLE_STRATIFIED = 1,  /* positions (u_i + i)/N, one uniform per particle                            */
     PSMC_RESAMPLE_MULTINOMIAL = 2, /* positions u_i: N independent draws from Categorical(W)                     */
     PSMC_RESAMPLE_RESIDUAL = 3     /* floor(N W_j) copies of j, the rest drawn from the residual weights          */
@@ -70,7 +70,7 @@ typedef enum {
 /* One group.  N particles (1..1024), V vocabulary size (>= 2), alpha >= 1 the
  * power exponent of Eq. 1, tau > 0 the proposal temperature at full alpha
  * (Corollary 1: tau = 1/alpha is the variance-optimal choice), ess_thresh =
- * kappa in (0,1] (resample when ESS < kappa*N, row 12), ramp = T_ramp tokens of
+ * kappa in (0,1] (resample when ESS < kappa*N, Algorithm 1), ramp = T_ramp tokens of
  * linear exponent bridging (Section 4.3; 0 = off), eos_id in [0,V).  History
  * capacity T_max = 4096, initial KV length 0.  Allocates device state on the
  * current CUDA device. */
@@ -92,7 +92,7 @@ psmc_status psmc_destroy(psmc_ctx*);                 /* syncs the device, frees 
 psmc_status psmc_reset(psmc_ctx*, uint64_t seed);    /* t=0, weights 1, S=0, done=0; syncs    */
 
 /* ------------------------------------------------------------------------- */
-/* One token (Algorithm 1 rows 4-17 without the cache move)                   */
+/* One token (the loop body of Algorithm 1 without the cache move)            */
 /* ------------------------------------------------------------------------- */
 
 /* logits: DEVICE [R, V] row-major, row stride `ld` elements (>= V), dtype dt.
@@ -164,7 +164,7 @@ psmc_status psmc_logits_pass_static(const void* logits, psmc_dtype dt, int R, in
                                     int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------- */
-/* KV-cache reindex (Algorithm 1 row 14, Appendix C)                          */
+/* KV-cache reindex (Algorithm 1's cache reorder, Appendix C)                  */
 /* ------------------------------------------------------------------------- */
 typedef struct {
     int n_layers;
@@ -204,7 +204,7 @@ psmc_status psmc_reindex_kv(psmc_ctx*, const psmc_kv_desc* src, const psmc_kv_de
 /* ------------------------------------------------------------------------- */
 /* Paged KV cache with copy-on-write resampling (Appendix C on a block table)  */
 /* ------------------------------------------------------------------------- */
-/* The reorder of Algorithm 1 row 14 asks that slot k hold the cache of its ancestor.  With the cache cut into
+/* The cache reorder of Algorithm 1 asks that slot k hold the cache of its ancestor.  With the cache cut into
  * blocks of block_len positions that are reached through a per-row block table, a duplicated particle can SHARE
  * its ancestor's full blocks (a table entry and a reference count instead of a copy); only the last, partly
  * filled block is copied, because both particles go on appending to it.  The bytes moved per rewritten slot drop
@@ -245,7 +245,7 @@ const int32_t* psmc_kv_paged_refcount(psmc_ctx*);   /* [n_blocks]              *
 const int32_t* psmc_kv_paged_free_count(psmc_ctx*); /* [1] blocks on the free list */
 
 /* ------------------------------------------------------------------------- */
-/* Output (Algorithm 1 row 18)                                                */
+/* Output (last step of Algorithm 1)                                          */
 /* ------------------------------------------------------------------------- */
 
 /* Per group draws I ~ Categorical(W) from the current weights and writes the

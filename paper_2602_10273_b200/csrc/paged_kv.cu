@@ -1,4 +1,4 @@
-// Paged KV cache with copy-on-write resampling: the cache reorder of Algorithm 1 row 14 / Appendix C carried out
+// Paged KV cache with copy-on-write resampling: the cache reorder of Algorithm 1's resampling branch / Appendix C carried out
 // on a block table.  A rewritten slot gives its blocks back, takes a reference to every full block of its ancestor
 // and a private copy of the ancestor's partly filled last block.  Position p of row r lives in block
 // table[r][p / block_len] at offset p % block_len of pools laid out [n_blocks, H, block_len, D].

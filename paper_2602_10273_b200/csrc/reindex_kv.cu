@@ -1,4 +1,4 @@
-// KV-cache reindex (Algorithm 1 row 14, Appendix C): copy the live prefix of surviving rows
+// KV-cache reindex (the cache reorder of Algorithm 1's resampling branch, Appendix C): copy the live prefix of surviving rows
 // onto the rows of discarded particles, for every layer, K and V, and head.
 //
 // The move list comes from the resampling kernel as "sources": one record per surviving row

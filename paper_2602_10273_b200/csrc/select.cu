@@ -1,4 +1,4 @@
-// Output of Algorithm 1 (row 18): per group draw I ~ Categorical(W) and return the token string of
+// Output step of Algorithm 1: per group draw I ~ Categorical(W) and return the token string of
 // particle I.  Prefixes are not copied at resampling time; each step logs the tokens drawn and the
 // slot map applied, and the string is recovered here by walking that log backwards:
 //   cur = I;  for t = T..1:  cur = map_t[cur];  y_t = tok_t[cur].

@@ -1,4 +1,4 @@
-// Per-group part of the step (Algorithm 1 rows 5-16): weight update with the stage-boundary term of Section 4.3 /
+// Per-group part of the step (Algorithm 1: the per-particle updates, normalisation, trigger and resampling of its loop body): weight update with the stage-boundary term of Section 4.3 /
 // Appendix B, absorbing EOS (Appendix D), normalisation and ESS (Eq. 5), the trigger ESS < kappa N, systematic
 // resampling, the hazard-free slot map, the gather of the particle state by that map and the move records for the
 // KV reindex.  One thread per particle; a team of `nw` warps (the first threads of a CTA, or one warp on its own
