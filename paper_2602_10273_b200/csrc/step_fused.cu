@@ -1,5 +1,5 @@
-// The whole per-token step as ONE kernel (groups of up to 32 particles, 16-byte aligned rows): Algorithm 1 rows
-// 5-16 without the cache move.
+// The whole per-token step as ONE kernel (groups of up to 32 particles, 16-byte aligned rows): the loop body of
+// Algorithm 1 without the cache move.
 //
 // Every CTA (one per SM) runs up to 16 streaming warps (logits_stream.cuh) plus kFinishers finishing warps.
 // The streaming warps take the (row, span) tasks of the logit block in short runs dealt round-robin over the whole
