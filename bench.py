@@ -339,6 +339,10 @@ def run_ours(args):
         "gpu_launches": int(K * (2 + (4 if args.paged_kv else (cfg.n_layers + 63) // 64))),
         "roofline": roofline,
         "kernels": roofs,
+        # the whole step against the HBM roofline: algorithmic bytes of all its kernels over the headline time
+        "step_roofline": {"bound": "hbm", "bytes_per_step": (k1_bytes + k3_bytes) / K,
+                          "achieved": (k1_bytes + k3_bytes) * world / (ms_total * 1e-3) / 1e9 / world, "peak": hbm_peak,
+                          "unit": "GB/s", "frac": (k1_bytes + k3_bytes) / (ms_total * 1e-3) / 1e9 / hbm_peak},
         "kv_reindex": {"gb_per_s": k3_gbs, "frac_of_hbm_peak": k3_gbs / hbm_peak,
                        "slots_moved_per_step": float(np.mean(moved_slots[Wm:])),
                        "gb_moved_per_step": k3_bytes / K / 1e9},
