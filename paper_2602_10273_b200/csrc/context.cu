@@ -1,13 +1,32 @@
 // Context, argument checks and the extern "C" face of libpsmc.so.  The arithmetic of the step
 // lives in the kernels; this file owns device state, computes the exponent schedule of
 // Section 4.3 for the token at hand and enqueues the kernels on the caller's stream.
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 #include <string.h>
 #include <vector>
 
 #include "internal.h"
 
 using namespace psmc;
+
+namespace psmc {
+cudaError_t allow_dynamic_smem(const void* kernel, int bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, int> granted;  // (kernel, device) -> bytes already allowed
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    int& have = granted[std::make_pair(kernel, dev)];
+    if (have >= bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) have = bytes;
+    return e;
+}
+}  // namespace psmc
 
 struct psmc_ctx {
     int device;

@@ -13,6 +13,10 @@ namespace psmc {
 // while the previous kernel of the stream drains, which hides launch latency between the kernels of a step.
 // Every kernel launched this way calls chain_begin() before it touches global memory, and every grid of the
 // step fits the GPU in one wave, so early CTAs never keep a predecessor's CTAs from being scheduled.
+// Opt a kernel in to `bytes` of dynamic shared memory on the current device (the attribute is per function and per
+// device); remembered per (kernel, device), so the runtime is asked once each.
+cudaError_t allow_dynamic_smem(const void* kernel, int bytes);
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                   Args&&... args) {

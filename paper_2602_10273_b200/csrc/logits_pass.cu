@@ -161,17 +161,8 @@ cudaError_t launch_logits_stream(const LogitsStreamArgs& a, cudaStream_t stream)
     int64_t blocks = (n_tasks + warps - 1) / warps;
     if (blocks > kSMs) blocks = kSMs;
     const size_t smem = (size_t)warps * kDepth * kStageBytes;
-    {
-        static std::mutex mu;
-        static bool configured[2][5] = {};
-        std::lock_guard<std::mutex> lock(mu);
-        if (!configured[a.dt][g.mode]) {
-            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 kMaxWarps * kDepth * kStageBytes);
-            if (e != cudaSuccess) return e;
-            configured[a.dt][g.mode] = true;
-        }
-    }
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kMaxWarps * kDepth * kStageBytes);
+    if (e != cudaSuccess) return e;
     return launch_chained(fn, dim3((unsigned)blocks), dim3((unsigned)(warps * 32)), smem, stream, p);
 }
 

@@ -230,13 +230,9 @@ __global__ void __launch_bounds__(1024) build_moves_kernel(const int32_t* idx, i
 
 cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream) {
     if (k.bulk_ok) {
-        static bool configured = false;
         const int smem = kStages * kChunk;
-        if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(reindex_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
+        cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(reindex_bulk_kernel), smem);
+        if (e != cudaSuccess) return e;
         return launch_chained(reindex_bulk_kernel, dim3(kSMs * kBulkCtasPerSm), dim3(32), (size_t)smem, stream, k);
     }
     // widest unit that divides every address, stride and row size

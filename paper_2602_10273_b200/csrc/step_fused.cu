@@ -173,17 +173,8 @@ cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa,
     if (blocks > kSMs) blocks = kSMs;
     const size_t smem = (size_t)warps * kDepth * kStageBytes;
     FusedFn fn = la.dt == PSMC_F32 ? pick_fused<PSMC_F32>(g.mode) : pick_fused<PSMC_BF16>(g.mode);
-    {
-        static std::mutex mu;
-        static bool configured[2][5] = {};
-        std::lock_guard<std::mutex> lock(mu);
-        if (!configured[la.dt][g.mode]) {
-            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 kMaxWarps * kDepth * kStageBytes);
-            if (e != cudaSuccess) return e;
-            configured[la.dt][g.mode] = true;
-        }
-    }
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kMaxWarps * kDepth * kStageBytes);
+    if (e != cudaSuccess) return e;
     return launch_chained(fn, dim3((unsigned)blocks), dim3((unsigned)((warps + kFinishers) * 32)), smem, stream, fp);
 }
 
