@@ -105,7 +105,8 @@ psmc_status psmc_step(psmc_ctx*, const void* logits, psmc_dtype dt, int64_t ld, 
 /* The same step fed from HOST memory: copies [R,V] logits (row stride ld) to a
  * staging buffer owned by the context, runs the step, copies the R drawn
  * tokens (as seen by each slot after resampling, i.e. the next LM input) back
- * to tokens_out_host, and synchronises the stream.  Pinned host memory makes
+ * to tokens_out_host, and synchronises the stream.  The logits travel on a stream of the context's own, so the copy
+ * overlaps work still queued on `stream` (the previous token's cache move).  Pinned host memory makes
  * the copies asynchronous with respect to the host until that final sync. */
 psmc_status psmc_step_host(psmc_ctx*, const void* logits_host, psmc_dtype dt, int64_t ld,
                            int32_t* tokens_out_host, void* stream);

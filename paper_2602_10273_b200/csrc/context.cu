@@ -56,6 +56,8 @@ struct psmc_ctx {
     void* scratch;       // logit-pass tickets and span triples
     void* staging;       // psmc_step_host: device copy of the host logits
     size_t staging_bytes;
+    cudaStream_t copy_stream;  // psmc_step_host: the logits travel on a stream of their own, so that the copy
+    cudaEvent_t staged;        // overlaps whatever the caller still has running on its stream (the cache move)
     // optional per-kernel timing (psmc_timing_enable): event pairs recorded around every launch
     int timing_on;
     struct Timed { cudaEvent_t a, b; int kind; };
@@ -140,6 +142,8 @@ void free_ctx(psmc_ctx* c) {
     if (!c) return;
     for (auto& t : c->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : c->event_pool) cudaEventDestroy(e);
+    if (c->staged) cudaEventDestroy(c->staged);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
@@ -287,8 +291,15 @@ extern "C" psmc_status psmc_step_host(psmc_ctx* c, const void* logits_host, psmc
         if (cudaMalloc(&c->staging, need) != cudaSuccess) return PSMC_E_NOMEM;
         c->staging_bytes = need;
     }
+    // The staging buffer is free here: the previous call returned after its step had consumed it.  Work the caller
+    // queued since (the cache move of the previous token) keeps running while the new logits come in.
+    if (!c->copy_stream) {
+        if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PSMC_E_CUDA;
+        if (cudaEventCreateWithFlags(&c->staged, cudaEventDisableTiming) != cudaSuccess) return PSMC_E_CUDA;
+    }
     if (cudaMemcpy2DAsync(c->staging, ld_dev * esize, logits_host, ld * esize, (size_t)c->V * esize, c->R,
-                          cudaMemcpyHostToDevice, s) != cudaSuccess)
+                          cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess ||
+        cudaEventRecord(c->staged, c->copy_stream) != cudaSuccess || cudaStreamWaitEvent(s, c->staged, 0) != cudaSuccess)
         return PSMC_E_CUDA;
     psmc_status st = psmc_step(c, c->staging, dt, ld_dev, stream);
     if (st != PSMC_OK) return st;
