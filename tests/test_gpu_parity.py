@@ -78,6 +78,36 @@ def test_logits_pass_matches_oracle(dtype, beta, V):
     assert abs(loginc[4] - (1.0 - beta) * math.log(V)) < 1e-5
 
 
+def test_logits_pass_random_shapes():
+    """Forty seeded draws of (rows, vocabulary, row stride, dtype, beta, alpha_t, finished rows, -inf stretches)."""
+    rng = np.random.default_rng(20260211)
+    for case in range(40):
+        R = int(rng.integers(1, 70))
+        V = int(rng.choice([2, 3, 7, 8, 9, 31, 257, 1023, 1024, 1025, 4097, 8999]) if case % 2 else rng.integers(2, 9000))
+        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        ld = V + int(rng.choice([0, 0, 1, 3, 8, 13]))
+        beta = float(rng.choice([1.0, 2.0, 4.0, 8.0, 1.0 + 6.0 * rng.random()]))
+        alpha_t = beta if rng.random() < 0.6 else beta + 2.0 * rng.random()
+        buf = torch.full((R, ld), 7.0, device="cuda").to(dtype)          # the padding must never be read as logits
+        vals = torch.from_numpy(rng.normal(0.0, 3.0, size=(R, V)).astype(np.float32)).cuda()
+        if rng.random() < 0.4:
+            lo = int(rng.integers(0, V))
+            vals[int(rng.integers(0, R)), lo: lo + int(rng.integers(1, V))] = -math.inf
+            vals[:, int(rng.integers(0, V))] = torch.maximum(vals[:, int(rng.integers(0, V))], torch.tensor(0.0, device="cuda"))
+        vals = vals.to(dtype)
+        if torch.isinf(vals).all(dim=1).any():
+            continue                                                      # a row without mass is the error case, tested elsewhere
+        buf[:, :V] = vals
+        logits = buf[:, :V]
+        done = (rng.random(R) < 0.2).astype(np.uint8)
+        u = np.array([O.uniform(O.hash5(77, 1, case, V, r)) for r in range(R)])
+        tok, logp, loginc, status = run_logits_pass(logits, beta, alpha_t, u, done=done)
+        assert status == B.OK, (case, R, V, ld, dtype, beta)
+        live = np.nonzero(done == 0)[0]
+        assert (tok[done == 1] == -7).all()
+        check_rows_against_oracle(logits, beta, alpha_t, u, tok, logp, loginc, rows=live)
+
+
 def test_logits_pass_very_long_rows():
     """More spans per row than a lane keeps in registers (300001 logits = 293 spans of 1024), ragged end included."""
     torch.manual_seed(7)
@@ -198,6 +228,22 @@ def test_closed_loop_other_resamplers(resampler):
     c = W.CONFIGS["batched_prompts"]
     st = P.closed_loop(c, seed=2, T=12, G=4, resampler=resampler)
     assert st.resample_events > 0
+
+
+def test_closed_loop_random_settings():
+    """Twenty seeded draws of (groups, particles, vocabulary, alpha, tau, kappa, ramp, resampler), twelve tokens each."""
+    rng = np.random.default_rng(20260212)
+    for case in range(20):
+        N = int(rng.choice([1, 2, 3, 5, 8, 17, 32, 33, 64]))
+        G = int(rng.integers(1, 5))
+        V = int(rng.choice([16, 100, 1024, 3001, 20000]))
+        alpha = float(rng.choice([1.0, 2.0, 4.0, 8.0, 1.0 + 4.0 * rng.random()]))
+        tau = 1.0 / alpha if rng.random() < 0.6 else float(0.2 + rng.random())
+        c = W.Workload("case%d" % case, G, N, V, "bf16" if rng.random() < 0.5 else "f32", float(rng.choice([1.0, 3.0, 6.0])),
+                       1.5, 12, 3, 9, alpha, tau, float(rng.choice([0.3, 0.5, 0.9, 1.0])), int(rng.choice([0, 0, 4, 30])),
+                       1, 2, 16, 32)
+        st = P.closed_loop(c, seed=100 + case, T=12, kv_shape=(1, 2, 32, 16), resampler=int(rng.integers(0, 4)))
+        assert st.steps == 12
 
 
 def test_closed_loop_llama_shape():
