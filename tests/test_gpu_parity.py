@@ -370,6 +370,22 @@ def test_reindex_out_of_place_is_index_select(dtype, D):
     ps.destroy()
 
 
+def test_reindex_more_layers_than_one_launch_takes():
+    """70 layers: the pointer table of a launch holds 64, so the call takes two launches that share the unit queue."""
+    R, H, ML, D, L = 6, 1, 8, 8, 70
+    ps = B.Psmc(R, 16, 2.0, 0.5, 0.5, 0, 1, 15, T_max=2)
+    ks = [torch.randn(R, H, ML, D, device="cuda").to(torch.bfloat16) for _ in range(L)]
+    vs = [torch.randn(R, H, ML, D, device="cuda").to(torch.bfloat16) for _ in range(L)]
+    want = [t.clone() for t in ks + vs]
+    idx = torch.tensor([2, 1, 2, 2, 4, 4], dtype=torch.int32, device="cuda")
+    for _ in range(2):                                      # twice: the queue must come back to zero in between
+        ps.reindex_kv(ps.make_kv_desc(ks, vs), None, idx)
+    assert ps.sync_status() == B.OK
+    for t, w in zip(ks + vs, want):
+        assert torch.equal(t, w[idx.long()])
+    ps.destroy()
+
+
 def test_reindex_in_place_override_and_hazard_detection():
     R, H, ML, D = 6, 2, 16, 64
     ps = B.Psmc(R, 16, 2.0, 0.5, 0.5, 0, 1, 15, T_max=2)
