@@ -285,6 +285,46 @@ int psmc_rows(const psmc_ctx*);              /* R                               
 psmc_status psmc_set_state(psmc_ctx*, const double* log_w, const double* cum_logp,
                            const uint8_t* done, const int32_t* lens);
 
+/* ------------------------------------------------------------------------- */
+/* The step with the vocabulary split over P ranks                            */
+/* ------------------------------------------------------------------------- */
+
+/* A tensor-parallel LM head leaves rank p with columns [v0_p, v0_p + V_p) of every logit row (the shards tile the
+ * vocabulary in rank order).  The proposal of Corollary 1 and the weight of Eq. 7 need two row sums and one token's
+ * logit, so the step splits into three calls around two small exchanges that the CALLER performs (an all-gather
+ * over its process group; this library does no communication):
+ *
+ *   psmc_shard_sweep   reads the local columns once and writes one triple per row to triples_out (DEVICE [R][3]
+ *                      doubles: the shard's reference exponent C_p, a whole number, then sum 2^{x - C_p} and
+ *                      sum 2^{beta_t (x - C_p)} over its columns, x = logit * log2 e; zeros for finished rows)
+ *   -- all-gather --   all_triples: DEVICE [P][R][3], the ranks' triples in rank order, identical on every rank
+ *   psmc_shard_locate  every rank derives the same row totals, target mass U * Sb and owner (the first rank whose
+ *                      inclusive mass prefix reaches the target); the owner finds the token among its columns.
+ *                      picks_out: DEVICE [R]; tok = token id in the WHOLE vocabulary (v0 + local column) and
+ *                      its logit on the owner, tok = -1 elsewhere and for finished rows
+ *   -- all-gather --   all_picks: DEVICE [P][R] in rank order
+ *   psmc_shard_finish  log p(y), log omega (Eq. 7) and the rest of the step (weights, ESS, trigger, resampling,
+ *                      slot map) exactly as psmc_step does, identically on every rank
+ *
+ * Every rank creates its context with the same parameters (V = the whole vocabulary, the same seed) and the same
+ * sequence of calls, so the replicated particle state stays bit-identical across ranks and psmc_reindex_kv /
+ * psmc_select work unchanged on each rank's share of the cache.  The token drawn is the one psmc_step draws from
+ * the whole row up to the rounding of the partial sums (the inverse CDF runs over the vocabulary in its natural
+ * order).  The three calls must come in this order (PSMC_E_STATE otherwise); the logits of the sweep must stay
+ * untouched until psmc_shard_locate has run.  V_local >= 2, sum over ranks = V; v0 >= 0, v0 + V_local <= V;
+ * 1 <= P <= 1024.  A shard whose columns are all -inf is fine.  Alignment rules for the fast path as in psmc_step,
+ * applied to the shard's first column. */
+typedef struct {
+    int32_t tok;   /* token id in the whole vocabulary, -1 = not this rank's row */
+    float logit;   /* the token's logit (bf16 and fp32 are both exact in a float) */
+} psmc_shard_pick;
+psmc_status psmc_shard_sweep(psmc_ctx*, const void* logits_local, psmc_dtype dt, int64_t ld, int V_local,
+                             double* triples_out, void* stream);
+psmc_status psmc_shard_locate(psmc_ctx*, int v0, const double* all_triples, int P, int rank,
+                              psmc_shard_pick* picks_out, void* stream);
+psmc_status psmc_shard_finish(psmc_ctx*, const double* all_triples, const psmc_shard_pick* all_picks, int P,
+                              void* stream);
+
 /* Snapshot of a run, for checkpointing and for moving a run to another context.  Because all randomness is a
  * counter hash of (seed, group, step, slot), a context that loads a snapshot continues bit for bit as the one that
  * saved it would have.  The snapshot holds the particle state, the results of the last step and the ancestry log

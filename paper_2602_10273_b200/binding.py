@@ -101,6 +101,12 @@ def lib():
         for name in ("psmc_kv_paged_table", "psmc_kv_paged_refcount", "psmc_kv_paged_free_count"):
             getattr(L, name).restype = C.c_void_p
             getattr(L, name).argtypes = [vp]
+        L.psmc_shard_sweep.restype = C.c_int
+        L.psmc_shard_sweep.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_int, vp, vp]
+        L.psmc_shard_locate.restype = C.c_int
+        L.psmc_shard_locate.argtypes = [vp, C.c_int, vp, C.c_int, C.c_int, vp, vp]
+        L.psmc_shard_finish.restype = C.c_int
+        L.psmc_shard_finish.argtypes = [vp, vp, vp, C.c_int, vp]
         L.psmc_state_bytes.restype = C.c_size_t
         L.psmc_state_bytes.argtypes = [vp]
         L.psmc_state_save.restype = C.c_int
@@ -215,6 +221,33 @@ class Psmc:
         assert logits.dim() == 2 and logits.stride(1) == 1 and logits.shape == (self.R, self.V)
         _check(lib().psmc_step_host(self._h, logits.data_ptr(), _dtype_code(logits), logits.stride(0),
                                     tokens_out.data_ptr(), _stream(stream)), "psmc_step_host")
+
+    # ---- the step with the vocabulary split over ranks: three calls around two all-gathers made by the caller ----
+    def shard_sweep(self, logits_local: torch.Tensor, triples_out: torch.Tensor, stream=None):
+        """logits_local: CUDA [R, V_local] columns of this rank (unit stride along V); triples_out: CUDA float64 [R, 3]."""
+        assert logits_local.is_cuda and logits_local.dim() == 2 and logits_local.stride(1) == 1
+        assert logits_local.shape[0] == self.R
+        assert triples_out.is_cuda and triples_out.dtype == torch.float64 and triples_out.is_contiguous()
+        assert triples_out.numel() == 3 * self.R
+        _check(lib().psmc_shard_sweep(self._h, logits_local.data_ptr(), _dtype_code(logits_local),
+                                      logits_local.stride(0), logits_local.shape[1], triples_out.data_ptr(),
+                                      _stream(stream)), "psmc_shard_sweep")
+
+    def shard_locate(self, v0: int, all_triples: torch.Tensor, rank: int, picks_out: torch.Tensor, stream=None):
+        """all_triples: CUDA float64 [P, R, 3] in rank order; picks_out: CUDA int32 [R, 2] (token id, logit bits)."""
+        assert all_triples.is_cuda and all_triples.dtype == torch.float64 and all_triples.is_contiguous()
+        assert all_triples.dim() == 3 and all_triples.shape[1:] == (self.R, 3)
+        assert picks_out.is_cuda and picks_out.dtype == torch.int32 and picks_out.is_contiguous()
+        assert picks_out.numel() == 2 * self.R
+        _check(lib().psmc_shard_locate(self._h, v0, all_triples.data_ptr(), all_triples.shape[0], rank,
+                                       picks_out.data_ptr(), _stream(stream)), "psmc_shard_locate")
+
+    def shard_finish(self, all_triples: torch.Tensor, all_picks: torch.Tensor, stream=None):
+        """all_picks: CUDA int32 [P, R, 2] in rank order."""
+        assert all_picks.is_cuda and all_picks.dtype == torch.int32 and all_picks.is_contiguous()
+        assert all_picks.dim() == 3 and all_picks.shape == (all_triples.shape[0], self.R, 2)
+        _check(lib().psmc_shard_finish(self._h, all_triples.data_ptr(), all_picks.data_ptr(), all_triples.shape[0],
+                                       _stream(stream)), "psmc_shard_finish")
 
     def make_kv_desc(self, k_layers, v_layers, skip_shared_prompt: bool = False):
         """k_layers / v_layers: lists of CUDA tensors [R, H, max_len, D] with (max_len, D) contiguous.

@@ -53,7 +53,11 @@ struct psmc_ctx {
     int32_t* group_arrivals;  // [G]
     int32_t* status;
     int32_t* kv_work;    // [2] unit queue of the reindex kernels (kept at zero between launches by the kernels)
-    void* scratch;       // logit-pass tickets and span triples
+    void* scratch;       // span triples of the logit pass
+    size_t scratch_bytes;
+    // the step with the vocabulary split over ranks: 0 = idle, 1 = swept, 2 = located; the local columns of the sweep
+    int shard_phase, shard_P;
+    LogitsStreamArgs shard_la;
     void* staging;       // psmc_step_host: device copy of the host logits
     size_t staging_bytes;
     cudaStream_t copy_stream;  // psmc_step_host: the logits travel on a stream of their own, so that the copy
@@ -105,6 +109,7 @@ psmc_status reset_device_state(psmc_ctx* c) {
     delete[] h;
     delete[] hd;
     c->t = 0;
+    c->shard_phase = 0;
     return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
@@ -197,7 +202,8 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     if (e == cudaSuccess) e = cudaMemcpy(c->prompt_len_dev, c->prompt_len_host, 4 * (size_t)G, cudaMemcpyHostToDevice);
     ok(dev_alloc(&c->status, 1));
     ok(dev_alloc(&c->kv_work, 2));
-    ok(cudaMalloc(&c->scratch, logits_pass_scratch_bytes(c->R, c->V)));
+    c->scratch_bytes = logits_pass_scratch_bytes(c->R, c->V);
+    ok(cudaMalloc(&c->scratch, c->scratch_bytes));
     if (e != cudaSuccess) { free_ctx(c); return e == cudaErrorMemoryAllocation ? PSMC_E_NOMEM : PSMC_E_CUDA; }
     psmc_status st = reset_device_state(c);
     if (st != PSMC_OK) { free_ctx(c); return st; }
@@ -233,24 +239,25 @@ extern "C" psmc_status psmc_reset(psmc_ctx* c, uint64_t seed) {
     return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
-extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt, int64_t ld, void* stream) {
-    if (!c || !logits || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
-    if (c->t >= c->T_max) return PSMC_E_STATE;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int t = c->t + 1;
-    const double alpha_t = alpha_at(c, t), alpha_prev = alpha_at(c, t - 1);
-    const double beta_t = alpha_t / (c->alpha * c->tau);  // tau = 1/alpha gives beta_t = alpha_t (Corollary 1)
+namespace {
 
-    LogitsStreamArgs la{};
-    la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = beta_t;
-    la.done = c->done; la.scratch = c->scratch;
-    la.status = c->status;
-    la.zero_words = c->counts[(t + 1) & 1];  // each step clears the pair of move counters the next step will use
+// The exponents of step t (Section 4.3 / Appendix B) and everything the per-group update reads and writes.
+struct StepExponents {
+    double alpha_t, alpha_prev, beta_t;
+};
+StepExponents exponents_at(const psmc_ctx* c, int t) {
+    StepExponents x;
+    x.alpha_t = alpha_at(c, t);
+    x.alpha_prev = alpha_at(c, t - 1);
+    x.beta_t = x.alpha_t / (c->alpha * c->tau);  // tau = 1/alpha gives beta_t = alpha_t (Corollary 1)
+    return x;
+}
 
+WeightsArgs weights_args(psmc_ctx* c, int t, const StepExponents& x) {
     WeightsArgs wa{};
     wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos; wa.resampler = c->resampler;
-    wa.alpha_t = alpha_t; wa.beta = beta_t; wa.delta = alpha_t - alpha_prev; wa.kappa = c->kappa; wa.seed = c->seed;
-    wa.logits = logits; wa.dt = dt; wa.V = c->V; wa.ld = ld; wa.scratch = c->scratch;
+    wa.alpha_t = x.alpha_t; wa.beta = x.beta_t; wa.delta = x.alpha_t - x.alpha_prev; wa.kappa = c->kappa;
+    wa.seed = c->seed;
     wa.logp = c->logp; wa.loginc = c->loginc;
     wa.logW = c->logW; wa.S = c->S; wa.done = c->done; wa.len = c->len;
     wa.tok = c->tok; wa.last_tok = c->last_tok; wa.anc = c->anc; wa.map = c->map;
@@ -260,6 +267,26 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     wa.sources = c->sources[0]; wa.dst_rows = c->dst_rows[0];
     wa.n_sources = c->counts[t & 1]; wa.n_moves = c->counts[t & 1] + 1;
     wa.status = c->status;
+    return wa;
+}
+
+}  // namespace
+
+extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt, int64_t ld, void* stream) {
+    if (!c || !logits || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
+    if (c->t >= c->T_max || c->shard_phase != 0) return PSMC_E_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int t = c->t + 1;
+    const StepExponents x = exponents_at(c, t);
+
+    LogitsStreamArgs la{};
+    la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = x.beta_t;
+    la.done = c->done; la.scratch = c->scratch;
+    la.status = c->status;
+    la.zero_words = c->counts[(t + 1) & 1];  // each step clears the pair of move counters the next step will use
+
+    WeightsArgs wa = weights_args(c, t, x);
+    wa.logits = logits; wa.dt = dt; wa.V = c->V; wa.ld = ld; wa.scratch = c->scratch;
     LaunchTimer whole(c, s, 0, 2);
     if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
         LaunchTimer lt(c, s, 0);
@@ -273,6 +300,71 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
         if (launch_weights_resample(wa, s) != cudaSuccess) return PSMC_E_CUDA;
     }
     c->t = t;
+    return PSMC_OK;
+}
+
+// ---- the step with the vocabulary split over ranks (vocab_shard.cu) ----
+extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, psmc_dtype dt, int64_t ld, int V_local,
+                                        double* triples_out, void* stream) {
+    if (!c || !logits_local || !triples_out || V_local < 2 || V_local > c->V || ld < V_local ||
+        (dt != PSMC_F32 && dt != PSMC_BF16))
+        return PSMC_E_INVAL;
+    if (c->t >= c->T_max || c->shard_phase != 0) return PSMC_E_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // a shard is cut into spans of its own; with many ranks that can take a few more triples than the whole row
+    const size_t need = logits_pass_scratch_bytes(c->R, V_local);
+    if (need > c->scratch_bytes) {
+        if (cudaStreamSynchronize(s) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+        cudaFree(c->scratch);
+        c->scratch = nullptr;
+        c->scratch_bytes = 0;
+        if (cudaMalloc(&c->scratch, need) != cudaSuccess) return PSMC_E_NOMEM;
+        c->scratch_bytes = need;
+    }
+    const int t = c->t + 1;
+    const StepExponents x = exponents_at(c, t);
+    LogitsStreamArgs la{};
+    la.logits = logits_local; la.dt = dt; la.R = c->R; la.V = V_local; la.ld = ld; la.beta = x.beta_t;
+    la.done = c->done; la.scratch = c->scratch;
+    la.status = c->status;
+    la.zero_words = c->counts[(t + 1) & 1];
+    LaunchTimer lt(c, s, 0);
+    if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
+    if (launch_shard_triples(la, triples_out, s) != cudaSuccess) return PSMC_E_CUDA;
+    c->shard_la = la;
+    c->shard_phase = 1;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_shard_locate(psmc_ctx* c, int v0, const double* all_triples, int P, int rank,
+                                         psmc_shard_pick* picks_out, void* stream) {
+    if (!c || !all_triples || !picks_out || P < 1 || P > 1024 || rank < 0 || rank >= P || v0 < 0) return PSMC_E_INVAL;
+    if (c->shard_phase != 1) return PSMC_E_STATE;
+    if ((int64_t)v0 + c->shard_la.V > c->V) return PSMC_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int t = c->t + 1;
+    ShardLocateArgs sa{};
+    sa.all_triples = all_triples; sa.P = P; sa.rank = rank; sa.N = c->N; sa.t = t; sa.v0 = v0;
+    sa.alpha_t = alpha_at(c, t); sa.seed = c->seed; sa.picks_out = picks_out;
+    LaunchTimer lt(c, s, 0);
+    if (launch_shard_locate(c->shard_la, sa, s) != cudaSuccess) return PSMC_E_CUDA;
+    c->shard_P = P;
+    c->shard_phase = 2;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_shard_finish(psmc_ctx* c, const double* all_triples, const psmc_shard_pick* all_picks,
+                                         int P, void* stream) {
+    if (!c || !all_triples || !all_picks) return PSMC_E_INVAL;
+    if (c->shard_phase != 2) return PSMC_E_STATE;
+    if (P != c->shard_P) return PSMC_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int t = c->t + 1;
+    const WeightsArgs wa = weights_args(c, t, exponents_at(c, t));
+    LaunchTimer lt(c, s, 1);
+    if (launch_shard_weights(wa, all_triples, all_picks, P, s) != cudaSuccess) return PSMC_E_CUDA;
+    c->t = t;
+    c->shard_phase = 0;
     return PSMC_OK;
 }
 
@@ -493,6 +585,7 @@ extern "C" size_t psmc_state_bytes(const psmc_ctx* c) {
 
 extern "C" psmc_status psmc_state_save(psmc_ctx* c, void* host_buf, size_t bytes) {
     if (!c || !host_buf || bytes < snapshot_bytes(c, c->t)) return PSMC_E_INVAL;
+    if (c->shard_phase != 0) return PSMC_E_STATE;  // between the calls of a sharded step there is no consistent state
     if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
     SnapshotHeader h{};
     h.magic = kSnapshotMagic;
@@ -529,6 +622,7 @@ extern "C" psmc_status psmc_state_load(psmc_ctx* c, const void* host_buf, size_t
         in += ps[i].bytes;
     }
     c->t = h.t; c->ramp = h.ramp; c->eos = h.eos; c->resampler = h.resampler;
+    c->shard_phase = 0;
     c->alpha = h.alpha; c->tau = h.tau; c->kappa = h.kappa; c->seed = h.seed;
     return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }

@@ -107,6 +107,21 @@ bool step_can_fuse(const LogitsStreamArgs& la, int N);
 cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, int32_t* row_arrivals,
                               int32_t* group_arrivals, cudaStream_t stream);
 
+// ---------------------------------------------------------------- the step with the vocabulary split over ranks
+struct ShardLocateArgs {
+    const double* all_triples;  // [P][R][3]
+    int P, rank, N, t, v0;
+    double alpha_t;
+    uint64_t seed;
+    psmc_shard_pick* picks_out;  // [R]
+};
+// la describes the local columns (V = their number); its scratch holds the span triples of the streaming kernel
+cudaError_t launch_shard_triples(const LogitsStreamArgs& la, double* triples_out, cudaStream_t stream);
+cudaError_t launch_shard_locate(const LogitsStreamArgs& la, const ShardLocateArgs& sa, cudaStream_t stream);
+// a.logits / a.scratch are not used: the row results come from the gathered triples and picks
+cudaError_t launch_shard_weights(const WeightsArgs& a, const double* all_triples, const psmc_shard_pick* all_picks, int P,
+                                 cudaStream_t stream);
+
 // ---------------------------------------------------------------- KV reindex (Appendix C)
 constexpr int kMaxKvPtrs = 128;  // K and V pointers per launch (64 layers); more layers take more launches
 struct KvLaunch {

@@ -117,8 +117,18 @@ __device__ __forceinline__ void span_scales(float dcf, double beta, double& f1, 
     else fb = exp2(beta * (double)dc);
 }
 
-template <int MODE>
-__device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane) {
+// When the row is one part of a longer row (a vocabulary shard): the reference exponent of the whole row, the
+// target mass in that scale, and the mass of everything before this part.
+struct RowFrame {
+    float C;
+    double target, base;
+};
+
+// FRAMED: the triples are rescaled to fr->C instead of the row's own largest reference exponent, the prefix over the
+// spans starts at fr->base and looks for fr->target (U is not used).
+template <int MODE, bool FRAMED = false>
+__device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane,
+                                                   const RowFrame* fr = nullptr) {
     constexpr int kKeep = 8;  // span masses a lane keeps in registers between the two sweeps (rows of <= 256 spans)
     RowTotals t;
     t.ok = false;
@@ -126,8 +136,12 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     const float4* P = p.partials + (size_t)row * n;
 
     float cf = kRefFloor;
-    for (int j = lane; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
-    cf = warp_max(cf);
+    if (FRAMED) {
+        cf = fr->C;
+    } else {
+        for (int j = lane; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
+        cf = warp_max(cf);
+    }
     t.C = cf;
 
     // totals, every term rescaled to the row's reference in fp64
@@ -149,11 +163,11 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     }
     t.S1 = warp_sum(a_sum);
     t.Sb = warp_sum(b_sum);
-    if (!(t.S1 > 0.0) || !(t.Sb > 0.0) || isinf(t.S1) || isinf(t.Sb)) return t;
+    if (!FRAMED && (!(t.S1 > 0.0) || !(t.Sb > 0.0) || isinf(t.S1) || isinf(t.Sb))) return t;
 
     // span that holds the target: inclusive prefix over spans in order, 32 spans per round
-    t.target = U * t.Sb;
-    double carry = 0.0, base = 0.0, last_base = 0.0;
+    t.target = FRAMED ? fr->target : U * t.Sb;
+    double carry = FRAMED ? fr->base : 0.0, base = 0.0, last_base = 0.0;
     int jsel = -1, last_pos = -1;
     for (int c = 0, i = 0; c < n && jsel < 0; c += 32, ++i) {
         const int j = c + lane;
@@ -286,6 +300,25 @@ __device__ __forceinline__ RowResult row_result(const FinishParams& p, const voi
     return r;
 }
 
+// The token inside span t.jsel, by one warp: every lane sums its share of the span, the lane whose share reaches the
+// target is searched 32 logits at a time.  Every lane returns the same position (-1: nothing in the span has mass).
+template <int DT, int MODE>
+__device__ __forceinline__ int locate_token_warp(const FinishParams& p, const void* rowp, const RowTotals& t, int lane) {
+    const float neg_C = -t.C;
+    const int a0 = t.jsel * p.span, b0 = min(p.V, a0 + p.span);
+    const int E = p.span >> 5;
+    const double lm = lane_share<DT, MODE>(p, rowp, a0 + lane * E, E, b0, neg_C);
+    const double r_incl = t.base + warp_scan_incl(lm, lane);
+    const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+    if (hit2) {
+        const int owner = __ffs(hit2) - 1;
+        const double run = __shfl_sync(kFull, r_incl - lm, owner);
+        const int o0 = a0 + owner * E;
+        return locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+    }
+    return last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);  // the re-read sums fall short of the target
+}
+
 // ---- the finish of one row by one warp on its own (no shared memory, no CTA barrier) ----
 // Every lane returns the same RowResult.
 template <int DT, int MODE>
@@ -294,21 +327,7 @@ __device__ __forceinline__ RowResult finish_row_warp(const FinishParams& p, int 
     const RowTotals t = combine_spans<MODE>(p, row, U, lane);
     if (!t.ok) return bad;
     const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
-    const float neg_C = -t.C;
-    const int a0 = t.jsel * p.span, b0 = min(p.V, a0 + p.span);
-    const int E = p.span >> 5;
-    const double lm = lane_share<DT, MODE>(p, rowp, a0 + lane * E, E, b0, neg_C);
-    const double r_incl = t.base + warp_scan_incl(lm, lane);
-    const unsigned hit2 = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
-    int y;
-    if (hit2) {
-        const int owner = __ffs(hit2) - 1;
-        const double run = __shfl_sync(kFull, r_incl - lm, owner);
-        const int o0 = a0 + owner * E;
-        y = locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
-    } else {
-        y = last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);  // the re-read sums fall short of the target
-    }
+    const int y = locate_token_warp<DT, MODE>(p, rowp, t, lane);
     if (y < 0) return bad;
     return row_result<DT>(p, rowp, t, y, lane);
 }

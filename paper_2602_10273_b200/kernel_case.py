@@ -6,6 +6,7 @@ what-does-this-shape-cost questions:
   python -m paper_2602_10273_b200.kernel_case logits --rows 512 --vocab 128256 --beta 4 --iters 5
   python -m paper_2602_10273_b200.kernel_case reindex --rows 64 --layers 8 --heads 8 --len 1024 --iters 3
   python -m paper_2602_10273_b200.kernel_case step --workload qwen25_7b --iters 20
+  python -m paper_2602_10273_b200.kernel_case shard_step --workload batched_prompts --ranks 8 --iters 20
 
 Each case rotates through enough distinct input buffers to exceed the L2 cache, so that the
 device-time and DRAM counters describe HBM-bound behaviour.
@@ -129,9 +130,68 @@ def case_step(a):
             "gb_per_s": wl.R * cfg.logit_bytes_per_row / (np.median(us) * 1e-6) / 1e9}
 
 
+def case_shard_step(a):
+    """One rank's share of the step on a vocabulary split over --ranks ranks (this GPU plays every rank in turn; the
+    all-gathers are a stack on the device and are not timed).  Reports rank 0's three calls."""
+    from . import vocab_shard as VS
+    cfg = gen.CONFIGS[a.workload]
+    G = cfg.G if a.groups is None else a.groups
+    wl = WC.DeviceWorkload(cfg, 1, G=G)
+    shards = VS.vocab_shards(cfg.V, a.ranks)
+    n_buf = min(64, max(2, -(-2 * L2_BYTES * a.ranks // (wl.R * cfg.logit_bytes_per_row))))
+    T = a.iters + 4
+    ranks = [B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
+                    T_max=T, prompt_len=wl.prompt_len) for _ in shards]
+    bufs = [wl.new_logits() for _ in range(n_buf)]
+    prev = wl.first_prev.clone()
+    for i, b in enumerate(bufs):
+        wl.fill(b, 1 + i, prev)
+    tr = [torch.empty((wl.R, 3), dtype=torch.float64, device="cuda") for _ in shards]
+    pk = [torch.empty((wl.R, 2), dtype=torch.int32, device="cuda") for _ in shards]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = []
+    for i in range(T - 1):
+        lg = bufs[i % n_buf]
+        m = [ev() for _ in range(6)]
+        for p in range(len(shards) - 1, -1, -1):          # rank 0 last, so that its bracket is followed by the stack
+            v0, vl = shards[p]
+            if p == 0:
+                m[0].record()
+            ranks[p].shard_sweep(lg[:, v0:v0 + vl], tr[p])
+            if p == 0:
+                m[1].record()
+        all_tr = torch.stack(tr)
+        for p in range(len(shards) - 1, -1, -1):
+            if p == 0:
+                m[2].record()
+            ranks[p].shard_locate(shards[p][0], all_tr, p, pk[p])
+            if p == 0:
+                m[3].record()
+        all_pk = torch.stack(pk)
+        for p in range(len(shards) - 1, -1, -1):
+            if p == 0:
+                m[4].record()
+            ranks[p].shard_finish(all_tr, all_pk)
+            if p == 0:
+                m[5].record()
+        marks.append(m)
+    torch.cuda.synchronize()
+    assert all(r.sync_status() == B.OK for r in ranks)
+    marks = marks[-a.iters:]
+    med = lambda k: float(np.median([m[k].elapsed_time(m[k + 1]) * 1e3 for m in marks]))
+    for r in ranks:
+        r.destroy()
+    local_bytes = wl.R * shards[0][1] * (2 if cfg.dtype == "bf16" else 4)
+    return {"case": "shard_step", "workload": cfg.name, "rows": wl.R, "vocab": cfg.V, "ranks": a.ranks,
+            "local_columns": shards[0][1], "buffers": n_buf, "sweep_us": med(0), "locate_us": med(2), "finish_us": med(4),
+            "local_logit_bytes": local_bytes, "sweep_gb_per_s": local_bytes / (med(0) * 1e-6) / 1e9,
+            "gathered_bytes_per_rank": wl.R * (24 + 8)}
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("case", choices=["logits", "reindex", "step"])
+    ap.add_argument("case", choices=["logits", "reindex", "step", "shard_step"])
+    ap.add_argument("--ranks", type=int, default=8)
     ap.add_argument("--rows", type=int, default=512)
     ap.add_argument("--vocab", type=int, default=128256)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
@@ -146,7 +206,7 @@ def main():
     ap.add_argument("--no-ramp", action="store_true")
     ap.add_argument("--iters", type=int, default=5)
     a = ap.parse_args()
-    out = {"logits": case_logits, "reindex": case_reindex, "step": case_step}[a.case](a)
+    out = {"logits": case_logits, "reindex": case_reindex, "step": case_step, "shard_step": case_shard_step}[a.case](a)
     print(json.dumps(out))
 
 
