@@ -59,6 +59,13 @@ def lib():
         L.orc_row.restype = C.c_int
         L.orc_row.argtypes = [_f64p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_int,
                               C.POINTER(C.c_int), C.POINTER(C.c_int)] + [_f64p] * 6
+        L.orc_row_masked.restype = C.c_int
+        L.orc_row_masked.argtypes = [_f64p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_int, C.c_double, C.c_int,
+                                     C.c_int] + [C.POINTER(C.c_int)] * 4 + [_f64p] * 5
+        L.orc_set_proposal_mask.restype = C.c_int
+        L.orc_set_proposal_mask.argtypes = [C.c_void_p, C.c_int, C.c_double]
+        L.orc_set_force_k.restype = None
+        L.orc_set_force_k.argtypes = [C.c_void_p, _i32p]
         L.orc_ess.restype = None
         L.orc_ess.argtypes = [_f64p, C.c_int] + [_f64p] * 4
         L.orc_systematic.restype = None
@@ -93,7 +100,8 @@ def lib():
                           ("orc_anc_own", _i32p), ("orc_anc_margin", _f64p),
                           ("orc_slot_map_view", _i32p), ("orc_resampled", _i32p),
                           ("orc_resampled_own", _i32p), ("orc_ess_view", _f64p), ("orc_log_z", _f64p),
-                          ("orc_lens", _i32p), ("orc_done", _u8p)):
+                          ("orc_lens", _i32p), ("orc_done", _u8p), ("orc_k_used", _i32p), ("orc_k_own", _i32p),
+                          ("orc_k_margin", _f64p)):
             f = getattr(L, name)
             f.restype = typ
             f.argtypes = [C.c_void_p]
@@ -142,6 +150,23 @@ def row(logits, beta: float, alpha_t: float, U: float, force: int = -1) -> dict:
     names = ("logp_y", "logq_y", "log_omega", "L1", "Lbeta", "margin")
     d = {n: o.value for n, o in zip(names, out)}
     d["y"], d["y_own"] = y.value, y_own.value
+    return d
+
+
+def row_masked(logits, beta: float, alpha_t: float, U: float, top_k: int = 0, top_p: float = 0.0, force_k: int = 0,
+               force: int = -1) -> dict:
+    """One row with the proposal restricted to the top_k best tokens, or to the nucleus of mass top_p."""
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    ints = [C.c_int() for _ in range(4)]
+    out = [C.c_double() for _ in range(5)]
+    rc = lib().orc_row_masked(_ptr(l, _f64p), l.size, beta, alpha_t, U, top_k, top_p, force_k, force,
+                              *[C.byref(o) for o in ints], *[C.byref(o) for o in out])
+    if rc == 1:
+        raise ValueError("exactly one of top_k and top_p must be set")
+    if rc:
+        raise FloatingPointError("row has a NaN, a +inf or no finite logit")
+    d = {n: o.value for n, o in zip(("k_margin", "logp_y", "logq_y", "log_omega", "margin"), out)}
+    d.update({n: o.value for n, o in zip(("y", "y_own", "k", "k_own"), ints)})
     return d
 
 
@@ -226,9 +251,15 @@ class Oracle:
         if lib().orc_set_resampler(self._h, kind):
             raise ValueError("unknown resampling scheme")
 
-    def step(self, logits, dtype=None, ld=None, force_tok=None, force_resample=None, force_anc=None):
+    def set_proposal_mask(self, top_k: int = 0, top_p: float = 0.0):
+        if lib().orc_set_proposal_mask(self._h, top_k, top_p):
+            raise ValueError("at most one of top_k and top_p, top_p in (0, 1]")
+
+    def step(self, logits, dtype=None, ld=None, force_tok=None, force_resample=None, force_anc=None, force_k=None):
         """logits: numpy [R, V] of float64 / float32, or uint16 holding bf16 bit patterns."""
         a = np.ascontiguousarray(logits)
+        fk = None if force_k is None else np.ascontiguousarray(force_k, dtype=np.int32)
+        lib().orc_set_force_k(self._h, _ptr(fk, _i32p))
         if dtype is None:
             dtype = {np.dtype(np.float64): F64, np.dtype(np.float32): F32, np.dtype(np.uint16): BF16}[a.dtype]
         if ld is None:
@@ -237,6 +268,7 @@ class Oracle:
         fr = None if force_resample is None else np.ascontiguousarray(force_resample, dtype=np.int32)
         fa = None if force_anc is None else np.ascontiguousarray(force_anc, dtype=np.int32)
         rc = lib().orc_step(self._h, a.ctypes.data, dtype, ld, _ptr(ft, _i32p), _ptr(fr, _i32p), _ptr(fa, _i32p))
+        lib().orc_set_force_k(self._h, None)
         if rc == 5:
             raise FloatingPointError("a row has a NaN, a +inf or no finite logit")
         if rc:
@@ -279,6 +311,9 @@ class Oracle:
     log_z = property(lambda s: s._view("orc_log_z", s.G, np.float64))
     lens = property(lambda s: s._view("orc_lens", s.R, np.int32))
     done = property(lambda s: s._view("orc_done", s.R, np.uint8))
+    k_used = property(lambda s: s._view("orc_k_used", s.R, np.int32))
+    k_own = property(lambda s: s._view("orc_k_own", s.R, np.int32))
+    k_margin = property(lambda s: s._view("orc_k_margin", s.R, np.float64))
 
     @property
     def log_z_final(self):

@@ -109,6 +109,109 @@ int orc_row(const double* l, int V, double beta, double alpha_t, double U, int f
 }
 
 /* ------------------------------------------------------------------ */
+/* one row, proposal restricted to the top of the row                  */
+/* ------------------------------------------------------------------ */
+typedef struct { double l; int v; } ranked_t;
+static int by_logit_then_id(const void* a, const void* b) {
+    const ranked_t* x = (const ranked_t*)a;
+    const ranked_t* y = (const ranked_t*)b;
+    if (x->l > y->l) return -1;
+    if (x->l < y->l) return 1;
+    return (x->v > y->v) - (x->v < y->v);
+}
+
+int orc_row_masked(const double* l, int V, double beta, double alpha_t, double U, int top_k, double top_p,
+                   int force_k, int force_tok, int* y, int* y_own, int* k_used, int* k_own, double* k_margin,
+                   double* logp_y, double* logq_y, double* log_omega, double* margin) {
+    if ((top_k > 0) == (top_p > 0.0) || top_p > 1.0) return 1; /* exactly one rule */
+    double m = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        if (isnan(l[v]) || l[v] == INFINITY) return 5;
+        if (l[v] > m) m = l[v];
+    }
+    if (m == -INFINITY) return 5;
+    double sum1 = 0.0;
+    for (int v = 0; v < V; ++v) sum1 += exp(l[v] - m);
+    double l1 = m + log(sum1); /* p is the model's own softmax over the WHOLE vocabulary */
+
+    /* rank the tokens: larger logit first, lower id first among equals */
+    ranked_t* rk = (ranked_t*)malloc(sizeof(ranked_t) * (size_t)V);
+    for (int v = 0; v < V; ++v) { rk[v].l = l[v]; rk[v].v = v; }
+    qsort(rk, (size_t)V, sizeof(ranked_t), by_logit_then_id);
+
+    int k;
+    double kmg = 1.0;
+    if (top_k > 0) {
+        k = top_k < V ? top_k : V;
+    } else {
+        /* nucleus on the proposal: the shortest run of ranked tokens whose mass under softmax(beta l) reaches top_p */
+        double total = 0.0;
+        for (int j = 0; j < V; ++j) total += exp(beta * (rk[j].l - m));
+        double cum = 0.0;
+        k = V;
+        for (int j = 0; j < V; ++j) {
+            double prev = cum;
+            cum += exp(beta * (rk[j].l - m));
+            if (cum >= top_p * total) {
+                k = j + 1;
+                kmg = fmin(fabs(cum / total - top_p), fabs(top_p - prev / total));
+                break;
+            }
+        }
+    }
+    *k_own = k;
+    if (force_k > 0) {
+        /* how far an imposed size is from satisfying the rule (0 when it does): cum_{k-1} < top_p <= cum_k */
+        if (top_k == 0 && force_k != k) {
+            double total = 0.0, cum = 0.0, before = 0.0;
+            for (int j = 0; j < V; ++j) total += exp(beta * (rk[j].l - m));
+            for (int j = 0; j < force_k && j < V; ++j) { before = cum; cum += exp(beta * (rk[j].l - m)); }
+            double short_by = top_p - cum / total;    /* > 0: the imposed set does not reach top_p */
+            double over_by = before / total - top_p;  /* >= 0: one token fewer would have done */
+            kmg = fmax(fmax(short_by, over_by), 0.0);
+        }
+        k = force_k < V ? force_k : V;
+    }
+    *k_used = k;
+    *k_margin = kmg;
+
+    unsigned char* in = (unsigned char*)calloc((size_t)V, 1);
+    for (int j = 0; j < k; ++j) in[rk[j].v] = 1;
+    free(rk);
+
+    /* proposal q_S = softmax(beta l) restricted to S and renormalised; inverse CDF in vocabulary order over S */
+    double total = 0.0;
+    for (int v = 0; v < V; ++v) if (in[v]) total += exp(beta * (l[v] - m));
+    double lb = beta * m + log(total);
+    double target = U * total, cum = 0.0, below = 0.0, at = 0.0;
+    int pick = -1, last_pos = -1;
+    for (int v = 0; v < V; ++v) {
+        if (!in[v]) continue;
+        double e = exp(beta * (l[v] - m));
+        double prev = cum;
+        cum += e;
+        if (e > 0.0) last_pos = v;
+        if (pick < 0 && cum >= target) { pick = v; below = prev; at = cum; }
+    }
+    free(in);
+    if (pick < 0) { pick = last_pos; below = at = total; }
+    double mg = 1.0;
+    if (below > 0.0) mg = fmin(mg, fabs(U - below / total));
+    if (pick < last_pos) mg = fmin(mg, fabs(at / total - U));
+
+    int tok = force_tok >= 0 ? force_tok : pick;
+    double lp = l[tok] - l1;
+    double lq = beta * l[tok] - lb;
+    *y = tok;
+    *y_own = pick;
+    *logp_y = lp;
+    *logq_y = lq;
+    *log_omega = alpha_t * lp - lq; /* Eq. 7 with the proposal actually used */
+    *margin = mg;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
 /* Eq. 5                                                               */
 /* ------------------------------------------------------------------ */
 void orc_ess(const double* logW, int N, double* M, double* s1, double* s2, double* ess) {
@@ -269,6 +372,11 @@ struct orc_ctx {
     uint8_t* done;
     int32_t *len, *tok, *tok_own, *last_tok, *anc, *anc_own, *map, *resampled, *resampled_own;
     int32_t *tok_hist, *map_hist; /* [T_max][R] */
+    int top_k;                    /* proposal restricted to the top of the row: at most one of the two is set */
+    double top_p;
+    const int32_t* force_k;       /* [R] sizes to impose at the next step (borrowed), or NULL */
+    int32_t *k_used, *k_own;      /* [R] */
+    double* k_margin;             /* [R] */
 };
 
 static void* zalloc(size_t n) { return calloc(n ? n : 1, 1); }
@@ -298,6 +406,7 @@ orc_ctx* orc_create(int G, int N, int V, double alpha, double tau, double kappa,
     c->resampled_own = (int32_t*)zalloc(4 * (size_t)G);
     c->tok_hist = (int32_t*)zalloc(4 * R * (size_t)T_max);
     c->map_hist = (int32_t*)zalloc(4 * R * (size_t)T_max);
+    c->k_used = (int32_t*)zalloc(4 * R); c->k_own = (int32_t*)zalloc(4 * R); c->k_margin = (double*)zalloc(8 * R);
     orc_reset(c, seed);
     return c;
 }
@@ -308,7 +417,7 @@ void orc_destroy(orc_ctx* c) {
     free(c->tok_margin); free(c->ess); free(c->logZ); free(c->anc_margin); free(c->done);
     free(c->len); free(c->tok); free(c->tok_own); free(c->last_tok); free(c->anc);
     free(c->anc_own); free(c->map); free(c->resampled); free(c->resampled_own);
-    free(c->tok_hist); free(c->map_hist); free(c);
+    free(c->tok_hist); free(c->map_hist); free(c->k_used); free(c->k_own); free(c->k_margin); free(c);
 }
 
 void orc_reset(orc_ctx* c, uint64_t seed) {
@@ -365,8 +474,17 @@ int orc_step(orc_ctx* c, const void* logits, int dtype, int64_t ld, const int32_
         double U = orc_uniform(orc_hash5(c->seed, ORC_STREAM_TOKEN, (uint64_t)g, (uint64_t)t, (uint64_t)i));
         int y, y_own;
         double lp, lq, lw, l1, lb, mg;
-        int rc = orc_row(l, V, beta_t, alpha_t, U, force_tok ? force_tok[r] : -1, &y, &y_own, &lp, &lq,
+        int rc;
+        if (c->top_k > 0 || c->top_p > 0.0) {
+            int ku, ko;
+            double kmg;
+            rc = orc_row_masked(l, V, beta_t, alpha_t, U, c->top_k, c->top_p, c->force_k ? c->force_k[r] : 0,
+                                force_tok ? force_tok[r] : -1, &y, &y_own, &ku, &ko, &kmg, &lp, &lq, &lw, &mg);
+            c->k_used[r] = ku; c->k_own[r] = ko; c->k_margin[r] = kmg;
+        } else {
+            rc = orc_row(l, V, beta_t, alpha_t, U, force_tok ? force_tok[r] : -1, &y, &y_own, &lp, &lq,
                          &lw, &l1, &lb, &mg);
+        }
         free(l);
         if (rc) { bad |= 1; continue; }
         c->tok[r] = y; c->tok_own[r] = y_own; c->tok_margin[r] = mg;
@@ -507,6 +625,16 @@ const double* orc_log_inc(const orc_ctx* c) { return c->log_inc; }
 const double* orc_logp_tok(const orc_ctx* c) { return c->logp_tok; }
 const double* orc_cum_logp(const orc_ctx* c) { return c->S; }
 const int32_t* orc_ancestors(const orc_ctx* c) { return c->anc; }
+int orc_set_proposal_mask(orc_ctx* c, int top_k, double top_p) {
+    if (!c || top_k < 0 || top_p < 0.0 || top_p > 1.0 || (top_k > 0 && top_p > 0.0)) return 1;
+    c->top_k = top_k;
+    c->top_p = top_p;
+    return 0;
+}
+void orc_set_force_k(orc_ctx* c, const int32_t* force_k) { c->force_k = force_k; }
+const int32_t* orc_k_used(const orc_ctx* c) { return c->k_used; }
+const int32_t* orc_k_own(const orc_ctx* c) { return c->k_own; }
+const double* orc_k_margin(const orc_ctx* c) { return c->k_margin; }
 int orc_set_resampler(orc_ctx* c, int kind) {
     if (kind < 0 || kind > 3) return 1;
     c->resampler = kind;

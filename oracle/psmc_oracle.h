@@ -50,6 +50,21 @@ int orc_row(const double* l, int V, double beta, double alpha_t, double U, int f
             int* y, int* y_own, double* logp_y, double* logq_y, double* log_omega,
             double* L1, double* Lbeta, double* margin);
 
+/* ---- one row with the proposal restricted to a set S of tokens (a reading: the paper names top-k and nucleus
+ * only as decoding heuristics; used as an SMC proposal, the importance weight of Eq. 7 takes the proposal actually
+ * sampled from, q_S(v) = exp(beta l_v) 1[v in S] / sum_{u in S} exp(beta l_u), while p stays the model's softmax
+ * over the whole vocabulary; the target is thereby restricted to sequences the proposal can reach).
+ * Tokens are ranked by logit, larger first, lower id first among equal logits; S = the first k of that ranking.
+ *   top_k > 0, top_p == 0: k = min(top_k, V).
+ *   top_k == 0, 0 < top_p <= 1: k = the smallest k whose ranked tokens hold at least top_p of the mass of
+ *     softmax(beta l) (the proposal's own distribution, the one the temperature acts on).
+ * Exactly one of the two must be set (returns 1 otherwise).  force_k > 0 imposes the size; *k_margin then tells by
+ * how much (in mass units) that size misses the rule (0 if it satisfies it), and otherwise how close the oracle's
+ * own decision was.  The draw is the inverse CDF over S in vocabulary order; *margin as in orc_row. */
+int orc_row_masked(const double* l, int V, double beta, double alpha_t, double U, int top_k, double top_p,
+                   int force_k, int force_tok, int* y, int* y_own, int* k_used, int* k_own, double* k_margin,
+                   double* logp_y, double* logq_y, double* log_omega, double* margin);
+
 /* ---- Eq. 5 on unnormalised log-weights ---- */
 void orc_ess(const double* logW, int N, double* M, double* s1, double* s2, double* ess);
 
@@ -86,6 +101,13 @@ orc_ctx* orc_create(int G, int N, int V, double alpha, double tau, double kappa,
 void orc_destroy(orc_ctx*);
 void orc_reset(orc_ctx*, uint64_t seed);
 int orc_set_resampler(orc_ctx*, int kind); /* ORC_RESAMPLE_*; default systematic (Algorithm 1); 0 = ok */
+/* restrict the proposal of every later step as in orc_row_masked (0, 0 = whole vocabulary, the paper's proposal) */
+int orc_set_proposal_mask(orc_ctx*, int top_k, double top_p);
+/* sizes to impose at the next steps, [G*N] (0 = the oracle's own), borrowed until replaced; NULL = none */
+void orc_set_force_k(orc_ctx*, const int32_t* force_k);
+const int32_t* orc_k_used(const orc_ctx*);  /* [R] size of S as applied at the last step */
+const int32_t* orc_k_own(const orc_ctx*);   /* [R] the oracle's own size                 */
+const double* orc_k_margin(const orc_ctx*); /* [R]                                       */
 
 /* One token for every group.  logits: [G*N, V] row-major with row stride ld
  * elements, dtype ORC_*.  Hooks (each may be NULL): force_tok[G*N] (>=0 to

@@ -535,3 +535,135 @@ def test_reindex_is_index_select_on_the_particle_dimension():
             want[k, :, start[k]: lens[k]] = src[m[k], :, start[k]: lens[k]]
     assert np.array_equal(buf, want)
     assert np.array_equal(buf[0, :, :3], src[0, :, :3]) and np.array_equal(buf[0, :, 3:7], src[1, :, 3:7])
+
+
+# ---------------------------------------------------------------- proposal restricted to top-k / a nucleus
+def test_masked_proposal_hand_worked(golden_dir):
+    l = np.array([math.log(4.0), 0.0, math.log(2.0), 0.0])
+    for line in open(os.path.join(golden_dir, "masked_proposal_row.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        top_k, top_p, U, k, tok, lw, lq = line.split()
+        r = O.row_masked(l, 2.0, 2.0, float(U), top_k=int(top_k), top_p=float(top_p))
+        assert (r["k"], r["y"]) == (int(k), int(tok))
+        assert r["log_omega"] == pytest.approx(float(lw), abs=1e-13)
+        assert r["logq_y"] == pytest.approx(float(lq), abs=1e-13)
+
+
+def test_masked_proposal_with_the_whole_vocabulary_is_the_plain_row():
+    rng = np.random.default_rng(3)
+    l = rng.normal(0, 3, 50)
+    l[7] = -np.inf
+    for U in (0.01, 0.37, 0.93):
+        a, b = O.row(l, 1.7, 2.5, U), O.row_masked(l, 1.7, 2.5, U, top_k=50)
+        c = O.row_masked(l, 1.7, 2.5, U, top_k=10**6)
+        for key in ("y", "logp_y", "logq_y", "log_omega", "margin"):
+            assert a[key] == b[key] == c[key]
+
+
+def test_top_1_is_greedy_with_weight_p_to_the_alpha():
+    l = np.array([0.3, 2.0, -1.0, 2.0, 0.5])                     # two equal maxima: the lower id wins
+    lp = l - special.logsumexp(l)
+    for U in (0.001, 0.5, 0.999):
+        r = O.row_masked(l, 3.0, 4.0, U, top_k=1)
+        assert r["y"] == 1 and r["logq_y"] == 0.0
+        assert r["log_omega"] == pytest.approx(4.0 * lp[1], abs=1e-14)
+
+
+@pytest.mark.parametrize("rule", [dict(top_k=6), dict(top_p=0.8)])
+def test_masked_weight_is_constant_on_the_set_when_beta_equals_alpha(rule):
+    """Theorem 1 carried over to S: with beta = alpha_t, omega = sum_{v in S} p_v^alpha for every token of S."""
+    rng = np.random.default_rng(5)
+    l = rng.normal(0, 2, 20)
+    p = special.softmax(l)
+    seen = {}
+    for U in np.linspace(0.0005, 0.9995, 400):
+        r = O.row_masked(l, 3.0, 3.0, float(U), **rule)
+        seen[r["y"]] = r["log_omega"]
+        k = r["k"]
+    S = np.argsort(-l, kind="stable")[:k]
+    assert set(seen) <= set(S.tolist()) and len(seen) >= min(k, 4)
+    want = math.log((p[S] ** 3.0).sum())
+    for lw in seen.values():
+        assert lw == pytest.approx(want, abs=1e-12)
+
+
+@pytest.mark.parametrize("alpha,beta,rule", [(2.0, 1.3, dict(top_k=5)), (4.0, 4.0, dict(top_p=0.9)), (3.0, 0.8, dict(top_p=0.5))])
+def test_masked_weights_average_to_the_restricted_normaliser(alpha, beta, rule):
+    """sum_{v in S} q_S(v) omega(v) = sum_{v in S} p_v^alpha: enumerate S through the forcing hook, and check that
+    the frequencies of the draws over a fine grid of U are q_S."""
+    rng = np.random.default_rng(11)
+    l = rng.normal(0, 2.5, 16)
+    p = special.softmax(l)
+    k = O.row_masked(l, beta, alpha, 0.5, **rule)["k"]
+    S = np.argsort(-l, kind="stable")[:k]
+    qS = np.zeros(16)
+    qS[S] = special.softmax(beta * l[S])
+    acc = 0.0
+    for v in S:
+        r = O.row_masked(l, beta, alpha, 0.5, force=int(v), **rule)
+        assert r["logq_y"] == pytest.approx(math.log(qS[v]), abs=1e-12)
+        assert r["logp_y"] == pytest.approx(math.log(p[v]), abs=1e-12)          # p over the WHOLE vocabulary
+        acc += qS[v] * math.exp(r["log_omega"])
+    assert acc == pytest.approx((p[S] ** alpha).sum(), rel=1e-12)
+    n = 20000
+    counts = np.zeros(16)
+    for U in (np.arange(n) + 0.5) / n:
+        counts[O.row_masked(l, beta, alpha, float(U), **rule)["y"]] += 1
+    assert np.abs(counts / n - qS).max() <= 1.0 / n + 1e-12                       # inverse CDF on a grid: exact to 1/n
+    assert counts[np.setdiff1d(np.arange(16), S)].sum() == 0
+
+
+def test_nucleus_size_rule_ties_and_uniform_rows():
+    # uniform row: every token has mass 1/V, so k = ceil(top_p V), lower ids first
+    l = np.zeros(10)
+    for top_p, k in ((0.05, 1), (0.31, 4), (0.95, 10), (1.0, 10)):
+        r = O.row_masked(l, 2.0, 2.0, 0.999999, top_p=top_p)
+        assert r["k"] == k and r["y"] == k - 1                                  # the last token of S is id k-1
+    # ranked masses 0.5, 0.3, 0.15, 0.05 under beta = 1, stored out of order
+    l = np.log(np.array([0.15, 0.5, 0.05, 0.3]))
+    for top_p, k, last in ((0.4, 1, 1), (0.7, 2, 3), (0.85, 3, 3), (0.96, 4, 3)):
+        r = O.row_masked(l, 1.0, 2.0, 0.999999, top_p=top_p)
+        assert r["k"] == k and r["y"] == last
+    # the margin is the distance of top_p to the nearer of the two cumulative masses that fence the decision
+    r = O.row_masked(l, 1.0, 2.0, 0.5, top_p=0.7)
+    assert r["k_margin"] == pytest.approx(0.1, abs=1e-12)
+    # an imposed size: zero margin if it satisfies the rule, else by how much it misses
+    assert O.row_masked(l, 1.0, 2.0, 0.5, top_p=0.7, force_k=2)["k_margin"] == pytest.approx(0.1, abs=1e-12)
+    assert O.row_masked(l, 1.0, 2.0, 0.5, top_p=0.7, force_k=1)["k_margin"] == pytest.approx(0.2, abs=1e-12)   # 0.5 < 0.7
+    assert O.row_masked(l, 1.0, 2.0, 0.5, top_p=0.7, force_k=3)["k_margin"] == pytest.approx(0.1, abs=1e-12)   # 0.8 > 0.7 already
+    with pytest.raises(ValueError):
+        O.row_masked(l, 1.0, 2.0, 0.5, top_k=2, top_p=0.5)
+    with pytest.raises(ValueError):
+        O.row_masked(l, 1.0, 2.0, 0.5)
+
+
+def test_masked_steps_keep_the_normaliser_estimate_unbiased_for_the_restricted_target():
+    """With top-k proposals the particle system targets p^alpha restricted to strings whose every token lies in its
+    step's top-k set: E[Z-hat] is the sum of p(y)^alpha over exactly those strings (brute force on a tiny LM)."""
+    V, T, alpha, k = 4, 3, 3.0, 2
+    lm = TinyLM(V, 41)
+    eos = V - 1
+    # enumerate reachable strings by walking the tiny LM with the same top-k rule
+    Z = 0.0
+    stack = [((), 0.0, -1)]
+    while stack:
+        pref, logp, last = stack.pop()
+        if len(pref) == T or last == eos:
+            Z += math.exp(alpha * logp)
+            continue
+        l = lm.logits(np.array([last]))[0].astype(np.float64)
+        lp = l - special.logsumexp(l)
+        for v in np.argsort(-l, kind="stable")[:k]:
+            stack.append((pref + (int(v),), logp + lp[v], int(v)))
+    n = 12000
+    o = O.Oracle(N=4, V=V, alpha=alpha, tau=1.0 / alpha, kappa=0.9, ramp=0, seed=0, eos=eos, T_max=T)
+    o.set_proposal_mask(top_k=k)
+    zs = np.empty(n)
+    for s in range(n):
+        o.reset(9000 + s)
+        run_smc(lm, o, T)
+        zs[s] = math.exp(o.log_z_final[0])
+        assert (o.k_used[:] == k).all()
+    sem = zs.std(ddof=1) / math.sqrt(n)
+    assert abs(zs.mean() - Z) < 4.0 * sem + 1e-12, (zs.mean(), Z, sem)
