@@ -88,6 +88,23 @@ psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, float alpha, 
  * residual resampling the ancestor vector is in drawing order, not sorted. */
 psmc_status psmc_set_resampler(psmc_ctx*, psmc_resampler kind);
 
+/* Restrict the proposal of the following steps to a set S of tokens per row.  (The paper's proposal is the whole
+ * tempered distribution of Corollary 1; it names top-k and nucleus sampling only as decoding heuristics.  Used as an
+ * SMC proposal they enter Eq. 7 as the distribution actually sampled from:
+ *   q_S(v) = exp(beta_t l_v) / sum_{u in S} exp(beta_t l_u) for v in S,  log omega = alpha_t log p(y) - log q_S(y),
+ * with p the model's softmax over the WHOLE vocabulary; the particle system then targets p^alpha restricted to the
+ * sequences the proposal can reach.)  Tokens rank by logit, larger first, lower id first among equal logits (-0 and
+ * +0 are equal); S is the first k of that ranking:
+ *   top_k > 0, top_p == 0:      k = min(top_k, V)
+ *   top_k == 0, 0 < top_p <= 1: k = the smallest k whose ranked tokens hold a share top_p of softmax(beta_t l)
+ *                               (masses are compared as 2^-40 fixed-point fractions of the largest token's mass)
+ *   0, 0:                       the whole vocabulary again (the default)
+ * PSMC_E_INVAL for anything else.  The draw is the inverse CDF over S in vocabulary order with the same uniforms as
+ * the unrestricted step.  psmc_mask_sizes() holds k of every row that was live at the last step.  The restricted
+ * step runs as a pass of its own (one CTA per row: a radix search over the logits' bit patterns for the k-th ranked
+ * key, then the masked sums), not combinable with the sharded step (PSMC_E_STATE there). */
+psmc_status psmc_set_proposal_mask(psmc_ctx*, int top_k, double top_p);
+
 psmc_status psmc_destroy(psmc_ctx*);                 /* syncs the device, frees everything   */
 psmc_status psmc_reset(psmc_ctx*, uint64_t seed);    /* t=0, weights 1, S=0, done=0; syncs    */
 
@@ -272,6 +289,7 @@ const int32_t* psmc_slot_map(psmc_ctx*);     /* [R] hazard-free map applied to s
 const int32_t* psmc_resampled(psmc_ctx*);    /* [G] 0/1                                                  */
 const double*  psmc_ess(psmc_ctx*);          /* [G] ESS of Eq. 5 before resampling                       */
 const double*  psmc_log_z(psmc_ctx*);        /* [G] running log of the normaliser estimate               */
+const int32_t* psmc_mask_sizes(psmc_ctx*);    /* [R] size of the proposal's support at the last step (psmc_set_proposal_mask) */
 const int32_t* psmc_lens(psmc_ctx*);         /* [R] live KV length                                       */
 const uint8_t* psmc_done(psmc_ctx*);         /* [R]                                                      */
 const int32_t* psmc_move_count(psmc_ctx*);   /* [1] slots rewritten by the last step's maps (ask again after each step:

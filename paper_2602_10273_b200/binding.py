@@ -60,6 +60,8 @@ def lib():
         L.psmc_destroy.argtypes = [vp]
         L.psmc_set_resampler.restype = C.c_int
         L.psmc_set_resampler.argtypes = [vp, C.c_int]
+        L.psmc_set_proposal_mask.restype = C.c_int
+        L.psmc_set_proposal_mask.argtypes = [vp, C.c_int, C.c_double]
         L.psmc_reset.restype = C.c_int
         L.psmc_reset.argtypes = [vp, C.c_uint64]
         L.psmc_step.restype = C.c_int
@@ -80,7 +82,7 @@ def lib():
         L.psmc_select.argtypes = [vp, i32p, i32p, i32p, vp]
         for name in ("psmc_tokens", "psmc_last_tokens", "psmc_log_weights", "psmc_log_inc", "psmc_logp_tok",
                      "psmc_cum_logp", "psmc_ancestors", "psmc_slot_map", "psmc_resampled", "psmc_ess",
-                     "psmc_log_z", "psmc_lens", "psmc_done", "psmc_move_count"):
+                     "psmc_log_z", "psmc_lens", "psmc_done", "psmc_move_count", "psmc_mask_sizes"):
             f = getattr(L, name)
             f.restype = C.c_void_p
             f.argtypes = [vp]
@@ -161,7 +163,7 @@ _VIEW_DTYPES = {"psmc_tokens": torch.int32, "psmc_last_tokens": torch.int32, "ps
                 "psmc_log_inc": torch.float64, "psmc_logp_tok": torch.float64, "psmc_cum_logp": torch.float64,
                 "psmc_ancestors": torch.int32, "psmc_slot_map": torch.int32, "psmc_resampled": torch.int32,
                 "psmc_ess": torch.float64, "psmc_log_z": torch.float64, "psmc_lens": torch.int32,
-                "psmc_done": torch.uint8, "psmc_move_count": torch.int32, "psmc_kv_paged_table": torch.int32,
+                "psmc_mask_sizes": torch.int32, "psmc_done": torch.uint8, "psmc_move_count": torch.int32, "psmc_kv_paged_table": torch.int32,
                 "psmc_kv_paged_refcount": torch.int32, "psmc_kv_paged_free_count": torch.int32}
 
 
@@ -205,6 +207,10 @@ class Psmc:
     def set_resampler(self, kind: int) -> None:
         """psmc_set_resampler: SYSTEMATIC (default), STRATIFIED, MULTINOMIAL or RESIDUAL."""
         _check(lib().psmc_set_resampler(self._h, kind), "psmc_set_resampler")
+
+    def set_proposal_mask(self, top_k: int = 0, top_p: float = 0.0) -> None:
+        """psmc_set_proposal_mask: proposal restricted to the top_k tokens or to the nucleus of share top_p (0, 0 = off)."""
+        _check(lib().psmc_set_proposal_mask(self._h, top_k, top_p), "psmc_set_proposal_mask")
 
     def reset(self, seed):
         _check(lib().psmc_reset(self._h, seed), "psmc_reset")
@@ -373,6 +379,7 @@ class Psmc:
     ess = property(lambda s: s._view("psmc_ess", s.G))
     log_z = property(lambda s: s._view("psmc_log_z", s.G))
     lens = property(lambda s: s._view("psmc_lens", s.R))
+    mask_sizes = property(lambda s: s._view("psmc_mask_sizes", s.R))
     done = property(lambda s: s._view("psmc_done", s.R))
     move_count = property(lambda s: int(s._view("psmc_move_count", 1)[0]))
 

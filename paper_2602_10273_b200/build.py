@@ -17,8 +17,8 @@ LIB_WORKLOAD = os.path.join(PKG, "libpsmc_workload.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 
-PRODUCT_SOURCES = ["context.cu", "logits_pass.cu", "step_fused.cu", "weights_resample.cu", "vocab_shard.cu", "reindex_kv.cu",
-                   "paged_kv.cu", "select.cu"]
+PRODUCT_SOURCES = ["context.cu", "logits_pass.cu", "step_fused.cu", "weights_resample.cu", "vocab_shard.cu",
+                   "masked_proposal.cu", "reindex_kv.cu", "paged_kv.cu", "select.cu"]
 WORKLOAD_SOURCES = ["workload.cu"]
 
 

@@ -33,6 +33,9 @@ struct psmc_ctx {
     int G, N, V, R, ramp, eos, T_max, t, resampler;
     double alpha, tau, kappa;
     uint64_t seed;
+    int top_k;        // proposal restricted to the top of the row (masked_proposal.cu): at most one of the two is set
+    double top_p;
+    int32_t* set_size;  // [R] size of the proposal's support at the last step
     int32_t* prompt_len_host;  // [G]
     int32_t* prompt_len_dev;   // [G] the same on the device (for the shared-prompt form of the KV reindex)
     PagedState paged;          // block table, reference counts and free list of the paged cache (zero until created)
@@ -90,7 +93,7 @@ psmc_status reset_device_state(psmc_ctx* c) {
     z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
     z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
     z(c->counts[0], 8); z(c->counts[1], 8); z(c->counts[2], 8); z(c->status, 4); z(c->kv_work, 8);
-    z(c->row_arrivals, 4 * R); z(c->group_arrivals, 4 * G);
+    z(c->row_arrivals, 4 * R); z(c->group_arrivals, 4 * G); z(c->set_size, 4 * R);
     if (e != cudaSuccess) return PSMC_E_CUDA;
     // lens = prompt length of the group; identity maps; tokens -1; ESS = N
     int32_t* h = new (std::nothrow) int32_t[R];
@@ -152,7 +155,7 @@ void free_ctx(psmc_ctx* c) {
     void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
-                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev};
+                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev, c->set_size};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     void* paged_ptrs[] = {c->paged.table, c->paged.refc, c->paged.free_list, c->paged.free_top};
@@ -191,6 +194,7 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     ok(dev_alloc(&c->tok, R)); ok(dev_alloc(&c->last_tok, R));
     ok(dev_alloc(&c->anc, R)); ok(dev_alloc(&c->map, R)); ok(dev_alloc(&c->resampled, (size_t)G));
     ok(dev_alloc(&c->logp, R)); ok(dev_alloc(&c->loginc, R)); ok(dev_alloc(&c->ess, (size_t)G));
+    ok(dev_alloc(&c->set_size, R));
     ok(dev_alloc(&c->logZ, (size_t)G));
     ok(dev_alloc(&c->hist_tok, R * (size_t)T_max)); ok(dev_alloc(&c->hist_map, R * (size_t)T_max));
     for (int s = 0; s < 2; ++s) {
@@ -220,6 +224,14 @@ extern "C" psmc_status psmc_init(psmc_ctx** out, int N, int V, float alpha, floa
 extern "C" psmc_status psmc_set_resampler(psmc_ctx* c, psmc_resampler kind) {
     if (!c || (int)kind < 0 || (int)kind > 3) return PSMC_E_INVAL;
     c->resampler = (int)kind;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_set_proposal_mask(psmc_ctx* c, int top_k, double top_p) {
+    if (!c || top_k < 0 || !(top_p >= 0.0) || top_p > 1.0 || (top_k > 0 && top_p > 0.0)) return PSMC_E_INVAL;
+    if (c->shard_phase != 0) return PSMC_E_STATE;
+    c->top_k = top_k;
+    c->top_p = top_p;
     return PSMC_OK;
 }
 
@@ -288,7 +300,10 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
     WeightsArgs wa = weights_args(c, t, x);
     wa.logits = logits; wa.dt = dt; wa.V = c->V; wa.ld = ld; wa.scratch = c->scratch;
     LaunchTimer whole(c, s, 0, 2);
-    if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
+    if (c->top_k > 0 || c->top_p > 0.0) {  // proposal restricted to the top of the row: a pass of its own
+        LaunchTimer lt(c, s, 0);
+        if (launch_step_masked(la, wa, c->top_k, c->top_p, c->set_size, s) != cudaSuccess) return PSMC_E_CUDA;
+    } else if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
         LaunchTimer lt(c, s, 0);
         if (launch_step_fused(la, wa, c->row_arrivals, c->group_arrivals, s) != cudaSuccess) return PSMC_E_CUDA;
     } else {
@@ -310,6 +325,7 @@ extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, p
         (dt != PSMC_F32 && dt != PSMC_BF16))
         return PSMC_E_INVAL;
     if (c->t >= c->T_max || c->shard_phase != 0) return PSMC_E_STATE;
+    if (c->top_k > 0 || c->top_p > 0.0) return PSMC_E_STATE;  // ranking a row needs all of its columns
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // a shard is cut into spans of its own; with many ranks that can take a few more triples than the whole row
     const size_t need = logits_pass_scratch_bytes(c->R, V_local);
@@ -549,8 +565,10 @@ struct SnapshotHeader {
     int32_t G, N, V, T_max, t, ramp, eos, resampler;
     double alpha, tau, kappa;
     uint64_t seed;
+    double top_p;
+    int32_t top_k, reserved;
 };
-constexpr uint64_t kSnapshotMagic = 0x31434d5350ull;  // "PSMC1"
+constexpr uint64_t kSnapshotMagic = 0x32434d5350ull;  // "PSMC2"
 
 // the device arrays of a snapshot, in file order; hist arrays only up to step t
 struct Piece {
@@ -591,6 +609,7 @@ extern "C" psmc_status psmc_state_save(psmc_ctx* c, void* host_buf, size_t bytes
     h.magic = kSnapshotMagic;
     h.G = c->G; h.N = c->N; h.V = c->V; h.T_max = c->T_max; h.t = c->t; h.ramp = c->ramp; h.eos = c->eos;
     h.resampler = c->resampler; h.alpha = c->alpha; h.tau = c->tau; h.kappa = c->kappa; h.seed = c->seed;
+    h.top_k = c->top_k; h.top_p = c->top_p;
     char* out = static_cast<char*>(host_buf);
     memcpy(out, &h, sizeof(h));
     out += sizeof(h);
@@ -622,6 +641,7 @@ extern "C" psmc_status psmc_state_load(psmc_ctx* c, const void* host_buf, size_t
         in += ps[i].bytes;
     }
     c->t = h.t; c->ramp = h.ramp; c->eos = h.eos; c->resampler = h.resampler;
+    c->top_k = h.top_k; c->top_p = h.top_p;
     c->shard_phase = 0;
     c->alpha = h.alpha; c->tau = h.tau; c->kappa = h.kappa; c->seed = h.seed;
     return cudaDeviceSynchronize() == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
@@ -683,6 +703,7 @@ extern "C" const int32_t* psmc_slot_map(psmc_ctx* c) { return c ? c->map : nullp
 extern "C" const int32_t* psmc_resampled(psmc_ctx* c) { return c ? c->resampled : nullptr; }
 extern "C" const double* psmc_ess(psmc_ctx* c) { return c ? c->ess : nullptr; }
 extern "C" const double* psmc_log_z(psmc_ctx* c) { return c ? c->logZ : nullptr; }
+extern "C" const int32_t* psmc_mask_sizes(psmc_ctx* c) { return c ? c->set_size : nullptr; }
 extern "C" const int32_t* psmc_lens(psmc_ctx* c) { return c ? c->len : nullptr; }
 extern "C" const uint8_t* psmc_done(psmc_ctx* c) { return c ? c->done : nullptr; }
 extern "C" const int32_t* psmc_move_count(psmc_ctx* c) { return c ? c->counts[c->t & 1] + 1 : nullptr; }

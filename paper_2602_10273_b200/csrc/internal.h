@@ -107,6 +107,11 @@ bool step_can_fuse(const LogitsStreamArgs& la, int N);
 cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, int32_t* row_arrivals,
                               int32_t* group_arrivals, cudaStream_t stream);
 
+// The step with the proposal restricted to the top_k tokens of each row, or to the nucleus of share top_p (exactly one
+// of the two > 0): one CTA per row for the logit pass, then the per-group update.  set_size: [R].
+cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa, int top_k, double top_p,
+                               int32_t* set_size, cudaStream_t stream);
+
 // ---------------------------------------------------------------- the step with the vocabulary split over ranks
 struct ShardLocateArgs {
     const double* all_triples;  // [P][R][3]

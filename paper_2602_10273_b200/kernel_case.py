@@ -106,6 +106,8 @@ def case_step(a):
     T = 2 * a.iters + 4
     ps = B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
                 T_max=T, prompt_len=wl.prompt_len)
+    if a.top_k or a.top_p:
+        ps.set_proposal_mask(a.top_k, a.top_p)
     bufs = [wl.new_logits() for _ in range(n_buf)]
     prev = wl.first_prev.clone()
     for i, b in enumerate(bufs):
@@ -125,6 +127,7 @@ def case_step(a):
     ps.timing_enable(False)
     ps.destroy()
     return {"case": "step", "workload": cfg.name, "rows": wl.R, "vocab": cfg.V, "buffers": n_buf, "us": us,
+            "top_k": a.top_k, "top_p": a.top_p,
             "logits_stream_us": 1e3 * kms[0] / max(kn[0], 1), "finish_weights_us": 1e3 * kms[1] / max(kn[1], 1),
             "us_median": float(np.median(us)), "bytes": wl.R * cfg.logit_bytes_per_row,
             "gb_per_s": wl.R * cfg.logit_bytes_per_row / (np.median(us) * 1e-6) / 1e9}
@@ -192,6 +195,8 @@ def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("case", choices=["logits", "reindex", "step", "shard_step"])
     ap.add_argument("--ranks", type=int, default=8)
+    ap.add_argument("--top-k", type=int, default=0, help="step: proposal restricted to the top-k tokens")
+    ap.add_argument("--top-p", type=float, default=0.0, help="step: proposal restricted to the nucleus of this share")
     ap.add_argument("--rows", type=int, default=512)
     ap.add_argument("--vocab", type=int, default=128256)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])

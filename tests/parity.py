@@ -23,6 +23,7 @@ TOL_LOGINC = 1e-5    # absolute, per step
 TOK_MARGIN = 1e-6    # CDF units
 ESS_MARGIN = 1e-4    # times N
 ANC_MARGIN = 2e-4    # normalised weight-prefix units
+K_MARGIN = 4e-6      # share of the proposal's mass: how far a nucleus size may miss the rule (fp32 masses, 2^-40 fixed point)
 
 
 @dataclasses.dataclass
@@ -30,6 +31,7 @@ class LoopStats:
     steps: int = 0
     live_rows: int = 0
     tok_adopted: int = 0
+    k_adopted: int = 0
     ess_adopted: int = 0
     anc_adopted: int = 0
     resample_events: int = 0
@@ -47,7 +49,7 @@ def logits_to_numpy(t: torch.Tensor) -> np.ndarray:
 
 
 def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp: int = None, kappa: float = None,
-              resampler: int = 0):
+              resampler: int = 0, top_k: int = 0, top_p: float = 0.0):
     G = cfg.G if G is None else G
     T_max = cfg.T if T_max is None else T_max
     ramp = cfg.ramp if ramp is None else ramp
@@ -59,16 +61,25 @@ def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp
                    ramp, seed, cfg.eos_id, G=G, T_max=T_max, prompt_len=wl.prompt_len)
     ps.set_resampler(resampler)
     orc.set_resampler(resampler)
+    if top_k or top_p:
+        ps.set_proposal_mask(top_k, top_p)
+        orc.set_proposal_mask(top_k, top_p)
     return wl, ps, orc
 
 
-def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, kappa: float):
+def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, kappa: float, masked: bool = False):
     """Feed the oracle the same block (adopting flagged CUDA choices) and compare everything."""
     N, G = ps.N, ps.G
     g_tok, g_res, g_anc = ps.tokens.numpy(), ps.resampled.numpy(), ps.ancestors.numpy()
     done_before = orc.done.astype(bool)
-    orc.step(lg_host, force_tok=g_tok, force_resample=g_res, force_anc=g_anc)
+    g_k = ps.mask_sizes.numpy() if masked else None
+    orc.step(lg_host, force_tok=g_tok, force_resample=g_res, force_anc=g_anc, force_k=g_k)
     assert ps.sync_status() == B.OK
+    if masked:  # size of the proposal's support: equal, or (nucleus) the imposed size misses the rule by a rounding error
+        k_own, k_mg = orc.k_own, orc.k_margin
+        for r in np.nonzero((k_own != g_k) & ~done_before)[0]:
+            assert k_mg[r] <= K_MARGIN, "row %d: support %d vs oracle %d, margin %.3e" % (r, g_k[r], k_own[r], k_mg[r])
+            st.k_adopted += 1
 
     # tokens: equal, or the oracle's own draw sat within TOK_MARGIN of a CDF boundary
     own, mg = orc.tokens_own, orc.tok_margin
@@ -120,10 +131,12 @@ def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, 
 
 
 def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = None, kappa: float = None,
-                kv_shape=None, logit_bias_fn=None, resampler: int = 0, skip_shared_prompt: bool = False) -> LoopStats:
+                kv_shape=None, logit_bias_fn=None, resampler: int = 0, skip_shared_prompt: bool = False,
+                top_k: int = 0, top_p: float = 0.0) -> LoopStats:
     """Run T tokens on both sides.  kv_shape=(layers, heads, max_len, dim) also carries a KV cache
     through every reindex on both sides and compares the whole buffers at the end."""
-    wl, ps, orc = make_pair(cfg, seed, G=G, T_max=T, ramp=ramp, kappa=kappa, resampler=resampler)
+    wl, ps, orc = make_pair(cfg, seed, G=G, T_max=T, ramp=ramp, kappa=kappa, resampler=resampler, top_k=top_k,
+                            top_p=top_p)
     kappa_f = float(np.float32(cfg.kappa if kappa is None else kappa))
     st = LoopStats()
     lg = wl.new_logits()
@@ -157,7 +170,7 @@ def closed_loop(cfg: W.Workload, seed: int, T: int, G: int = None, ramp: int = N
         ps.step(lg)
         if kv is not None:
             ps.reindex_kv(kv["desc"])
-        compare_step(ps, orc, logits_to_numpy(lg), st, kappa_f)
+        compare_step(ps, orc, logits_to_numpy(lg), st, kappa_f, masked=bool(top_k or top_p))
         if kv is not None:
             m = orc.slot_map.reshape(ps.G, ps.N) + (np.arange(ps.G) * ps.N)[:, None]
             idx, ln = m.reshape(-1).astype(np.int32), orc.lens
