@@ -5,15 +5,32 @@
 // with p the softmax over the WHOLE row.
 //
 // One CTA per row.  A logit's bit pattern maps to an unsigned key that orders like the value, so S is
-// {key > T} plus the first `need` tokens with key == T in id order.  (T, need) come from a radix search over the
-// key, 8 bits a level from the top (2 levels for bf16, 4 for fp32): a level counts, per digit, the tokens whose
-// higher digits equal the prefix found so far -- and for the nucleus their mass 2^{beta (x - C)} as a 64-bit
-// fixed-point number (2^-40 units, integer adds: the totals do not depend on the order of the atomics) -- then picks
-// the digit in which the running count reaches k (the running mass reaches top_p of the total).  Counters live in
-// shared memory as [digit][lane] columns, so the lanes of a warp never meet on an address however the logits
-// cluster.  Tokens with equal key have equal mass, so on the last level need = ceil(remaining mass / mass of one).
-// Then two ordered sweeps (every warp owns a contiguous stretch of the row): the mass of S per warp, and, in the
-// warp whose stretch holds U * sum, the token.  The row is read from HBM once; the other sweeps hit L2.
+// {key > T} plus the first `need` tokens with key == T in id order.
+//
+// A top_k of up to half the CTA's threads goes by a threshold: every thread sees its own share of the row, so the
+// k-th largest of the threads' maxima has at least k logits at or above it (and, the shares being interleaved, hardly
+// more).  One sweep finds the maxima, a second collects the logits at or above the threshold into a candidate list in
+// shared memory (and sums the normaliser of p), and the search for (T, need) runs on that list.
+//
+// Otherwise (T, need) come from a radix search over the key, 8 bits a level from the top (2 levels for bf16, 4 for
+// fp32): a level counts, per digit, the tokens whose higher digits equal the prefix found so far -- and for the
+// nucleus their mass 2^{beta (x - C)} as a 64-bit fixed-point number (2^-40 units, integer adds: the totals do not
+// depend on the order of the atomics) -- then picks the digit in which the running count reaches k (the running mass
+// reaches top_p of the total).  Counters live in shared memory as [digit][lane] columns (masses: two lanes a column),
+// so the lanes of a warp do not pile up on an address however the logits cluster.  Tokens with equal key have equal
+// mass, so on the last level need = ceil(remaining mass / mass of one).  Sweeps over the row when counting:
+//   1  the largest logit, NaN / +inf check; for top-k also the counts of the first level (digits need no reference)
+//   2  nucleus only: counts and masses of the first level
+//   3  the second level, and sum 2^{x - C} over the whole row (the normaliser of p)
+//   4  every token whose leading 16 key bits are at or above the 16 chosen goes to the candidate list (id, bits): for
+//      bf16 exactly S and the ties at the cut, for fp32 also the tokens that agree with the cut to bf16 precision
+//
+// Everything else works on the list: the levels not yet decided; then the candidates at or above the cut are kept and
+// sorted by id (bitonic; k plus the ties at the cut, a short list), and the ties' ranks, the masses of S and the
+// inverse CDF are block scans over threads that hold consecutive entries.  The first sweep comes from HBM, the others
+// mostly from L2; all use 16-byte loads, four in flight per thread.  Rows whose candidates do not fit the list (a
+// top_k in the tens of thousands, a nearly flat nucleus, a crowd of equal logits) fall back to sweeps over the row
+// for every remaining step.
 #include "internal.h"
 #include "logits_common.cuh"
 #include "weights_core.cuh"
@@ -23,7 +40,12 @@ namespace {
 
 constexpr int kDigits = 256;
 constexpr float kFixOne = 1099511627776.f;  // 2^40: fixed-point unit of the nucleus masses (masses are <= 1)
-constexpr size_t kHistBytes = (size_t)kDigits * 32 * (sizeof(uint32_t) + sizeof(unsigned long long));
+// Dynamic shared memory: the counters ([256][32] counts; for the nucleus also [256][16] 64-bit masses, two lanes a
+// column), then the candidate list (8 bytes an entry).  The counters' memory later takes the sorted list, so the
+// list is no longer than the counts are.  64 KB (top-k) or 96 KB (nucleus) in all, so two CTAs of 512 threads share
+// an SM: one sweeps its row while the other is in the barrier-heavy work on its list.
+constexpr int kCountBytes = kDigits * 32 * 4, kMassBytes = kDigits * 16 * 8;
+constexpr int kListCap = kCountBytes / 8;  // 4096 entries
 
 struct MaskedParams {
     const void* logits;
@@ -46,10 +68,18 @@ struct MaskedParams {
 
 template <int DT>
 __device__ __forceinline__ uint32_t key_of(uint32_t b) {
-    constexpr uint32_t sign = DT == PSMC_BF16 ? 0x8000u : 0x80000000u;
-    constexpr uint32_t all = DT == PSMC_BF16 ? 0xffffu : 0xffffffffu;
-    if (b == sign) b = 0;  // -0 ranks with +0
-    return (b & sign) ? (~b & all) : (b | sign);
+    constexpr int kTop = DT == PSMC_BF16 ? 15 : 31;
+    constexpr uint32_t sign = 1u << kTop, all = DT == PSMC_BF16 ? 0xffffu : 0xffffffffu;
+    // negative values: every bit flipped; others: the sign bit set.  -0 would land one below +0: moved up onto it.
+    const uint32_t key = (b ^ ((0u - (b >> kTop)) | sign)) & all;
+    return key + (key == sign - 1u);
+}
+// the bit pattern a key came from (of +0 for the key the two zeros share)
+template <int DT>
+__device__ __forceinline__ uint32_t bits_of_key(uint32_t key) {
+    constexpr int kTop = DT == PSMC_BF16 ? 15 : 31;
+    constexpr uint32_t sign = 1u << kTop, all = DT == PSMC_BF16 ? 0xffffu : 0xffffffffu;
+    return (key & sign) ? (key ^ sign) : (~key & all);
 }
 template <int DT>
 __device__ __forceinline__ float value_of(uint32_t b) {
@@ -61,30 +91,46 @@ __device__ __forceinline__ uint32_t load_bits(const void* rowp, int i) {
     return __ldg(reinterpret_cast<const unsigned short*>(rowp) + i);
 }
 
-// f(bits) for every logit of the row, in no particular order: 16-byte loads between the first and the last
-// 16-byte boundary, single loads for the ragged ends.
-template <int DT, class F>
-__device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f) {
+// f(bits, id) for every logit of the row, in no particular order: 16-byte loads between the first and the last
+// 16-byte boundary (four in flight per thread), single loads for the ragged ends.  flush() runs after every group of
+// up to eight logits handed to f (so that f can sum in fp32 and flush can fold the partial sum into a double).
+template <int DT, class F, class G>
+__device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f, G flush) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4, kEs = DT == PSMC_BF16 ? 2 : 4;
     int head = (int)(((16 - (reinterpret_cast<uintptr_t>(rowp) & 15)) & 15) / kEs);
     if (head > V) head = V;
     const int nvec = (V - head) / kPer, tail0 = head + nvec * kPer;
     const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)head * kEs);
-    for (int j = threadIdx.x; j < nvec; j += blockDim.x) {
-        const uint4 v = __ldg(&q[j]);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (int j0 = threadIdx.x; j0 < nvec; j0 += 4 * blockDim.x) {
+        uint4 v[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (DT == PSMC_BF16) {
-                f(w[c] & 0xffffu);
-                f(w[c] >> 16);
-            } else {
-                f(w[c]);
+        for (int u = 0; u < 4; ++u)
+            if (j0 + u * (int)blockDim.x < nvec) v[u] = __ldg(&q[j0 + u * blockDim.x]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u * (int)blockDim.x;
+            if (j >= nvec) break;
+            const int i0 = head + j * kPer;
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (DT == PSMC_BF16) {
+                    f(w[c] & 0xffffu, i0 + 2 * c);
+                    f(w[c] >> 16, i0 + 2 * c + 1);
+                } else {
+                    f(w[c], i0 + c);
+                }
             }
+            flush();
         }
     }
-    for (int i = threadIdx.x; i < head; i += blockDim.x) f(load_bits<DT>(rowp, i));
-    for (int i = tail0 + threadIdx.x; i < V; i += blockDim.x) f(load_bits<DT>(rowp, i));
+    for (int i = threadIdx.x; i < head; i += blockDim.x) f(load_bits<DT>(rowp, i), i);
+    for (int i = tail0 + threadIdx.x; i < V; i += blockDim.x) f(load_bits<DT>(rowp, i), i);
+    flush();
+}
+template <int DT, class F>
+__device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f) {
+    for_each_logit<DT>(rowp, V, f, [] {});
 }
 
 struct Selection {      // what the radix search has settled so far (shared, written by warp 0)
@@ -173,18 +219,88 @@ __device__ __forceinline__ void pick_digit(Selection& sel, const uint32_t* tot_c
     }
 }
 
+// One level of the search over candidates held in the shared-memory list: entries whose key matches the prefix so far
+// (level 0 has no prefix to match).
+template <int DT, int MODE>
+__device__ __forceinline__ void count_list_level(const unsigned long long* list, int n_list, int level, uint32_t prefix,
+                                                 bool nucleus, float neg_C, float bf, uint32_t* cnt,
+                                                 unsigned long long* mass, int lane) {
+    constexpr int kKeyBits = DT == PSMC_BF16 ? 16 : 32;
+    const int shift = kKeyBits - 8 * (level + 1);
+    for (int j = threadIdx.x; j < n_list; j += blockDim.x) {
+        const uint32_t b = (uint32_t)list[j];
+        const uint32_t key = key_of<DT>(b);
+        if (level > 0 && (key >> (shift + 8)) != prefix) continue;
+        const uint32_t d = (key >> shift) & 255u;
+        atomicAdd(&cnt[d * 32 + lane], 1u);
+        if (nucleus)
+            atomicAdd(&mass[d * 16 + (lane & 15)],
+                      __float2ull_rn(logit_mass<MODE>(value_of<DT>(b), neg_C, bf) * kFixOne));
+    }
+}
+
+// Sum the [digit][lane] columns into per-digit totals (every thread of the CTA calls this; ends on a barrier).
+__device__ __forceinline__ void fold_columns(const uint32_t* cnt, const unsigned long long* mass, bool nucleus,
+                                             uint32_t* tot_cnt, unsigned long long* tot_mass) {
+    __syncthreads();
+    for (int d = threadIdx.x; d < kDigits; d += blockDim.x) {
+        uint32_t c = 0;
+        unsigned long long m = 0;
+        for (int j = 0; j < 32; ++j) {  // thread d starts at column d, so the threads of a warp read different banks
+            const int col = (j + d) & 31;
+            c += cnt[d * 32 + col];
+            if (nucleus && j < 16) m += mass[d * 16 + (col & 15)];
+        }
+        tot_cnt[d] = c;
+        tot_mass[d] = m;
+    }
+    __syncthreads();
+}
+__device__ __forceinline__ void clear_columns(uint32_t* cnt, unsigned long long* mass, bool nucleus) {
+    for (int i = threadIdx.x; i < kDigits * 32; i += blockDim.x) {
+        cnt[i] = 0;
+        if (nucleus && i < kDigits * 16) mass[i] = 0;
+    }
+    __syncthreads();
+}
+
+// Ascending bitonic sort of n2 (a power of two) 64-bit words in shared memory by the whole CTA.
+__device__ __forceinline__ void sort_words(unsigned long long* a, int n2) {
+    for (int k = 2; k <= n2; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < n2; i += blockDim.x) {
+                const int o = i ^ j;
+                if (o > i) {
+                    const unsigned long long x = a[i], y = a[o];
+                    const bool up = (i & k) == 0;
+                    if ((x > y) == up) {
+                        a[i] = y;
+                        a[o] = x;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
 template <int DT, int MODE>
 __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_constant__ MaskedParams p) {
     extern __shared__ __align__(16) unsigned char hist_raw[];
-    uint32_t* cnt = reinterpret_cast<uint32_t*>(hist_raw);                                       // [256][32]
-    unsigned long long* mass = reinterpret_cast<unsigned long long*>(hist_raw + kDigits * 32 * 4);  // [256][32]
+    const bool nucleus = p.top_k == 0;
+    uint32_t* cnt = reinterpret_cast<uint32_t*>(hist_raw);                                      // [256][32]
+    unsigned long long* mass = reinterpret_cast<unsigned long long*>(hist_raw + kCountBytes);  // [256][16], nucleus only
+    unsigned long long* list =                                                                  // [kListCap] id << 32 | bits
+        reinterpret_cast<unsigned long long*>(hist_raw + kCountBytes + (nucleus ? kMassBytes : 0));
     __shared__ double red[33];
-    __shared__ float redf[33];
+    __shared__ uint32_t redu[64];
+    __shared__ int redi[33];
     __shared__ uint32_t tot_cnt[kDigits];
     __shared__ unsigned long long tot_mass[kDigits];
     __shared__ Selection sel;
     __shared__ double wmass[32];
     __shared__ int wties[32];
+    __shared__ int n_list_sh, first_hit, last_mass;
 
     constexpr int kKeyBits = DT == PSMC_BF16 ? 16 : 32, kLevels = kKeyBits / 8;
     const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -193,18 +309,46 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
     if (p.done[row]) return;
     const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
-    const bool nucleus = p.top_k == 0;
+    const int g = row / p.N;
+    const double U = hash_uniform(hash5(p.seed, kStreamToken, (uint64_t)g, (uint64_t)p.t, (uint64_t)(row - g * p.N)));
 
-    // ---- the row's largest logit; NaN and +inf make the row unusable ----
-    float mx = -INFINITY;
-    int bad = 0;
-    for_each_logit<DT>(rowp, V, [&](uint32_t b) {
-        const float l = value_of<DT>(b);
-        bad |= (l != l) || l == INFINITY;
-        mx = fmaxf(mx, l);
+    if (threadIdx.x == 0) {
+        sel.prefix = 0;
+        sel.k_rem = (uint32_t)min(p.top_k, V);
+        sel.m_rem = 0;
+        sel.above = 0;
+        n_list_sh = 0;
+        first_hit = 0x7fffffff;
+        last_mass = -1;
+    }
+    clear_columns(cnt, mass, nucleus);
+
+    // ---- sweep 1: the row's largest logit; NaN and +inf make the row unusable; top-k by counting: first-level counts ----
+    const bool by_threshold = !nucleus && 2 * p.top_k <= (int)blockDim.x;
+    constexpr int kShift0 = kKeyBits - 8;
+    // (on keys: a NaN or +inf ranks at or above +inf's key, or below -inf's)
+    constexpr uint32_t kPosInf = DT == PSMC_BF16 ? 0xff80u : 0xff800000u, kNegInf = DT == PSMC_BF16 ? 0x007fu : 0x007fffffu;
+    uint32_t kmax = 0u, kmin = 0xffffffffu;
+    for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
+        const uint32_t key = key_of<DT>(b);
+        kmax = max(kmax, key);
+        kmin = min(kmin, key);
+        if (!nucleus && !by_threshold) atomicAdd(&cnt[(key >> kShift0) * 32 + lane], 1u);
     });
-    mx = block_max(mx, redf, nw);
-    bad = __syncthreads_or(bad);
+    const uint32_t my_max = kmax;
+    kmax = __reduce_max_sync(kFull, kmax);
+    kmin = __reduce_min_sync(kFull, kmin);
+    if (lane == 0) {
+        redu[warp] = kmax;
+        redu[32 + warp] = kmin;
+    }
+    __syncthreads();
+    for (int w = 0; w < nw; ++w) {
+        kmax = max(kmax, redu[w]);
+        kmin = min(kmin, redu[32 + w]);
+    }
+    const bool bad = kmax >= kPosInf || kmin < kNegInf;
+    const float mx = value_of<DT>(bits_of_key<DT>(kmax));
     if (bad || mx == -INFINITY) {
         if (threadIdx.x == 0) {
             raise_status(p.status, PSMC_E_NUMERIC);
@@ -217,45 +361,207 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     }
     const float C = ref_exponent(mx), neg_C = -C;
 
-    // ---- radix search for (T, need); the first level also sums 2^{x - C} over the whole row ----
-    if (threadIdx.x == 0) {
-        sel.prefix = 0;
-        sel.k_rem = (uint32_t)min(p.top_k, V);
-        sel.m_rem = 0;
-        sel.above = 0;
-    }
+    bool have_list = false;
+    int first_list_level = 2;
     double s1 = 0.0;
     uint32_t prefix = 0;
-    for (int level = 0; level < kLevels; ++level) {
-        const int shift = kKeyBits - 8 * (level + 1);
-        for (int i = threadIdx.x; i < kDigits * 32; i += blockDim.x) {
-            cnt[i] = 0;
-            if (nucleus) mass[i] = 0;
+    auto append = [&](uint32_t b, int i) {
+        const int pos = atomicAdd(&n_list_sh, 1);
+        if (pos < kListCap) list[pos] = ((unsigned long long)(uint32_t)i << 32) | b;
+    };
+
+    if (by_threshold) {
+        // ---- the threshold: the k-th largest of the threads' maxima ----
+        const int n_thr = (int)blockDim.x;  // a power of two
+        list[threadIdx.x] = my_max;
+        __syncthreads();
+        sort_words(list, n_thr);
+        const uint32_t theta = (uint32_t)list[n_thr - min(p.top_k, V)];
+        __syncthreads();  // the list's memory is handed over to the candidates
+        // ---- sweep 2: the normaliser of p, and every logit at or above the threshold into the list ----
+        float part = 0.f;
+        for_each_logit<DT>(
+            rowp, V,
+            [&](uint32_t b, int i) {
+                part += ex2(rel_exponent(value_of<DT>(b), neg_C));
+                if (key_of<DT>(b) >= theta) append(b, i);
+            },
+            [&] {
+                s1 += (double)part;
+                part = 0.f;
+            });
+        __syncthreads();
+        if (n_list_sh <= kListCap) {
+            have_list = true;
+            first_list_level = 0;
+        } else {  // a crowd at the threshold (a row of equal logits, say): count digits after all
+            __syncthreads();
+            if (threadIdx.x == 0) n_list_sh = 0;
+            s1 = 0.0;
+            for_each_logit<DT>(rowp, V, [&](uint32_t b, int) { atomicAdd(&cnt[(key_of<DT>(b) >> kShift0) * 32 + lane], 1u); });
+        }
+    }
+
+    bool listed = have_list;
+    if (!have_list) {
+        // ---- sweep 2 (nucleus): first-level counts and masses, which need the reference exponent ----
+        if (nucleus) {
+            for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
+                const uint32_t d = key_of<DT>(b) >> kShift0;
+                atomicAdd(&cnt[d * 32 + lane], 1u);
+                atomicAdd(&mass[d * 16 + (lane & 15)],
+                          __float2ull_rn(logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf) * kFixOne));
+            });
+        }
+        fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+        if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, true, kLevels == 1, p.top_p, lane);
+        __syncthreads();
+        prefix = sel.prefix;
+
+        // ---- sweep 3: the second level (tokens whose first digit is the chosen one), and the normaliser of p ----
+        constexpr int kShift1 = kKeyBits - 16;
+        clear_columns(cnt, mass, nucleus);
+        float part = 0.f;
+        for_each_logit<DT>(
+            rowp, V,
+            [&](uint32_t b, int) {
+                const float l = value_of<DT>(b);
+                part += ex2(rel_exponent(l, neg_C));
+                const uint32_t key = key_of<DT>(b);
+                if ((key >> kShift0) != prefix) return;
+                const uint32_t d = (key >> kShift1) & 255u;
+                atomicAdd(&cnt[d * 32 + lane], 1u);
+                if (nucleus)
+                    atomicAdd(&mass[d * 16 + (lane & 15)], __float2ull_rn(logit_mass<MODE>(l, neg_C, p.bf) * kFixOne));
+            },
+            [&] {
+                s1 += (double)part;
+                part = 0.f;
+            });
+        fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+        if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, false, kLevels == 2, p.top_p, lane);
+        __syncthreads();
+        prefix = sel.prefix;
+        // tokens whose leading 16 key bits are at or above the 16 chosen so far: S, the ties at the cut, and (fp32)
+        // the tokens that share the cut's leading bits
+        listed = (int)(sel.above + tot_cnt[prefix & 255u]) <= kListCap;
+        if (listed) {
+            // ---- sweep 4: the candidates into the list ----
+            const uint32_t cut = prefix << (kKeyBits - 16);
+            for_each_logit<DT>(rowp, V, [&](uint32_t b, int i) {
+                if (key_of<DT>(b) >= cut) append(b, i);
+            });
+        }
+    }
+
+    if (listed) {
+        __syncthreads();
+        const int n_cands = min(n_list_sh, kListCap);
+
+        // ---- the levels not yet decided, over the candidates in whatever order they arrived ----
+        for (int level = first_list_level; level < kLevels; ++level) {
+            clear_columns(cnt, mass, nucleus);
+            count_list_level<DT, MODE>(list, n_cands, level, prefix, nucleus, neg_C, p.bf, cnt, mass, lane);
+            fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+            if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, level == 0, level == kLevels - 1, p.top_p, lane);
+            __syncthreads();
+            prefix = sel.prefix;
+        }
+        const double S1 = block_sum(s1, red, nw);
+        const uint32_t T = prefix, need = sel.need;
+        const bool all_ties = need == sel.n_ties;
+        const int set_size = (int)(sel.above + need);
+
+        // ---- keep the candidates at or above the cut (S and the ties at T), sorted by token id ----
+        // The counters are done with; their memory takes the second list.
+        unsigned long long* kept = reinterpret_cast<unsigned long long*>(hist_raw);
+        if (threadIdx.x == 0) n_list_sh = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < n_cands; j += blockDim.x) {
+            const unsigned long long w = list[j];
+            if (key_of<DT>((uint32_t)w) >= T) kept[atomicAdd(&n_list_sh, 1)] = w;
         }
         __syncthreads();
-        for_each_logit<DT>(rowp, V, [&](uint32_t b) {
-            const float l = value_of<DT>(b);
-            if (level == 0) s1 += (double)ex2(rel_exponent(l, neg_C));
+        const int n_list = n_list_sh;  // = tokens above the cut + ties at it <= n_cands
+        int n2 = 1;
+        while (n2 < n_list) n2 <<= 1;
+        for (int i = n_list + threadIdx.x; i < n2; i += blockDim.x) kept[i] = ~0ull;
+        __syncthreads();
+        sort_words(kept, n2);  // vocabulary order
+
+        // ---- ordered part: thread t holds entries [e0, e1) of the sorted list ----
+        const int E = (n_list + (int)blockDim.x - 1) / (int)blockDim.x;
+        const int e0 = min(n_list, (int)threadIdx.x * E), e1 = min(n_list, e0 + E);
+        int c = 0;
+        for (int j = e0; j < e1; ++j) c += key_of<DT>((uint32_t)kept[j]) == T;
+        const int tie_base = block_scan_incl(c, redi, (int*)nullptr, nw) - c;
+        auto entry_mass = [&](unsigned long long w, int& rank) -> double {  // mass of an entry if it is in S, else 0
+            const uint32_t b = (uint32_t)w, key = key_of<DT>(b);
+            bool in = key > T;
+            if (key == T) {
+                in = all_ties || (uint32_t)rank < need;
+                ++rank;
+            }
+            return in ? (double)logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf) : 0.0;
+        };
+        double acc = 0.0;
+        int rank = tie_base;
+        for (int j = e0; j < e1; ++j) acc += entry_mass(kept[j], rank);
+        double Sb;
+        const double incl = block_scan_incl(acc, red, &Sb, nw);
+        const double target = U * Sb;
+        if (acc > 0.0) {
+            if (incl >= target) atomicMin(&first_hit, (int)threadIdx.x);
+            atomicMax(&last_mass, (int)threadIdx.x);
+        }
+        __syncthreads();
+        const int owner = first_hit != 0x7fffffff ? first_hit : last_mass;
+        if ((int)threadIdx.x != owner) {
+            if (threadIdx.x == 0 && owner < 0) {  // no entry of S has mass: cannot happen while the largest logit is in S
+                raise_status(p.status, PSMC_E_NUMERIC);
+                p.tok[row] = -1;
+                p.logp[row] = 0.0;
+                p.loginc[row] = 0.0;
+                p.set_size[row] = set_size;
+            }
+            return;
+        }
+        double run = incl - acc;
+        int y = -1, last = -1;
+        rank = tie_base;
+        for (int j = e0; j < e1 && y < 0; ++j) {
+            const double m = entry_mass(kept[j], rank);
+            run += m;
+            if (m > 0.0) {
+                last = (int)(kept[j] >> 32);
+                if (run >= target) y = last;
+            }
+        }
+        if (y < 0) y = last;
+        const double dl = (double)load_elem<DT>(rowp, y) - (double)C * kLn2;
+        const double ln_s1 = log(S1), ln_sb = log(Sb);
+        p.tok[row] = y;
+        p.logp[row] = dl - ln_s1;
+        p.loginc[row] = (p.alpha_t - p.beta) * dl - p.alpha_t * ln_s1 + ln_sb;
+        p.set_size[row] = set_size;
+        return;
+    }
+
+    // ---- too many candidates for the list: every remaining step sweeps the row ----
+    for (int level = 2; level < kLevels; ++level) {
+        const int shift = kKeyBits - 8 * (level + 1);
+        clear_columns(cnt, mass, nucleus);
+        for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
             const uint32_t key = key_of<DT>(b);
-            if (level > 0 && (key >> (shift + 8)) != prefix) return;
+            if ((key >> (shift + 8)) != prefix) return;
             const uint32_t d = (key >> shift) & 255u;
             atomicAdd(&cnt[d * 32 + lane], 1u);
             if (nucleus)
-                atomicAdd(&mass[d * 32 + lane], __float2ull_rn(logit_mass<MODE>(l, neg_C, p.bf) * kFixOne));
+                atomicAdd(&mass[d * 16 + (lane & 15)],
+                          __float2ull_rn(logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf) * kFixOne));
         });
-        __syncthreads();
-        for (int d = threadIdx.x; d < kDigits; d += blockDim.x) {
-            uint32_t c = 0;
-            unsigned long long m = 0;
-            for (int j = 0; j < 32; ++j) {
-                c += cnt[d * 32 + j];
-                if (nucleus) m += mass[d * 32 + j];
-            }
-            tot_cnt[d] = c;
-            tot_mass[d] = m;
-        }
-        __syncthreads();
-        if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, level == 0, level == kLevels - 1, p.top_p, lane);
+        fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+        if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, false, level == kLevels - 1, p.top_p, lane);
         __syncthreads();
         prefix = sel.prefix;
     }
@@ -264,7 +570,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     const bool all_ties = need == sel.n_ties;
     const int set_size = (int)(sel.above + need);
 
-    // ---- ordered sweeps: warp w owns logits [lo, hi) ----
+    // ordered sweeps: warp w owns logits [lo, hi)
     const int seg = (((V + nw - 1) / nw) + 31) & ~31;
     const int lo = min(V, warp * seg), hi = min(V, lo + seg);
     int tie_base = 0;
@@ -279,7 +585,6 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         __syncthreads();
         for (int w = 0; w < warp; ++w) tie_base += wties[w];
     }
-    // is token i (key, tie rank within the row) in S
     auto in_set = [&](uint32_t key, bool tie, int rank) { return key > T || (tie && (all_ties || (uint32_t)rank < need)); };
     {
         double acc = 0.0;
@@ -301,8 +606,6 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     __syncthreads();
     double Sb = 0.0;
     for (int w = 0; w < nw; ++w) Sb += wmass[w];
-    const int g = row / p.N, k = row - g * p.N;
-    const double U = hash_uniform(hash5(p.seed, kStreamToken, (uint64_t)g, (uint64_t)p.t, (uint64_t)k));
     const double target = U * Sb;
     int wsel = -1, wlast = -1;
     double run0 = 0.0, run_last = 0.0;
@@ -327,7 +630,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     }
     if (warp != wsel) return;  // (wsel >= 0: the row's largest logit is in S and has mass)
 
-    // ---- the warp that holds the target: the token ----
+    // the warp that holds the target: the token
     int y = -1, last_pos = -1;
     double run = run0;
     int tb = tie_base;
@@ -409,10 +712,11 @@ cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa
     p.status = la.status;
     const int mode = beta_mode(wa.beta);
     MaskedFn fn = la.dt == PSMC_F32 ? pick_masked<PSMC_F32>(mode) : pick_masked<PSMC_BF16>(mode);
-    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), (int)kHistBytes);
+    const size_t smem = (size_t)kCountBytes + (top_k == 0 ? kMassBytes : 0) + (size_t)kListCap * 8;
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kCountBytes + kMassBytes + kListCap * 8);
     if (e != cudaSuccess) return e;
-    const int threads = la.V >= 16384 ? 1024 : 256;
-    e = launch_chained(fn, dim3((unsigned)la.R), dim3((unsigned)threads), kHistBytes, stream, p);
+    const int threads = la.V < 16384 ? 256 : 512;
+    e = launch_chained(fn, dim3((unsigned)la.R), dim3((unsigned)threads), smem, stream, p);
     if (e != cudaSuccess) return e;
     const int warps = (wa.N + 31) >> 5;
     return launch_chained(rows_weights_kernel, dim3((unsigned)wa.G), dim3((unsigned)(warps * 32)), 0, stream, wa);

@@ -41,6 +41,20 @@ def test_masked_steps_model_vocabularies_bf16(name, G, T, rule):
     assert st.steps == T
 
 
+@pytest.mark.parametrize("name,rule,flat", [("llama2_7b", dict(top_k=20000), False), ("llama2_7b", dict(top_p=0.97), True),
+                                            ("qwen25_7b", dict(top_k=100000), False), ("qwen25_7b", dict(top_k=9000), True),
+                                            ("qwen25_7b", dict(top_k=100), True), ("tiny", dict(top_p=0.9), True)])
+def test_supports_too_large_for_the_candidate_list(name, rule, flat):
+    """More candidates at the cut than the kernel's shared-memory list holds (4096): it sweeps the row for every
+    remaining step instead (a large top_k; a flat row, which makes every nucleus large and puts crowds of equal
+    logits at a small top_k's threshold)."""
+    def flatten(t, lg):
+        lg.copy_((lg.float() * 0.02).to(lg.dtype))
+
+    st = P.closed_loop(W.CONFIGS[name], 6, 8, logit_bias_fn=flatten if flat else None, **rule)
+    assert st.steps == 8
+
+
 @pytest.mark.parametrize("rule", [dict(top_k=37), dict(top_k=300), dict(top_p=0.6)])
 @pytest.mark.parametrize("name", ["tiny", "llama2_7b"])
 def test_ties_at_the_cut_are_taken_in_id_order(name, rule):
