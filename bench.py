@@ -157,6 +157,8 @@ def run_ours(args):
     R, N = wl.R, cfg.N
     ps = B.Psmc(N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, cfg.ramp, seed, cfg.eos_id, G=G, T_max=T_total,
                 prompt_len=wl.prompt_len)
+    if args.top_k or args.top_p:  # supplementary run: proposal restricted to the top of each row
+        ps.set_proposal_mask(args.top_k, args.top_p)
     skip = wl.prompt_len if args.skip_shared_prompt else None
     PAGE = 16  # positions per block in the supplementary paged run
     if args.paged_kv:  # same capacity as the dense cache, cut into blocks reached through a table
@@ -268,10 +270,12 @@ def run_ours(args):
 
     dominant = int(np.argmax(kms))
     kv_name = "paged_release_acquire_copy_kernels" if args.paged_kv else "reindex_bulk_kernel"
-    names = ["logits_stream_kernel", "finish_weights_resample_kernel", kv_name]
+    # with a restricted proposal the logit pass and the group update are two other kernels, bracketed together
+    k1_name = "masked_rows_kernel+rows_weights_kernel" if (args.top_k or args.top_p) else "logits_stream_kernel"
+    names = [k1_name, "finish_weights_resample_kernel", kv_name]
     roofs = {
-        "logits_stream_kernel": {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
-                               "frac": k1_gbs / hbm_peak, "traffic": traffic("logits_stream_kernel", k1_bytes, kn[0]),
+        k1_name: {"bound": "hbm", "achieved": k1_gbs, "peak": hbm_peak, "unit": "GB/s",
+                               "frac": k1_gbs / hbm_peak, "traffic": traffic(k1_name, k1_bytes, kn[0]),
                                "peak_kind": peak_kind,
                                "avg_launch_us": 1e3 * kms[0] / max(kn[0], 1), "time_share": shares[0],
                                "bytes_per_launch": k1_bytes / max(kn[0], 1)},
@@ -330,6 +334,8 @@ def run_ours(args):
                        N_BLOCKS, R * cfg.logit_bytes_per_row / 1e6, G * per_group / 1e9),
                    "kv_reindex": ("paged cache, blocks of %d positions, copy on write" % PAGE) if args.paged_kv else
                                  ("prompt positions left in place" if args.skip_shared_prompt else "whole live prefix copied"),
+                   "proposal": ("top-k %d" % args.top_k) if args.top_k else ("nucleus %.3g" % args.top_p) if args.top_p
+                               else "softmax(beta l) over the whole vocabulary (Corollary 1)",
                    "parallelism": "replicas only (prompts sharded, no collective)"},
         "clocks": clk.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": R * cfg.logit_bytes_per_row,
@@ -464,6 +470,8 @@ def main():
     ap.add_argument("--skip-shared-prompt", action="store_true",
                     help="supplementary run: the KV reindex leaves each group's prompt positions in place (not the "
                          "headline configuration, which copies whole live prefixes)")
+    ap.add_argument("--top-k", type=int, default=0, help="supplementary run: proposal restricted to the top-k tokens")
+    ap.add_argument("--top-p", type=float, default=0.0, help="supplementary run: proposal restricted to a nucleus")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
