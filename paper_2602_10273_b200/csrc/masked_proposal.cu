@@ -91,27 +91,43 @@ __device__ __forceinline__ uint32_t load_bits(const void* rowp, int i) {
     return __ldg(reinterpret_cast<const unsigned short*>(rowp) + i);
 }
 
-// f(bits, id) for every logit of the row, in no particular order: 16-byte loads between the first and the last
-// 16-byte boundary (four in flight per thread), single loads for the ragged ends.  flush() runs after every group of
-// up to eight logits handed to f (so that f can sum in fp32 and flush can fold the partial sum into a double).
-template <int DT, class F, class G>
-__device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f, G flush) {
+// Two bf16 logits in one word -> their two keys in one word (the -0 adjustment of key_of left out: such a key is one
+// too low, which the callers allow for).
+__device__ __forceinline__ uint32_t keys_of_pair(uint32_t w) {
+    return w ^ ((((w >> 15) & 0x00010001u) * 0xffffu) | 0x80008000u);
+}
+
+// The row in no particular order: fv(v, id of its first logit) for every aligned 16 bytes between the first and the
+// last 16-byte boundary (four loads in flight per thread), fs(bits, id) for the logits of the ragged ends.
+template <int DT, class FV, class FS>
+__device__ __forceinline__ void for_each_vector(const void* rowp, int V, FV fv, FS fs) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4, kEs = DT == PSMC_BF16 ? 2 : 4;
     int head = (int)(((16 - (reinterpret_cast<uintptr_t>(rowp) & 15)) & 15) / kEs);
     if (head > V) head = V;
     const int nvec = (V - head) / kPer, tail0 = head + nvec * kPer;
     const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)head * kEs);
-    for (int j0 = threadIdx.x; j0 < nvec; j0 += 4 * blockDim.x) {
+    const int stride = (int)blockDim.x;
+    int j0 = (int)threadIdx.x;
+    for (; j0 + 3 * stride < nvec; j0 += 4 * stride) {  // full rounds: no bounds checks between the loads
         uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (j0 + u * (int)blockDim.x < nvec) v[u] = __ldg(&q[j0 + u * blockDim.x]);
+        for (int u = 0; u < 4; ++u) v[u] = __ldg(&q[j0 + u * stride]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * (int)blockDim.x;
-            if (j >= nvec) break;
-            const int i0 = head + j * kPer;
-            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        for (int u = 0; u < 4; ++u) fv(v[u], head + (j0 + u * stride) * kPer);
+    }
+    for (; j0 < nvec; j0 += stride) fv(__ldg(&q[j0]), head + j0 * kPer);
+    for (int i = threadIdx.x; i < head; i += blockDim.x) fs(load_bits<DT>(rowp, i), i);
+    for (int i = tail0 + threadIdx.x; i < V; i += blockDim.x) fs(load_bits<DT>(rowp, i), i);
+}
+
+// f(bits, id) for every logit of the row, in no particular order.  flush() runs after every group of up to eight
+// logits handed to f (so that f can sum in fp32 and flush can fold the partial sum into a double).
+template <int DT, class F, class G>
+__device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f, G flush) {
+    for_each_vector<DT>(
+        rowp, V,
+        [&](const uint4& v, int i0) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 if (DT == PSMC_BF16) {
@@ -122,10 +138,8 @@ __device__ __forceinline__ void for_each_logit(const void* rowp, int V, F f, G f
                 }
             }
             flush();
-        }
-    }
-    for (int i = threadIdx.x; i < head; i += blockDim.x) f(load_bits<DT>(rowp, i), i);
-    for (int i = tail0 + threadIdx.x; i < V; i += blockDim.x) f(load_bits<DT>(rowp, i), i);
+        },
+        f);
     flush();
 }
 template <int DT, class F>
@@ -297,7 +311,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     __shared__ int redi[33];
     __shared__ uint32_t tot_cnt[kDigits];
     __shared__ unsigned long long tot_mass[kDigits];
-    __shared__ Selection sel;
+    __shared__ Selection sel, thr;
     __shared__ double wmass[32];
     __shared__ int wties[32];
     __shared__ int n_list_sh, first_hit, last_mass;
@@ -321,20 +335,43 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         first_hit = 0x7fffffff;
         last_mass = -1;
     }
-    clear_columns(cnt, mass, nucleus);
+    const bool by_threshold = !nucleus && 2 * p.top_k <= (int)blockDim.x;
+    if (by_threshold) __syncthreads();
+    else clear_columns(cnt, mass, nucleus);
 
     // ---- sweep 1: the row's largest logit; NaN and +inf make the row unusable; top-k by counting: first-level counts ----
-    const bool by_threshold = !nucleus && 2 * p.top_k <= (int)blockDim.x;
     constexpr int kShift0 = kKeyBits - 8;
     // (on keys: a NaN or +inf ranks at or above +inf's key, or below -inf's)
     constexpr uint32_t kPosInf = DT == PSMC_BF16 ? 0xff80u : 0xff800000u, kNegInf = DT == PSMC_BF16 ? 0x007fu : 0x007fffffu;
     uint32_t kmax = 0u, kmin = 0xffffffffu;
-    for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
-        const uint32_t key = key_of<DT>(b);
-        kmax = max(kmax, key);
-        kmin = min(kmin, key);
-        if (!nucleus && !by_threshold) atomicAdd(&cnt[(key >> kShift0) * 32 + lane], 1u);
-    });
+    if (DT == PSMC_BF16 && by_threshold) {  // nothing to count: two keys at a time, packed maxima and minima
+        uint32_t mx2 = 0u, mn2 = 0xffffffffu;
+        for_each_vector<DT>(
+            rowp, V,
+            [&](const uint4& v, int) {
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t k2 = keys_of_pair(w[c]);
+                    mx2 = __vmaxu2(mx2, k2);
+                    mn2 = __vminu2(mn2, k2);
+                }
+            },
+            [&](uint32_t b, int) {
+                const uint32_t key = keys_of_pair(b) & 0xffffu;
+                kmax = max(kmax, key);
+                kmin = min(kmin, key);
+            });
+        kmax = max(kmax, max(mx2 & 0xffffu, mx2 >> 16));
+        kmin = min(kmin, min(mn2 & 0xffffu, mn2 >> 16));
+    } else {
+        for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
+            const uint32_t key = key_of<DT>(b);
+            kmax = max(kmax, key);
+            kmin = min(kmin, key);
+            if (!nucleus && !by_threshold) atomicAdd(&cnt[(key >> kShift0) * 32 + lane], 1u);
+        });
+    }
     const uint32_t my_max = kmax;
     kmax = __reduce_max_sync(kFull, kmax);
     kmin = __reduce_min_sync(kFull, kmin);
@@ -371,25 +408,63 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     };
 
     if (by_threshold) {
-        // ---- the threshold: the k-th largest of the threads' maxima ----
-        const int n_thr = (int)blockDim.x;  // a power of two
-        list[threadIdx.x] = my_max;
-        __syncthreads();
-        sort_words(list, n_thr);
-        const uint32_t theta = (uint32_t)list[n_thr - min(p.top_k, V)];
-        __syncthreads();  // the list's memory is handed over to the candidates
+        // ---- the threshold: the k-th largest of the threads' maxima, by the same digit search on a plain histogram ----
+        if (threadIdx.x == 0) {
+            thr.prefix = 0;
+            thr.k_rem = (uint32_t)min(p.top_k, V);
+            thr.m_rem = 0;
+            thr.above = 0;
+        }
+        for (int level = 0; level < kLevels; ++level) {
+            const int shift = kKeyBits - 8 * (level + 1);
+            if (threadIdx.x < kDigits) tot_cnt[threadIdx.x] = 0;
+            __syncthreads();
+            if (level == 0 || (my_max >> (shift + 8)) == thr.prefix) atomicAdd(&tot_cnt[(my_max >> shift) & 255u], 1u);
+            __syncthreads();
+            if (warp == 0) pick_digit(thr, tot_cnt, tot_mass, false, false, level == kLevels - 1, 0.0, lane);
+            __syncthreads();
+        }
+        const uint32_t theta = thr.prefix;
         // ---- sweep 2: the normaliser of p, and every logit at or above the threshold into the list ----
-        float part = 0.f;
-        for_each_logit<DT>(
-            rowp, V,
-            [&](uint32_t b, int i) {
-                part += ex2(rel_exponent(value_of<DT>(b), neg_C));
-                if (key_of<DT>(b) >= theta) append(b, i);
-            },
-            [&] {
-                s1 += (double)part;
-                part = 0.f;
-            });
+        if (DT == PSMC_BF16) {
+            // packed keys lack the -0 adjustment (one too low for -0), and so may the threshold: compare against one
+            // below +0's key when the threshold is +0's, so that either zero passes
+            constexpr uint32_t kZero = 0x8000u;
+            const uint32_t th = theta == kZero ? kZero - 1u : theta, th2 = th | (th << 16);
+            for_each_vector<DT>(
+                rowp, V,
+                [&](const uint4& v, int i0) {
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                    float part = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        part += ex2(rel_exponent(__uint_as_float(w[c] << 16), neg_C)) +
+                                ex2(rel_exponent(__uint_as_float(w[c] & 0xffff0000u), neg_C));
+                        const uint32_t ge = __vcmpgeu2(keys_of_pair(w[c]), th2);
+                        if (ge) {
+                            if (ge & 0xffffu) append(w[c] & 0xffffu, i0 + 2 * c);
+                            if (ge >> 16) append(w[c] >> 16, i0 + 2 * c + 1);
+                        }
+                    }
+                    s1 += (double)part;
+                },
+                [&](uint32_t b, int i) {
+                    s1 += (double)ex2(rel_exponent(value_of<DT>(b), neg_C));
+                    if ((keys_of_pair(b) & 0xffffu) >= th) append(b, i);
+                });
+        } else {
+            float part = 0.f;
+            for_each_logit<DT>(
+                rowp, V,
+                [&](uint32_t b, int i) {
+                    part += ex2(rel_exponent(value_of<DT>(b), neg_C));
+                    if (key_of<DT>(b) >= theta) append(b, i);
+                },
+                [&] {
+                    s1 += (double)part;
+                    part = 0.f;
+                });
+        }
         __syncthreads();
         if (n_list_sh <= kListCap) {
             have_list = true;
@@ -398,6 +473,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
             __syncthreads();
             if (threadIdx.x == 0) n_list_sh = 0;
             s1 = 0.0;
+            clear_columns(cnt, mass, nucleus);
             for_each_logit<DT>(rowp, V, [&](uint32_t b, int) { atomicAdd(&cnt[(key_of<DT>(b) >> kShift0) * 32 + lane], 1u); });
         }
     }
@@ -459,10 +535,29 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         const int n_cands = min(n_list_sh, kListCap);
 
         // ---- the levels not yet decided, over the candidates in whatever order they arrived ----
+        const bool short_list = n_cands <= 2 * (int)blockDim.x;  // few entries: no columns, one counter per digit
         for (int level = first_list_level; level < kLevels; ++level) {
-            clear_columns(cnt, mass, nucleus);
-            count_list_level<DT, MODE>(list, n_cands, level, prefix, nucleus, neg_C, p.bf, cnt, mass, lane);
-            fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+            if (short_list) {
+                if (threadIdx.x < kDigits) {
+                    tot_cnt[threadIdx.x] = 0;
+                    tot_mass[threadIdx.x] = 0;
+                }
+                __syncthreads();
+                const int shift = kKeyBits - 8 * (level + 1);
+                for (int j = threadIdx.x; j < n_cands; j += blockDim.x) {
+                    const uint32_t b = (uint32_t)list[j], key = key_of<DT>(b);
+                    if (level > 0 && (key >> (shift + 8)) != prefix) continue;
+                    const uint32_t d = (key >> shift) & 255u;
+                    atomicAdd(&tot_cnt[d], 1u);
+                    if (nucleus)
+                        atomicAdd(&tot_mass[d], __float2ull_rn(logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf) * kFixOne));
+                }
+                __syncthreads();
+            } else {
+                clear_columns(cnt, mass, nucleus);
+                count_list_level<DT, MODE>(list, n_cands, level, prefix, nucleus, neg_C, p.bf, cnt, mass, lane);
+                fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
+            }
             if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, level == 0, level == kLevels - 1, p.top_p, lane);
             __syncthreads();
             prefix = sel.prefix;
