@@ -12,6 +12,10 @@
 // more).  One sweep finds the maxima, a second collects the logits at or above the threshold into a candidate list in
 // shared memory (and sums the normaliser of p), and the search for (T, need) runs on that list.
 //
+// A nucleus of share top_p <= 0.9999 goes by a floor on the mass: tokens lighter than (1 - top_p) / V of the row's mass
+// cannot belong to it (all of them together weigh less than 1 - top_p).  Three sweeps: the largest logit; the row's
+// masses under p and under the proposal; the tokens above the floor into the list.
+//
 // Otherwise (T, need) come from a radix search over the key, 8 bits a level from the top (2 levels for bf16, 4 for
 // fp32): a level counts, per digit, the tokens whose higher digits equal the prefix found so far -- and for the
 // nucleus their mass 2^{beta (x - C)} as a 64-bit fixed-point number (2^-40 units, integer adds: the totals do not
@@ -336,7 +340,11 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         last_mass = -1;
     }
     const bool by_threshold = !nucleus && 2 * p.top_k <= (int)blockDim.x;
-    if (by_threshold) __syncthreads();
+    // A nucleus of share top_p < 1 holds no token of mass below (1 - top_p) / V of the row's: all such tokens together
+    // stay under 1 - top_p, so the tokens above the floor already reach top_p.  The floor turns into a threshold on the
+    // logit once the row's mass is known, and the search runs on the (usually short) list of tokens above it.
+    const bool by_floor = nucleus && p.top_p <= 0.9999;  // (closer to 1 the slack of the argument drowns in rounding)
+    if (by_threshold || by_floor) __syncthreads();
     else clear_columns(cnt, mass, nucleus);
 
     // ---- sweep 1: the row's largest logit; NaN and +inf make the row unusable; top-k by counting: first-level counts ----
@@ -344,7 +352,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     // (on keys: a NaN or +inf ranks at or above +inf's key, or below -inf's)
     constexpr uint32_t kPosInf = DT == PSMC_BF16 ? 0xff80u : 0xff800000u, kNegInf = DT == PSMC_BF16 ? 0x007fu : 0x007fffffu;
     uint32_t kmax = 0u, kmin = 0xffffffffu;
-    if (DT == PSMC_BF16 && by_threshold) {  // nothing to count: two keys at a time, packed maxima and minima
+    if (DT == PSMC_BF16 && (by_threshold || by_floor)) {  // nothing to count: two keys at a time, packed maxima and minima
         uint32_t mx2 = 0u, mn2 = 0xffffffffu;
         for_each_vector<DT>(
             rowp, V,
@@ -478,6 +486,74 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         }
     }
 
+    bool m_rem_preset = false;
+    if (by_floor) {
+        // ---- sweep 2: the masses of p and of the proposal over the whole row ----
+        double sb = 0.0;
+        float part1 = 0.f, partb = 0.f;
+        for_each_logit<DT>(
+            rowp, V,
+            [&](uint32_t b, int) {
+                const float d = rel_exponent(value_of<DT>(b), neg_C);
+                part1 += ex2(d);
+                partb += mass_beta<MODE>(d, p.bf);
+            },
+            [&] {
+                s1 += (double)part1;
+                sb += (double)partb;
+                part1 = 0.f;
+                partb = 0.f;
+            });
+        const double Sb_row = block_sum(sb, red, nw);
+        // floor on the mass, halved to stay on the safe side of rounding: 2^{beta (x - C)} >= (1 - top_p) Sb / (2 V)
+        const double x_floor = (double)C + log2((1.0 - p.top_p) * Sb_row / (2.0 * (double)V)) / p.beta;
+        float l_floor = (float)(x_floor * kLn2);
+        l_floor = nextafterf(l_floor, -INFINITY);
+        // a key at or below every key whose logit is >= l_floor (for bf16: the fp32 key's leading 16 bits)
+        const uint32_t key32 = key_of<PSMC_F32>(__float_as_uint(l_floor));
+        const uint32_t floor_key = (l_floor != l_floor || l_floor == -INFINITY) ? 0u
+                                   : (DT == PSMC_BF16 ? key32 >> 16 : key32);
+        // ---- sweep 3: the tokens at or above the floor into the list ----
+        if (DT == PSMC_BF16) {
+            const uint32_t th = floor_key > 0u ? floor_key - 1u : 0u, th2 = th | (th << 16);  // packed keys may be one low
+            for_each_vector<DT>(
+                rowp, V,
+                [&](const uint4& v, int i0) {
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t ge = __vcmpgeu2(keys_of_pair(w[c]), th2);
+                        if (ge) {
+                            if (ge & 0xffffu) append(w[c] & 0xffffu, i0 + 2 * c);
+                            if (ge >> 16) append(w[c] >> 16, i0 + 2 * c + 1);
+                        }
+                    }
+                },
+                [&](uint32_t b, int i) {
+                    if ((keys_of_pair(b) & 0xffffu) >= th) append(b, i);
+                });
+        } else {
+            for_each_logit<DT>(rowp, V, [&](uint32_t b, int i) {
+                if (key_of<DT>(b) >= floor_key) append(b, i);
+            });
+        }
+        __syncthreads();
+        if (n_list_sh <= kListCap) {
+            have_list = true;
+            first_list_level = 0;
+            m_rem_preset = true;  // the share is of the whole row's mass, not of the list's
+            if (threadIdx.x == 0) {
+                const double want = ceil(p.top_p * Sb_row * (double)kFixOne);
+                sel.m_rem = want < 1.0 ? 1ull : (unsigned long long)want;
+            }
+        } else {  // a flat row: count digits and masses over the row after all
+            __syncthreads();
+            if (threadIdx.x == 0) n_list_sh = 0;
+            s1 = 0.0;
+            clear_columns(cnt, mass, nucleus);
+        }
+    }
+
     bool listed = have_list;
     if (!have_list) {
         // ---- sweep 2 (nucleus): first-level counts and masses, which need the reference exponent ----
@@ -558,7 +634,8 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
                 count_list_level<DT, MODE>(list, n_cands, level, prefix, nucleus, neg_C, p.bf, cnt, mass, lane);
                 fold_columns(cnt, mass, nucleus, tot_cnt, tot_mass);
             }
-            if (warp == 0) pick_digit(sel, tot_cnt, tot_mass, nucleus, level == 0, level == kLevels - 1, p.top_p, lane);
+            if (warp == 0)
+                pick_digit(sel, tot_cnt, tot_mass, nucleus, level == 0 && !m_rem_preset, level == kLevels - 1, p.top_p, lane);
             __syncthreads();
             prefix = sel.prefix;
         }
@@ -665,35 +742,86 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     const bool all_ties = need == sel.n_ties;
     const int set_size = (int)(sel.above + need);
 
-    // ordered sweeps: warp w owns logits [lo, hi)
-    const int seg = (((V + nw - 1) / nw) + 31) & ~31;
+    // Ordered sweeps: warp w owns logits [lo, hi); in a round its lanes take kPer consecutive logits each (one 16-byte
+    // load where the row allows), so a round covers 32 * kPer logits in id order: lane 0's first.
+    constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
+    const bool aligned = (reinterpret_cast<uintptr_t>(rowp) & 15) == 0;
+    const int seg = (((V + nw - 1) / nw) + 32 * kPer - 1) / (32 * kPer) * (32 * kPer);
     const int lo = min(V, warp * seg), hi = min(V, lo + seg);
+    auto load_chunk = [&](int e0, uint32_t (&bits)[kPer]) -> int {  // -> how many of the kPer logits from e0 exist
+        if (e0 >= hi) return 0;
+        if (aligned && e0 + kPer <= hi) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) +
+                                                                 (size_t)e0 * (DT == PSMC_BF16 ? 2 : 4)));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (DT == PSMC_BF16) {
+                    bits[2 * c] = w[c] & 0xffffu;
+                    bits[2 * c + 1] = w[c] >> 16;
+                } else {
+                    bits[c] = w[c];
+                }
+            }
+            return kPer;
+        }
+        const int nv = min(kPer, hi - e0);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) bits[j] = j < nv ? load_bits<DT>(rowp, e0 + j) : 0u;
+        return nv;
+    };
     int tie_base = 0;
     if (!all_ties) {  // ties at T are taken in id order: how many lie before this warp's stretch
         int n = 0;
-        for (int base = lo; base < hi; base += 32) {
-            const int i = base + lane;
-            const bool tie = i < hi && key_of<DT>(load_bits<DT>(rowp, i)) == T;
-            n += __popc(__ballot_sync(kFull, tie));
+        for (int base = lo; base < hi; base += 32 * kPer) {
+            uint32_t bits[kPer];
+            const int nv = load_chunk(base + lane * kPer, bits);
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) n += (j < nv && key_of<DT>(bits[j]) == T) ? 1 : 0;
         }
-        if (lane == 0) wties[warp] = n;
+        n = warp_scan_incl(n, lane);
+        if (lane == 31) wties[warp] = n;
         __syncthreads();
         for (int w = 0; w < warp; ++w) tie_base += wties[w];
     }
-    auto in_set = [&](uint32_t key, bool tie, int rank) { return key > T || (tie && (all_ties || (uint32_t)rank < need)); };
+    // masses of this lane's logits that are in S; `rank` = ties at T before them in the row
+    auto chunk_masses = [&](const uint32_t (&bits)[kPer], int nv, int rank, double (&m)[kPer]) -> double {
+        double sum = 0.0;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            m[j] = 0.0;
+            if (j < nv) {
+                const uint32_t key = key_of<DT>(bits[j]);
+                bool in = key > T;
+                if (key == T) {
+                    in = all_ties || (uint32_t)rank < need;
+                    ++rank;
+                }
+                if (in) m[j] = (double)logit_mass<MODE>(value_of<DT>(bits[j]), neg_C, p.bf);
+                sum += m[j];
+            }
+        }
+        return sum;
+    };
+    auto ties_before_lane = [&](const uint32_t (&bits)[kPer], int nv, int& tb) -> int {  // and advances tb by the round's ties
+        if (all_ties) return 0;
+        int c = 0;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) c += (j < nv && key_of<DT>(bits[j]) == T) ? 1 : 0;
+        const int incl = warp_scan_incl(c, lane);
+        const int rank = tb + incl - c;
+        tb += __shfl_sync(kFull, incl, 31);
+        return rank;
+    };
     {
         double acc = 0.0;
         int tb = tie_base;
-        for (int base = lo; base < hi; base += 32) {
-            const int i = base + lane;
-            const bool valid = i < hi;
-            const uint32_t b = valid ? load_bits<DT>(rowp, i) : 0u;
-            const uint32_t key = key_of<DT>(b);
-            const bool tie = valid && key == T;
-            const unsigned bal = __ballot_sync(kFull, tie);
-            const int rank = tb + __popc(bal & ((1u << lane) - 1u));
-            tb += __popc(bal);
-            if (valid && in_set(key, tie, rank)) acc += (double)logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf);
+        for (int base = lo; base < hi; base += 32 * kPer) {
+            uint32_t bits[kPer];
+            double m[kPer];
+            const int nv = load_chunk(base + lane * kPer, bits);
+            const int rank = ties_before_lane(bits, nv, tb);
+            acc += chunk_masses(bits, nv, rank, m);
         }
         acc = warp_sum(acc);
         if (lane == 0) wmass[warp] = acc;
@@ -725,25 +853,40 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     }
     if (warp != wsel) return;  // (wsel >= 0: the row's largest logit is in S and has mass)
 
-    // the warp that holds the target: the token
+    // the warp that holds the target: the round, the lane, the token
     int y = -1, last_pos = -1;
     double run = run0;
     int tb = tie_base;
-    for (int base = lo; base < hi && y < 0; base += 32) {
-        const int i = base + lane;
-        const bool valid = i < hi;
-        const uint32_t b = valid ? load_bits<DT>(rowp, i) : 0u;
-        const uint32_t key = key_of<DT>(b);
-        const bool tie = valid && key == T;
-        const unsigned bal = __ballot_sync(kFull, tie);
-        const int rank = tb + __popc(bal & ((1u << lane) - 1u));
-        tb += __popc(bal);
-        const double e = (valid && in_set(key, tie, rank)) ? (double)logit_mass<MODE>(value_of<DT>(b), neg_C, p.bf) : 0.0;
+    for (int base = lo; base < hi && y < 0; base += 32 * kPer) {
+        uint32_t bits[kPer];
+        double m[kPer];
+        const int e0 = base + lane * kPer;
+        const int nv = load_chunk(e0, bits);
+        const int rank = ties_before_lane(bits, nv, tb);
+        const double e = chunk_masses(bits, nv, rank, m);
         const double incl = run + warp_scan_incl(e, lane);
         const unsigned hit = __ballot_sync(kFull, e > 0.0 && incl >= target);
         const unsigned pos = __ballot_sync(kFull, e > 0.0);
-        if (hit) y = base + __ffs(hit) - 1;
-        else if (pos) last_pos = base + 31 - __clz(pos);
+        const int src = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : -1);
+        if (src >= 0) {  // lane src: its first logit that reaches the target, else its last one with mass
+            int mine = -1;
+            if (lane == src) {
+                double r = incl - e;
+                int last = -1;
+#pragma unroll
+                for (int j = 0; j < kPer; ++j) {
+                    if (m[j] > 0.0) {
+                        r += m[j];
+                        last = e0 + j;
+                        if (mine < 0 && hit && r >= target) mine = last;
+                    }
+                }
+                if (mine < 0) mine = last;
+            }
+            mine = __shfl_sync(kFull, mine, src);
+            if (hit) y = mine;
+            else last_pos = mine;
+        }
         run = __shfl_sync(kFull, incl, 31);
     }
     if (y < 0) y = last_pos;  // the finer sums fell a rounding error short of the warp's total
