@@ -7,9 +7,10 @@
 // One CTA per row.  A logit's bit pattern maps to an unsigned key that orders like the value, so S is
 // {key > T} plus the first `need` tokens with key == T in id order.
 //
-// A top_k of up to half the CTA's threads goes by a threshold: every thread sees its own share of the row, so the
-// k-th largest of the threads' maxima has at least k logits at or above it (and, the shares being interleaved, hardly
-// more).  One sweep finds the maxima, a second collects the logits at or above the threshold into a candidate list in
+// A top_k of up to half the number of shares goes by a threshold: every thread sees its own share of the row, cut
+// once more into 8 (bf16) or 4 (fp32) sub-shares by position inside the 16-byte vectors -- 4096 or 2048 shares for 512
+// threads -- so the k-th largest of the shares' maxima has at least k logits at or above it (and, the shares being
+// interleaved, not many more).  One sweep finds the maxima, a second collects the logits at or above the threshold into a candidate list in
 // shared memory (and sums the normaliser of p), and the search for (T, need) runs on that list.
 //
 // A nucleus of share top_p <= 0.9999 goes by a floor on the mass: tokens lighter than (1 - top_p) / V of the row's mass
@@ -339,7 +340,9 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         first_hit = 0x7fffffff;
         last_mass = -1;
     }
-    const bool by_threshold = !nucleus && 2 * p.top_k <= (int)blockDim.x;
+    // (a thread's share is itself cut into kSub interleaved sub-shares, by position inside the 16-byte vectors)
+    constexpr int kSub = DT == PSMC_BF16 ? 8 : 4;
+    const bool by_threshold = !nucleus && 2 * p.top_k <= kSub * (int)blockDim.x;
     // A nucleus of share top_p < 1 holds no token of mass below (1 - top_p) / V of the row's: all such tokens together
     // stay under 1 - top_p, so the tokens above the floor already reach top_p.  The floor turns into a threshold on the
     // logit once the row's mass is known, and the search runs on the (usually short) list of tokens above it.
@@ -352,8 +355,11 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     // (on keys: a NaN or +inf ranks at or above +inf's key, or below -inf's)
     constexpr uint32_t kPosInf = DT == PSMC_BF16 ? 0xff80u : 0xff800000u, kNegInf = DT == PSMC_BF16 ? 0x007fu : 0x007fffffu;
     uint32_t kmax = 0u, kmin = 0xffffffffu;
+    uint32_t sub[kSub];  // largest key of each sub-share (threshold path)
+#pragma unroll
+    for (int j = 0; j < kSub; ++j) sub[j] = 0u;
     if (DT == PSMC_BF16 && (by_threshold || by_floor)) {  // nothing to count: two keys at a time, packed maxima and minima
-        uint32_t mx2 = 0u, mn2 = 0xffffffffu;
+        uint32_t mx2[4] = {0u, 0u, 0u, 0u}, mn2 = 0xffffffffu;
         for_each_vector<DT>(
             rowp, V,
             [&](const uint4& v, int) {
@@ -361,7 +367,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const uint32_t k2 = keys_of_pair(w[c]);
-                    mx2 = __vmaxu2(mx2, k2);
+                    mx2[c] = __vmaxu2(mx2[c], k2);
                     mn2 = __vminu2(mn2, k2);
                 }
             },
@@ -370,17 +376,47 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
                 kmax = max(kmax, key);
                 kmin = min(kmin, key);
             });
-        kmax = max(kmax, max(mx2 & 0xffffu, mx2 >> 16));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            sub[(2 * c) % kSub] = mx2[c] & 0xffffu;
+            sub[(2 * c + 1) % kSub] = mx2[c] >> 16;
+        }
+        sub[0] = max(sub[0], kmax);  // the ragged ends join the first sub-share
         kmin = min(kmin, min(mn2 & 0xffffu, mn2 >> 16));
+    } else if (by_threshold) {
+        for_each_vector<DT>(
+            rowp, V,
+            [&](const uint4& v, int) {
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (DT == PSMC_BF16) {
+                        const uint32_t a = key_of<DT>(w[c] & 0xffffu), b = key_of<DT>(w[c] >> 16);
+                        sub[(2 * c) % kSub] = max(sub[(2 * c) % kSub], a);
+                        sub[(2 * c + 1) % kSub] = max(sub[(2 * c + 1) % kSub], b);
+                        kmin = min(kmin, min(a, b));
+                    } else {
+                        const uint32_t a = key_of<DT>(w[c]);
+                        sub[c % kSub] = max(sub[c % kSub], a);
+                        kmin = min(kmin, a);
+                    }
+                }
+            },
+            [&](uint32_t b, int) {
+                const uint32_t key = key_of<DT>(b);
+                sub[0] = max(sub[0], key);
+                kmin = min(kmin, key);
+            });
     } else {
         for_each_logit<DT>(rowp, V, [&](uint32_t b, int) {
             const uint32_t key = key_of<DT>(b);
             kmax = max(kmax, key);
             kmin = min(kmin, key);
-            if (!nucleus && !by_threshold) atomicAdd(&cnt[(key >> kShift0) * 32 + lane], 1u);
+            if (!nucleus) atomicAdd(&cnt[(key >> kShift0) * 32 + lane], 1u);
         });
     }
-    const uint32_t my_max = kmax;
+#pragma unroll
+    for (int j = 0; j < kSub; ++j) kmax = max(kmax, sub[j]);
     kmax = __reduce_max_sync(kFull, kmax);
     kmin = __reduce_min_sync(kFull, kmin);
     if (lane == 0) {
@@ -427,7 +463,9 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
             const int shift = kKeyBits - 8 * (level + 1);
             if (threadIdx.x < kDigits) tot_cnt[threadIdx.x] = 0;
             __syncthreads();
-            if (level == 0 || (my_max >> (shift + 8)) == thr.prefix) atomicAdd(&tot_cnt[(my_max >> shift) & 255u], 1u);
+#pragma unroll
+            for (int j = 0; j < kSub; ++j)
+                if (level == 0 || (sub[j] >> (shift + 8)) == thr.prefix) atomicAdd(&tot_cnt[(sub[j] >> shift) & 255u], 1u);
             __syncthreads();
             if (warp == 0) pick_digit(thr, tot_cnt, tot_mass, false, false, level == kLevels - 1, 0.0, lane);
             __syncthreads();
