@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a bulk asynchronous copy engine (TMA, untiled form) and the shared-memory
-// mbarriers its loads complete on.  No multicast, no cluster-wide forms: every copy stays within one CTA.
+// mbarriers its loads complete on.  Every copy stays within one CTA (no cluster-wide forms).
 // Both addresses of a bulk copy must be 16-byte aligned and its size a multiple of 16 bytes.
 #pragma once
 

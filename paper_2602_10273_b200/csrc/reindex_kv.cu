@@ -8,7 +8,7 @@
 // Bulk path (sm_100a): one warp per CTA; lane 0 drives a ring of shared-memory stages with the
 // TMA engine: cp.async.bulk global->shared (completion on an mbarrier), then cp.async.bulk
 // shared->global per destination (bulk async-groups).  No thread touches the payload, so the copy
-// is bit-exact by construction and the SM's load/store units stay idle.  No multicast anywhere.
+// is bit-exact by construction and the SM's load/store units stay idle.
 // Every mbarrier wait is bounded; on expiry the kernel raises PSMC_E_TIMEOUT, drains its own
 // copies and returns.  Plain path: 256 threads copy with ordinary loads/stores of the widest unit
 // the alignment allows; used when the 16-byte rules of bulk copies do not hold.
