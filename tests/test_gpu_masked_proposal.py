@@ -41,6 +41,14 @@ def test_masked_steps_model_vocabularies_bf16(name, G, T, rule):
     assert st.steps == T
 
 
+@pytest.mark.parametrize("rule", [dict(top_k=50), dict(top_k=1000), dict(top_p=0.9)])
+def test_masked_steps_batched_prompts_full_size(rule):
+    """All 64 prompts x 8 particles x 128256 logits: the launch shape `bench.py --top-k / --top-p` times (one CTA per
+    row, two per SM), every row compared with the oracle."""
+    st = P.closed_loop(W.CONFIGS["batched_prompts"], 1, 3, **rule)
+    assert st.live_rows == 3 * 512
+
+
 @pytest.mark.parametrize("name,rule,flat", [("llama2_7b", dict(top_k=20000), False), ("llama2_7b", dict(top_p=0.97), True),
                                             ("qwen25_7b", dict(top_k=100000), False), ("qwen25_7b", dict(top_k=9000), True),
                                             ("qwen25_7b", dict(top_k=100), True), ("tiny", dict(top_p=0.9), True)])

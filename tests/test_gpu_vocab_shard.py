@@ -103,6 +103,14 @@ def test_sharded_step_model_vocabularies(name, world, T, G):
     assert st.steps == T and owners.sum() == st.live_rows
 
 
+def test_sharded_step_batched_prompts_full_size():
+    """All 64 prompts x 8 particles, the vocabulary of 128256 over 8 ranks: every row of rank 0 against the oracle's
+    whole-row step, every other rank bit-equal to rank 0."""
+    cfg = W.CONFIGS["batched_prompts"]
+    st, owners = sharded_loop(cfg, 1, 3, VS.vocab_shards(cfg.V, 8))
+    assert st.live_rows == 3 * 512 and (owners > 0).all()
+
+
 def test_sharded_step_three_ranks_need_more_span_triples_than_the_whole_row():
     """320 rows of 128256 logits are cut into 32 spans of 4096; a third of such a row is cut into 42 spans of 1024,
     so the context has to grow the scratch it sized for whole rows."""
