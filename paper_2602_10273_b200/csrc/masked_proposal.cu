@@ -340,6 +340,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         first_hit = 0x7fffffff;
         last_mass = -1;
     }
+    if (threadIdx.x < kDigits) tot_mass[threadIdx.x] = 0;  // read (and ignored) by the digit search when nothing weighs
     // (a thread's share is itself cut into kSub interleaved sub-shares, by position inside the 16-byte vectors)
     constexpr int kSub = DT == PSMC_BF16 ? 8 : 4;
     const bool by_threshold = !nucleus && 2 * p.top_k <= kSub * (int)blockDim.x;
