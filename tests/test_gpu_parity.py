@@ -533,3 +533,54 @@ def test_step_host_matches_device_step():
         prev.copy_(ps.device_view("psmc_last_tokens", ps.R))
     ps.destroy()
     ps2.destroy()
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other():
+    """Two runs with different seeds interleaved on two streams (each context owns its scratch, counters and move
+    lists): every state view equals that of the same run made alone, bit for bit."""
+    c = W.CONFIGS["llama2_7b"]
+    T, kv_shape = 12, (1, 2, c.prompt_hi + 20, c.head_dim)
+
+    def prepare(seed):
+        wl = WC.DeviceWorkload(c, seed)
+        ps = B.Psmc(c.N, c.V, c.alpha, c.tau, c.kappa, c.ramp, seed, c.eos_id, G=c.G, T_max=T, prompt_len=wl.prompt_len)
+        ks = [torch.empty((wl.R,) + kv_shape[1:], dtype=wl.tdtype, device="cuda") for _ in range(kv_shape[0])]
+        vs = [torch.empty_like(k) for k in ks]
+        for l, (k, v) in enumerate(zip(ks, vs)):
+            WC.fill_kv(k, seed, l, 0)
+            WC.fill_kv(v, seed, l, 1)
+        return dict(wl=wl, ps=ps, ks=ks, vs=vs, desc=ps.make_kv_desc(ks, vs), lg=wl.new_logits(),
+                    prev=wl.first_prev.clone(), last=ps.device_view("psmc_last_tokens", wl.R))
+
+    def advance(run, t, stream):
+        with torch.cuda.stream(stream):
+            run["wl"].fill(run["lg"], t, run["prev"])
+            run["ps"].step(run["lg"])
+            run["ps"].reindex_kv(run["desc"])
+            run["prev"].copy_(run["last"])
+
+    def snapshot(run):
+        torch.cuda.synchronize()
+        ps = run["ps"]
+        views = [getattr(ps, n).numpy().copy() for n in ("tokens", "last_tokens", "log_weights", "cum_logp", "slot_map",
+                                                         "ancestors", "ess", "log_z", "lens", "done")]
+        return views + [t.view(torch.int16).cpu().numpy().copy() for t in run["ks"] + run["vs"]]
+
+    alone = []
+    for seed in (21, 22):
+        run = prepare(seed)
+        for t in range(1, T + 1):
+            advance(run, t, torch.cuda.current_stream())
+        alone.append(snapshot(run))
+        run["ps"].destroy()
+    runs = [prepare(21), prepare(22)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for t in range(1, T + 1):
+        for run, s in zip(runs, streams):
+            advance(run, t, s)
+    for run, want in zip(runs, alone):
+        got = snapshot(run)
+        assert all(np.array_equal(a, b, equal_nan=True) for a, b in zip(got, want))
+        assert run["ps"].sync_status() == B.OK
+        run["ps"].destroy()
