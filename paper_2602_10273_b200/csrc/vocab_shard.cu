@@ -31,22 +31,28 @@ struct ShardTotals {
     double S1, Sb, target, base;
     int owner;
 };
-template <int MODE>
-__device__ __forceinline__ ShardTotals shard_combine(const double* all, int P, int R, int row, double beta, double U) {
+// get(p, C, s1, sb) hands out rank p's triple of the row (from registers, shared memory or global memory: the
+// arithmetic and its order are the same wherever the numbers are fetched from).
+template <int MODE, class Get>
+__device__ __forceinline__ ShardTotals shard_combine(Get get, int P, double beta, double U) {
     ShardTotals t;
     t.ok = false;
     t.owner = -1;
     t.base = 0.0;
     double C = (double)kRefFloor;
-    for (int p = 0; p < P; ++p) C = fmax(C, __ldcg(&all[((size_t)p * R + row) * 3]));
+    for (int p = 0; p < P; ++p) {
+        double c, s1, sb;
+        get(p, c, s1, sb);
+        C = fmax(C, c);
+    }
     t.C = (float)C;
     double S1 = 0.0, Sb = 0.0;
     for (int p = 0; p < P; ++p) {
-        const double* tr = all + ((size_t)p * R + row) * 3;
-        double f1, fb;
-        span_scales<MODE>((float)(__ldcg(&tr[0]) - C), beta, f1, fb);
-        S1 += __ldcg(&tr[1]) * f1;
-        Sb += __ldcg(&tr[2]) * fb;
+        double c, s1, sb, f1, fb;
+        get(p, c, s1, sb);
+        span_scales<MODE>((float)(c - C), beta, f1, fb);
+        S1 += s1 * f1;
+        Sb += sb * fb;
     }
     t.S1 = S1;
     t.Sb = Sb;
@@ -55,15 +61,14 @@ __device__ __forceinline__ ShardTotals shard_combine(const double* all, int P, i
     double incl = 0.0, last_base = 0.0;
     int last = -1;
     for (int p = 0; p < P; ++p) {
-        const double* tr = all + ((size_t)p * R + row) * 3;
-        double f1, fb;
-        span_scales<MODE>((float)(__ldcg(&tr[0]) - C), beta, f1, fb);
-        const double b = __ldcg(&tr[2]) * fb;
+        double c, s1, sb, f1, fb;
+        get(p, c, s1, sb);
+        span_scales<MODE>((float)(c - C), beta, f1, fb);
+        const double b = sb * fb;
         if (b > 0.0) {
-            if (incl + b >= t.target) {
+            if (t.owner < 0 && incl + b >= t.target) {
                 t.owner = p;
                 t.base = incl;
-                break;
             }
             last = p;
             last_base = incl;
@@ -77,6 +82,17 @@ __device__ __forceinline__ ShardTotals shard_combine(const double* all, int P, i
     t.ok = t.owner >= 0;
     return t;
 }
+// rank p's triple of `row` straight from the gathered array
+struct TriplesInGlobal {
+    const double* all;
+    int R, row;
+    __device__ __forceinline__ void operator()(int p, double& c, double& s1, double& sb) const {
+        const double* tr = all + ((size_t)p * R + row) * 3;
+        c = __ldcg(&tr[0]);
+        s1 = __ldcg(&tr[1]);
+        sb = __ldcg(&tr[2]);
+    }
+};
 
 // ---- sweep, second half: the span triples of the local columns become one triple per row ----
 template <int MODE>
@@ -131,7 +147,20 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) shard_locate_kernel(const __
     if (!lp.done[row]) {
         const int g = row / lp.N, k = row - g * lp.N;
         const double U = hash_uniform(hash5(lp.seed, kStreamToken, (uint64_t)g, (uint64_t)lp.t, (uint64_t)k));
-        const ShardTotals st = shard_combine<MODE>(lp.all, lp.P, lp.R, row, lp.f.beta, U);
+        ShardTotals st;
+        if (lp.P <= 32) {  // lane p fetches rank p's triple: one round trip instead of one per rank
+            double c = (double)kRefFloor, s1 = 0.0, sb = 0.0;
+            if (lane < lp.P) TriplesInGlobal{lp.all, lp.R, row}(lane, c, s1, sb);
+            st = shard_combine<MODE>(
+                [&](int p, double& c_, double& s1_, double& sb_) {
+                    c_ = __shfl_sync(kFull, c, p);
+                    s1_ = __shfl_sync(kFull, s1, p);
+                    sb_ = __shfl_sync(kFull, sb, p);
+                },
+                lp.P, lp.f.beta, U);
+        } else {
+            st = shard_combine<MODE>(TriplesInGlobal{lp.all, lp.R, row}, lp.P, lp.f.beta, U);
+        }
         if (st.ok && st.owner == lp.rank) {
             const RowFrame fr{st.C, st.target, st.base};
             const RowTotals t = combine_spans<MODE, true>(lp.f, row, U, lane, &fr);
@@ -155,13 +184,23 @@ struct ShardFinishParams {
     const double* all;
     const psmc_shard_pick* picks;  // [P][R]
     int P;
+    int staged;  // the group's triples fit the dynamic shared memory given to the launch
 };
 template <int MODE>
 __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_constant__ ShardFinishParams sp) {
     __shared__ GroupScratch<kMaxParticles> sc;
+    extern __shared__ double staged[];  // [N][P][3] when sp.staged: the group's triples, fetched by the whole CTA at once
     const WeightsArgs& a = sp.a;
     const int g = blockIdx.x, i = threadIdx.x, N = a.N;
     chain_begin();
+    if (sp.staged) {
+        const int per_rank = N * 3;
+        for (int j = threadIdx.x; j < sp.P * per_rank; j += blockDim.x) {
+            const int p = j / per_rank, rem = j - p * per_rank, k = rem / 3, q = rem - 3 * k;
+            staged[(k * sp.P + p) * 3 + q] = __ldcg(&sp.all[((size_t)p * a.R + (size_t)g * N + k) * 3 + q]);
+        }
+        __syncthreads();
+    }
     const bool on = i < N;
     ParticleState st{};
     int tk = -1;
@@ -171,7 +210,19 @@ __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_consta
         st = load_particle(a, r);
         if (!st.done) {
             const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)i));
-            const ShardTotals tot = shard_combine<MODE>(sp.all, sp.P, a.R, r, a.beta, U);
+            ShardTotals tot;
+            if (sp.staged) {
+                const double* mine = staged + (size_t)i * sp.P * 3;
+                tot = shard_combine<MODE>(
+                    [&](int p, double& c, double& s1, double& sb) {
+                        c = mine[3 * p];
+                        s1 = mine[3 * p + 1];
+                        sb = mine[3 * p + 2];
+                    },
+                    sp.P, a.beta, U);
+            } else {
+                tot = shard_combine<MODE>(TriplesInGlobal{sp.all, a.R, r}, sp.P, a.beta, U);
+            }
             if (tot.ok) {
                 const psmc_shard_pick pk = sp.picks[(size_t)tot.owner * a.R + r];
                 if (pk.tok >= 0) {
@@ -242,7 +293,9 @@ cudaError_t launch_shard_weights(const WeightsArgs& a, const double* all_triples
         default: fn = shard_weights_kernel<kBetaAny>; break;
     }
     const int warps = (a.N + 31) >> 5;
-    return launch_chained(fn, dim3((unsigned)a.G), dim3((unsigned)(warps * 32)), 0, stream, sp);
+    const size_t stage_bytes = (size_t)a.N * P * 3 * sizeof(double);
+    sp.staged = stage_bytes <= 4096 ? 1 : 0;  // (the static scratch of the group update takes most of the 48 KB)
+    return launch_chained(fn, dim3((unsigned)a.G), dim3((unsigned)(warps * 32)), sp.staged ? stage_bytes : 0, stream, sp);
 }
 
 }  // namespace psmc
