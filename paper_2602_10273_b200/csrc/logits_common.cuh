@@ -135,11 +135,14 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     const int n = p.n_spans;
     const float4* P = p.partials + (size_t)row * n;
 
+    // the lane's first triple is fetched once and kept (rows of up to 32 spans need no second trip to L2)
+    const float4 f0 = lane < n ? __ldcg(&P[lane]) : make_float4(kRefFloor, 0.f, 0.f, 0.f);
     float cf = kRefFloor;
     if (FRAMED) {
         cf = fr->C;
     } else {
-        for (int j = lane; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
+        cf = f0.x;
+        for (int j = lane + 32; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
         cf = warp_max(cf);
     }
     t.C = cf;
@@ -150,7 +153,7 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
 #pragma unroll
     for (int i = 0; i < kKeep; ++i) keep[i] = 0.0;
     for (int j = lane, i = 0; j < n; j += 32, ++i) {
-        const float4 f = __ldcg(&P[j]);
+        const float4 f = i == 0 ? f0 : __ldcg(&P[j]);
         double f1, fb;
         span_scales<MODE>(f.x - cf, p.beta, f1, fb);
         const double a = (double)f.y * f1;
