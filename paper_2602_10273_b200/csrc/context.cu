@@ -405,8 +405,13 @@ extern "C" psmc_status psmc_step_host(psmc_ctx* c, const void* logits_host, psmc
         if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return PSMC_E_CUDA;
         if (cudaEventCreateWithFlags(&c->staged, cudaEventDisableTiming) != cudaSuccess) return PSMC_E_CUDA;
     }
-    if (cudaMemcpy2DAsync(c->staging, ld_dev * esize, logits_host, ld * esize, (size_t)c->V * esize, c->R,
-                          cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess ||
+    // one flat copy when both sides are dense (the usual case), row by row otherwise
+    const cudaError_t copied =
+        (ld == c->V && ld_dev == c->V)
+            ? cudaMemcpyAsync(c->staging, logits_host, need, cudaMemcpyHostToDevice, c->copy_stream)
+            : cudaMemcpy2DAsync(c->staging, ld_dev * esize, logits_host, ld * esize, (size_t)c->V * esize, c->R,
+                                cudaMemcpyHostToDevice, c->copy_stream);
+    if (copied != cudaSuccess ||
         cudaEventRecord(c->staged, c->copy_stream) != cudaSuccess || cudaStreamWaitEvent(s, c->staged, 0) != cudaSuccess)
         return PSMC_E_CUDA;
     psmc_status st = psmc_step(c, c->staging, dt, ld_dev, stream);
