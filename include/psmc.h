@@ -238,7 +238,9 @@ psmc_status psmc_reindex_kv(psmc_ctx*, const psmc_kv_desc* src, const psmc_kv_de
 psmc_status psmc_kv_paged_create(psmc_ctx*, int n_blocks, int block_len, int max_blocks_per_row, int share_prompt);
 
 /* Before the language model writes position len[r] of every live row: rows whose next position starts a new block
- * get one from the free list.  Stream-ordered. */
+ * get one from the free list, unless they hold it already.  Stream-ordered.  Needed once, after
+ * psmc_kv_paged_create and the prefill: psmc_reindex_kv_paged does the same for the token that follows it (see
+ * there), and a call that finds every row provided for changes nothing. */
 psmc_status psmc_kv_paged_append(psmc_ctx*, void* stream);
 
 /* At most 64 layers per call; pools 16-byte aligned with head_dim*sizeof(elem) a multiple of 16. */
@@ -253,8 +255,10 @@ typedef struct {
 
 /* Applies the slot map of the most recent step: every rewritten slot gives its blocks back, takes a reference to
  * each full block of its ancestor and a private copy of the ancestor's partly filled last block (all layers, K and
- * V, all heads).  Groups that did not resample change nothing; without any resampling the kernels return after
- * reading one counter.  Stream-ordered, no host synchronisation. */
+ * V, all heads).  Groups that did not resample change nothing.  Unless the step was the last one the context can
+ * take (T_max), every live row is then given the block its next position needs, exactly as psmc_kv_paged_append
+ * would (same errors), so that a token costs three launches here and none for the append.  Stream-ordered, no host
+ * synchronisation. */
 psmc_status psmc_reindex_kv_paged(psmc_ctx*, const psmc_kv_pools* pools, void* stream);
 
 /* DEVICE views of the paging state (valid until psmc_destroy or the next psmc_kv_paged_create). */

@@ -531,8 +531,11 @@ extern "C" psmc_status psmc_reindex_kv_paged(psmc_ctx* c, const psmc_kv_pools* p
     if (bits % 16 != 0) return PSMC_E_INVAL;  // the block copy moves 16 bytes at a time
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     LaunchTimer lt(c, s, 2, c->timing_on ? c->timing_on : 1);
+    // unless this was the last step the context can take, the rows are also made ready for the next token
+    const bool more = c->t < c->T_max;
     return launch_paged_reindex(c->paged, pp, c->sources[0], c->dst_rows[0], c->counts[c->t & 1], c->counts[c->t & 1] + 1,
-                                c->status, s) == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
+                                more ? c->len : nullptr, more ? c->done : nullptr, c->status, s) == cudaSuccess
+               ? PSMC_OK : PSMC_E_CUDA;
 }
 
 extern "C" const int32_t* psmc_kv_paged_table(psmc_ctx* c) { return c ? c->paged.table : nullptr; }

@@ -172,9 +172,11 @@ cudaError_t launch_paged_init(const PagedState& ps, const int32_t* prompt_len_de
                               int32_t* status, cudaStream_t stream);
 cudaError_t launch_paged_append(const PagedState& ps, const int32_t* len, const uint8_t* done, int32_t* status,
                                 cudaStream_t stream);
+// len / done: NULL, or the rows' lengths and finished flags after the step: every live row then also gets the block
+// its next position needs
 cudaError_t launch_paged_reindex(const PagedState& ps, const PagedPools& pools, const MoveSource* sources,
                                  const int32_t* dst_rows, const int32_t* n_sources, const int32_t* n_moves,
-                                 int32_t* status, cudaStream_t stream);
+                                 const int32_t* len, const uint8_t* done, int32_t* status, cudaStream_t stream);
 
 // ---------------------------------------------------------------- final draw and back-trace
 struct SelectArgs {

@@ -8,7 +8,8 @@
 //   paged_append_kernel    a new block for every live row whose next position starts one (pops only)
 //   paged_release_kernel   rewritten slots return their blocks (pushes only)
 //   paged_acquire_kernel   table entries and reference counts of the ancestors' full blocks, a fresh block for
-//                          the partly filled one (pops only); leaves one copy order per rewritten slot
+//                          the partly filled one (pops only); leaves one copy order per rewritten slot; then the
+//                          append for the next token, so that a token costs three launches here, not four
 //   paged_copy_kernel      the copy orders: (layer, K/V, head) x live positions of the last block
 // Pushes and pops never meet in one kernel, so the free list needs nothing beyond one atomic counter.
 #include "common.cuh"
@@ -84,10 +85,10 @@ __global__ void __launch_bounds__(1024) paged_init_kernel(const PagedState ps, c
     if (!ok) raise_status(status, PSMC_E_NOMEM);
 }
 
-__global__ void paged_append_kernel(const PagedState ps, const int32_t* len, const uint8_t* done, int32_t* status) {
-    chain_begin();
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= ps.R || done[r]) return;
+// A block for row r's next position if that position starts a block and the row has none there yet (pops only).
+__device__ __forceinline__ void append_row(const PagedState& ps, int r, const int32_t* len, const uint8_t* done,
+                                           int32_t* status) {
+    if (done[r]) return;
     const int p = len[r];
     if (p % ps.block_len != 0) return;  // the row's last block still has room
     const int j = p / ps.block_len;
@@ -95,10 +96,18 @@ __global__ void paged_append_kernel(const PagedState ps, const int32_t* len, con
         raise_status(status, PSMC_E_STATE);
         return;
     }
+    int32_t* slot = ps.table + (int64_t)r * ps.max_blocks + j;
+    if (*slot >= 0) return;  // already there (an earlier call, or the reindex before this token)
     const int blk = pop_block(ps, status);
     if (blk < 0) return;
     ps.refc[blk] = 1;
-    ps.table[(int64_t)r * ps.max_blocks + j] = blk;
+    *slot = blk;
+}
+
+__global__ void paged_append_kernel(const PagedState ps, const int32_t* len, const uint8_t* done, int32_t* status) {
+    chain_begin();
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < ps.R) append_row(ps, r, len, done, status);
 }
 
 __global__ void paged_release_kernel(const PagedState ps, const int32_t* dst_rows, const int32_t* n_moves) {
@@ -115,30 +124,40 @@ __global__ void paged_release_kernel(const PagedState ps, const int32_t* dst_row
     }
 }
 
+// len / done non-NULL: the kernel also gives every live row the block its next position needs (what
+// paged_append_kernel does), so that the next token needs no launch of its own for that.
 __global__ void paged_acquire_kernel(const PagedState ps, const MoveSource* sources, const int32_t* dst_rows,
-                                     const int32_t* n_sources, int32_t* status) {
+                                     const int32_t* n_sources, const int32_t* len, const uint8_t* done,
+                                     int32_t* status) {
     chain_begin();
     const int n = *n_sources;
     CopyOrder* orders = orders_of(ps);
-    for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < n; s += gridDim.x * blockDim.x) {
+    const int lane = threadIdx.x & 31;
+    const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = (gridDim.x * blockDim.x) >> 5;
+    // one warp per surviving source: its lanes share the full blocks (a reference per destination, the table entries of
+    // every destination) and then the destinations (a fresh block each for the partly filled one)
+    for (int s = warp_global; s < n; s += n_warps) {
         const MoveSource ms = sources[s];
         const int nfull = ms.len / ps.block_len, rem = ms.len % ps.block_len;
         const int32_t* src_row = ps.table + (int64_t)ms.src_row * ps.max_blocks;
-        for (int j = 0; j < nfull; ++j)
-            if (src_row[j] >= 0) atomicAdd(&ps.refc[src_row[j]], ms.n_dst);
+        for (int j = lane; j < nfull; j += 32) {
+            const int blk = src_row[j];
+            if (blk >= 0) atomicAdd(&ps.refc[blk], ms.n_dst);
             else raise_status(status, PSMC_E_STATE);  // a live position without a block: the table was not kept up
-        for (int d = 0; d < ms.n_dst; ++d) {
+            for (int d = 0; d < ms.n_dst; ++d)
+                ps.table[(int64_t)dst_rows[ms.dst_begin + d] * ps.max_blocks + j] = blk;
+        }
+        const int last_blk = rem ? src_row[nfull] : -1;
+        if (rem && last_blk < 0 && lane == 0) raise_status(status, PSMC_E_STATE);
+        for (int d = lane; d < ms.n_dst; d += 32) {
             const int m = ms.dst_begin + d;
-            int32_t* dst_row = ps.table + (int64_t)dst_rows[m] * ps.max_blocks;
-            for (int j = 0; j < nfull; ++j) dst_row[j] = src_row[j];
             CopyOrder o{-1, -1, 0};
-            if (rem && src_row[nfull] < 0) raise_status(status, PSMC_E_STATE);
-            if (rem && src_row[nfull] >= 0) {
+            if (rem && last_blk >= 0) {
                 const int blk = pop_block(ps, status);
                 if (blk >= 0) {
                     ps.refc[blk] = 1;
-                    dst_row[nfull] = blk;
-                    o.src_blk = src_row[nfull];
+                    ps.table[(int64_t)dst_rows[m] * ps.max_blocks + nfull] = blk;
+                    o.src_blk = last_blk;
                     o.dst_blk = blk;
                     o.positions = rem;
                 }
@@ -146,6 +165,11 @@ __global__ void paged_acquire_kernel(const PagedState ps, const MoveSource* sour
             orders[m] = o;  // one order per rewritten slot, at the slot's place in the move list
         }
     }
+    // The next token's blocks.  A rewritten slot's entry for a block that starts at its length is touched by nothing
+    // above (full blocks end below it, a partly filled one excludes it), so this needs no ordering with the loops above.
+    if (len)
+        for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < ps.R; r += gridDim.x * blockDim.x)
+            append_row(ps, r, len, done, status);
 }
 
 // item = (rewritten slot m, pool q): all heads of the live positions of one block
@@ -193,11 +217,12 @@ cudaError_t launch_paged_append(const PagedState& ps, const int32_t* len, const 
 
 cudaError_t launch_paged_reindex(const PagedState& ps, const PagedPools& pools, const MoveSource* sources,
                                  const int32_t* dst_rows, const int32_t* n_sources, const int32_t* n_moves,
-                                 int32_t* status, cudaStream_t stream) {
+                                 const int32_t* len, const uint8_t* done, int32_t* status, cudaStream_t stream) {
     cudaError_t e = launch_chained(paged_release_kernel, dim3(kSMs), dim3(256), 0, stream, ps, dst_rows, n_moves);
     if (e != cudaSuccess) return e;
-    e = launch_chained(paged_acquire_kernel, dim3((unsigned)((ps.R + 127) / 128)), dim3(128), 0, stream, ps, sources,
-                       dst_rows, n_sources, status);
+    // a warp per source; there are at most R / 2 of them (each has at least one destination besides itself)
+    e = launch_chained(paged_acquire_kernel, dim3((unsigned)((ps.R / 2 + 7) / 8 + 1)), dim3(256), 0, stream, ps, sources,
+                       dst_rows, n_sources, len, done, status);
     if (e != cudaSuccess) return e;
     return launch_chained(paged_copy_kernel, dim3(kSMs * 4), dim3(256), 0, stream, ps, pools, n_moves);
 }
