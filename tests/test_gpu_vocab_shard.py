@@ -87,6 +87,14 @@ def test_sharded_step_small_vocabulary(world):
     assert st.resample_events > 0 and (owners > 0).all()
 
 
+def test_sharded_step_more_ranks_than_lanes():
+    """40 ranks: the row totals are then formed by walking the gathered triples in global memory instead of handing
+    one rank's triple to each lane of a warp."""
+    cfg = W.CONFIGS["tiny"]
+    st, owners = sharded_loop(cfg, 8, 12, VS.vocab_shards(cfg.V, 40))
+    assert st.steps == 12 and owners.sum() == st.live_rows
+
+
 def test_sharded_step_uneven_unaligned_shards():
     """Shards that start off the 16-byte grid (scalar load path) and differ widely in size."""
     cfg = W.CONFIGS["tiny"]                       # V = 1024, fp32
@@ -96,7 +104,7 @@ def test_sharded_step_uneven_unaligned_shards():
 
 
 @pytest.mark.parametrize("name,world,T,G", [("llama2_7b", 2, 24, None), ("llama2_7b", 8, 16, 3), ("qwen25_7b", 4, 12, None),
-                                            ("batched_prompts", 8, 6, 4)])
+                                            ("batched_prompts", 8, 6, 4), ("resample_stress", 8, 6, None)])
 def test_sharded_step_model_vocabularies(name, world, T, G):
     cfg = W.CONFIGS[name]
     st, owners = sharded_loop(cfg, 11, T, VS.vocab_shards(cfg.V, world), G=G)
