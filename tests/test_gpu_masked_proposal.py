@@ -141,3 +141,23 @@ def test_mask_argument_checks_and_snapshot():
     assert ps.sync_status() == B.OK and other.sync_status() == B.OK
     ps.destroy()
     other.destroy()
+
+
+def test_masked_steps_random_settings():
+    """Sixteen seeded draws of (groups, particles, vocabulary, dtype, alpha, tau, ramp) with a random rule each."""
+    rng = np.random.default_rng(20260213)
+    for case in range(16):
+        N = int(rng.choice([1, 3, 8, 17, 33]))
+        G = int(rng.integers(1, 4))
+        V = int(rng.choice([16, 100, 1024, 3001, 20000, 70001]))
+        alpha = float(rng.choice([1.0, 2.0, 4.0, 1.0 + 4.0 * rng.random()]))
+        tau = 1.0 / alpha if rng.random() < 0.6 else float(0.2 + rng.random())
+        c = W.Workload("masked%d" % case, G, N, V, "bf16" if rng.random() < 0.5 else "f32", float(rng.choice([1.0, 3.0, 6.0])),
+                       1.5, 12, 3, 9, alpha, tau, float(rng.choice([0.3, 0.5, 0.9])), int(rng.choice([0, 0, 4])),
+                       1, 2, 16, 32)
+        if rng.random() < 0.5:
+            rule = dict(top_k=int(rng.choice([1, 5, 40, 300, 2500, 10**6])))
+        else:
+            rule = dict(top_p=float(rng.choice([0.1, 0.5, 0.9, 0.99, 0.99995, 1.0])))
+        st = P.closed_loop(c, seed=200 + case, T=8, **rule)
+        assert st.steps == 8, (case, rule)
