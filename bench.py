@@ -303,6 +303,22 @@ def run_ours(args):
     step_us = 1e3 * cms[0] / max(cn[0], 1)
     step_gbs = k1_bytes / (cms[0] * 1e-3) / 1e9 if cms[0] > 0 else 0.0
 
+    # ---- pass D: the same K steps without the cache moves between them, per-kernel brackets: the logit pass when no
+    # reindex has left its writes in L2 for it to drain (the particle state does not depend on the caches) ----
+    reset_all()
+    for t in range(1, Wm + 1):
+        ps.step(blocks[(t - 1) % N_BLOCKS])
+    torch.cuda.synchronize(dev)
+    ps.timing_enable(True)
+    for t in range(Wm + 1, Wm + K + 1):
+        ps.step(blocks[(t - 1) % N_BLOCKS])
+    dms, dn = ps.timing_read()
+    ps.timing_enable(False)
+    if dms[0] > 0:
+        alone_gbs = k1_bytes / (dms[0] * 1e-3) / 1e9
+        roofs[k1_name]["without_cache_moves"] = {"avg_launch_us": 1e3 * dms[0] / max(dn[0], 1), "achieved": alone_gbs,
+                                                 "frac": alone_gbs / hbm_peak}
+
     # ---- e2e: host logits in, tokens out, every step, through psmc_step_host ----
     Ke = min(K, args.e2e_steps)
     host_blocks = [b.cpu().pin_memory() for b in blocks]
