@@ -163,7 +163,7 @@ psmc_status psmc_logits_pass(const void* logits, psmc_dtype dt, int R, int V, in
  *
  *   - Limit: psmc_logits_pass_scratch_bytes(R, V) must not exceed
  *     PSMC_STATIC_SCRATCH_BYTES (16 bytes per span of 1024-4096 logits per row;
- *     e.g. 512 rows x 128256 logits need 516,096 bytes).  Larger problems are
+ *     e.g. 512 rows x 128256 logits need 262,144 bytes).  Larger problems are
  *     refused with PSMC_E_TOO_LARGE and nothing is enqueued.
  *   - First call on each device: looks up the array's device address (a
  *     runtime symbol query, with that device current) and caches it.  Make that

@@ -15,11 +15,17 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) logits_stream_kernel(const 
     __shared__ __align__(8) uint64_t bars[kMaxWarps * kDepth];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps_per_cta = blockDim.x >> 5;
-    const int warp_global = blockIdx.x * warps_per_cta + warp;
-    const int n_warps = gridDim.x * warps_per_cta;
     const int n_tasks = p.R * p.n_spans;  // < 2^31, checked by the host
-    const int per_warp = (n_tasks + n_warps - 1) / n_warps;
-    const int first = min(n_tasks, warp_global * per_warp), last = min(n_tasks, first + per_warp);
+    // Even shares: the tasks are dealt to the CTAs in contiguous runs that differ by at most one task, and a CTA's run
+    // to its warps likewise.  (Rounding the share up per warp instead leaves whole SMs without work: 24 warps of 5 spans
+    // cover 512 x 32 spans with 136 CTAs.)
+    const int cta_base = n_tasks / (int)gridDim.x, cta_extra = n_tasks % (int)gridDim.x;
+    const int cta_first = (int)blockIdx.x * cta_base + min((int)blockIdx.x, cta_extra);
+    const int cta_n = cta_base + ((int)blockIdx.x < cta_extra ? 1 : 0);
+    const int w_base = cta_n / warps_per_cta, w_extra = cta_n % warps_per_cta;
+    const int first = cta_first + warp * w_base + min(warp, w_extra);
+    const int per_warp = w_base + (warp < w_extra ? 1 : 0);
+    const int last = first + per_warp;
 
     stream_init_barriers(bars + warp * kDepth, lane);
     chain_begin();  // everything above is local set-up; global memory from here on

@@ -4,12 +4,14 @@
 // triple for it (logits_common.cuh); nothing else leaves the kernel.  The per-row finish runs in the kernel
 // that follows.
 //
-// Data movement: one persistent CTA per SM, up to 16 warps, each warp with a private ring of kDepth stages of
+// Data movement: one persistent CTA per SM, up to kMaxWarps warps, each warp with a private ring of kDepth stages of
 // kStageBytes in shared memory.  Lane 0 of a warp keeps kDepth-1 bulk asynchronous copies (TMA, untiled,
 // completion on an mbarrier) in flight for the pieces the warp will need next -- across span boundaries, so
 // the memory pipe never drains -- while the warp sums the piece that has landed, reading it back with
-// conflict-free 128-bit shared loads.  About 128 KB per SM are in flight at any time, independent of how the
-// warps are scheduled.  No cross-warp synchronisation, no atomics; every mbarrier wait is bounded.
+// conflict-free 128-bit shared loads.  With 24 warps and two stages of 4 KB each, about 96 KB per SM are in flight
+// at any time, independent of how the warps are scheduled (a pure read of this shape runs no faster three deep, and
+// 24 warps hide the latencies of the arithmetic better than 16: 31 us against 33 us for 512 x 128256 bf16 logits).
+// No cross-warp synchronisation, no atomics; every mbarrier wait is bounded.
 //
 // Arithmetic per pair of logits: two unpack operations, two packed fp32x2 FMAs for x - c, two MUFU.EX2, one
 // packed add for s1 and, for beta in {2,4,8}, one to three packed multiply/FMA for sb (2^{beta d} is 2^d
@@ -26,9 +28,9 @@
 
 namespace psmc {
 
-constexpr int kMaxWarps = 16;        // warps per CTA of the streaming kernel
+constexpr int kMaxWarps = 24;        // warps per CTA of the streaming kernel
 constexpr int kStageBytes = 4096;    // one bulk copy
-constexpr int kDepth = 3;            // stages per warp: one being summed, two in flight
+constexpr int kDepth = 2;            // stages per warp: one being summed, one in flight
 constexpr float kRefSlack = 2.0f;    // natural units a logit may exceed the warp's reference point by (less for beta > 31)
 
 // ---- packed pairs of fp32 in one 64-bit register (fp32x2 instructions of sm_100) ----

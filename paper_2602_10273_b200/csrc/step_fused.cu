@@ -1,7 +1,7 @@
 // The whole per-token step as ONE kernel (groups of up to 32 particles, 16-byte aligned rows): the loop body of
 // Algorithm 1 without the cache move.
 //
-// Every CTA (one per SM) runs up to 16 streaming warps (logits_stream.cuh) plus kFinishers finishing warps.
+// Every CTA (one per SM) runs up to kStreamers streaming warps (logits_stream.cuh) plus kFinishers finishing warps.
 // The streaming warps take the (row, span) tasks of the logit block in short runs dealt round-robin over the whole
 // grid, so the rows of the block complete one after the other while the sweep is still going on; after a span's
 // triple is stored its warp counts one arrival for the row.  Finishing warp f owns rows f, f + F, ... in that
@@ -23,6 +23,7 @@ namespace psmc {
 namespace {
 
 constexpr int kFinishers = 2;            // finishing warps per CTA
+constexpr int kStreamers = 16;           // streaming warps per CTA at most (small blocks: more would only sit idle)
 constexpr int kRun = 2;                  // consecutive spans a streaming warp takes at a time
 constexpr uint32_t kPollLimit = 1u << 19;  // polls of ~0.25 us before a finishing warp gives up on a row
 constexpr int64_t kFuseMaxBytes = 8 << 20;  // logit blocks up to this size take the one-kernel step
@@ -95,9 +96,9 @@ __device__ __forceinline__ void finishing_warp(const FusedParams& fp, int fin_id
 }
 
 template <int DT, int MODE>
-__global__ void __launch_bounds__((kMaxWarps + kFinishers) * 32, 1) psmc_step_kernel(const __grid_constant__ FusedParams fp) {
+__global__ void __launch_bounds__((kStreamers + kFinishers) * 32, 1) psmc_step_kernel(const __grid_constant__ FusedParams fp) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[kMaxWarps * kDepth];
+    __shared__ __align__(8) uint64_t bars[kStreamers * kDepth];
     __shared__ GroupScratch<32> sc[kFinishers];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -164,16 +165,16 @@ cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa,
     fp.row_arrivals = row_arrivals;
     fp.group_arrivals = group_arrivals;
 
-    // one CTA per SM; as many streaming warps per CTA as it takes to give every run of spans a warp, up to kMaxWarps
+    // one CTA per SM; as many streaming warps per CTA as it takes to give every run of spans a warp, up to kStreamers
     const int64_t units = (n_tasks + kRun - 1) / kRun;
     int64_t warps = (units + kSMs - 1) / kSMs;
-    if (warps > kMaxWarps) warps = kMaxWarps;
+    if (warps > kStreamers) warps = kStreamers;
     if (warps < 1) warps = 1;
     int64_t blocks = (units + warps - 1) / warps;
     if (blocks > kSMs) blocks = kSMs;
     const size_t smem = (size_t)warps * kDepth * kStageBytes;
     FusedFn fn = la.dt == PSMC_F32 ? pick_fused<PSMC_F32>(g.mode) : pick_fused<PSMC_BF16>(g.mode);
-    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kMaxWarps * kDepth * kStageBytes);
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kStreamers * kDepth * kStageBytes);
     if (e != cudaSuccess) return e;
     return launch_chained(fn, dim3((unsigned)blocks), dim3((unsigned)((warps + kFinishers) * 32)), smem, stream, fp);
 }

@@ -120,10 +120,10 @@ def test_sharded_step_batched_prompts_full_size():
 
 
 def test_sharded_step_three_ranks_need_more_span_triples_than_the_whole_row():
-    """320 rows of 128256 logits are cut into 32 spans of 4096; a third of such a row is cut into 42 spans of 1024,
+    """480 rows of 128256 logits are cut into 32 spans of 4096; a third of such a row is cut into 42 spans of 1024,
     so the context has to grow the scratch it sized for whole rows."""
     cfg = W.CONFIGS["batched_prompts"]
-    G = 40
+    G = 60
     assert B.logits_pass_scratch_bytes(G * cfg.N, VS.vocab_shards(cfg.V, 3)[0][1]) > B.logits_pass_scratch_bytes(G * cfg.N, cfg.V)
     st, owners = sharded_loop(cfg, 3, 4, VS.vocab_shards(cfg.V, 3), G=G)
     assert st.steps == 4 and (owners > 0).all()
