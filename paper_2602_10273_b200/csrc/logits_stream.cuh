@@ -237,6 +237,8 @@ struct TaskDesc {
 template <int DT>
 struct TaskWalker {
     int task, end, row, sp, run, run_left, skip;
+    int flag_row;        // row whose finished flag is held in `flag` (-1: none yet)
+    unsigned char flag;
     __device__ __forceinline__ void seat(const StreamParams& p) {
         row = task / p.n_spans;
         sp = task - row * p.n_spans;
@@ -246,6 +248,8 @@ struct TaskWalker {
         end = last;
         run = run_left = run_len;
         skip = skip_len;
+        flag_row = -1;
+        flag = 0;
         seat(p);
     }
     __device__ __forceinline__ bool at_end() const { return task >= end; }
@@ -261,9 +265,13 @@ struct TaskWalker {
         }
     }
     // false: the row is finished and its logits are not to be read (absorbing state)
-    __device__ __forceinline__ bool describe(const StreamParams& p, TaskDesc& d) const {
+    __device__ __forceinline__ bool describe(const StreamParams& p, TaskDesc& d) {
         constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;  // logits per 16 bytes
-        if (p.done && p.done[row]) return false;
+        if (row != flag_row) {  // one trip to memory per row, not per span: the warp waits for it with nothing in flight
+            flag_row = row;
+            flag = p.done ? p.done[row] : 0;
+        }
+        if (flag) return false;
         d.row = row;
         d.sp = sp;
         const int a0 = sp * p.span;
