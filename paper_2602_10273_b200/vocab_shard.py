@@ -58,11 +58,18 @@ class TorchDistExchange(Exchange):
         self.group = group
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
+        self._flat = True
 
     def all_gather(self, t: torch.Tensor) -> torch.Tensor:
         out = torch.empty((self.world,) + tuple(t.shape), dtype=t.dtype, device=t.device)
-        # a list of views into `out`: works on every backend, and NCCL turns it into one flat all-gather
-        self._dist.all_gather([out[r] for r in range(self.world)], t.contiguous(), group=self.group)
+        t = t.contiguous()
+        if self._flat:
+            try:  # one flat collective straight into `out`
+                self._dist.all_gather_into_tensor(out.view(-1), t.view(-1), group=self.group)
+                return out
+            except (RuntimeError, NotImplementedError):
+                self._flat = False  # a backend without it: the list form from now on
+        self._dist.all_gather([out[r] for r in range(self.world)], t, group=self.group)
         return out
 
 
