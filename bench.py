@@ -9,6 +9,11 @@ Prints ONE JSON line.  `value` is particle-tokens/s with every input resident in
 same metric through psmc_step_host (pinned host logits copied in, tokens copied out, every step).
 Multi-GPU (torchrun): every rank runs its own set of prompts (no data-path collective; weak scaling);
 time is the max over ranks of the device time of the K timed steps.
+
+The K steps are made several times: once to record the bytes each step moves, once for the headline time, once with
+CUDA events around every kernel (`kernels`, `roofline`), once with one bracket per psmc_step (`step_without_kv`), once
+without the cache moves (`kernels.*.without_cache_moves`), and a few of them through psmc_step_host (`e2e`).
+Supplementary runs: --paged-kv, --skip-shared-prompt, --top-k K, --top-p P (see their help lines).
 """
 from __future__ import annotations
 
@@ -35,7 +40,7 @@ N_BLOCKS = 6           # distinct logit blocks rotated through (6 x 131 MB at th
 # under profiles/ (logits_stream_kernel__batched_prompts.md, reindex_bulk_kernel__64rows_8layers_len1024.md; the
 # reindex capture ran on a smaller cache and its traffic scales with the bytes moved).  An entry goes back to None
 # when its kernel changes, until the counters are taken again.
-TRAFFIC_PER_ALGORITHMIC_BYTE = {"logits_stream_kernel": 1.032, "reindex_bulk_kernel": 0.978}
+TRAFFIC_PER_ALGORITHMIC_BYTE = {"logits_stream_kernel": 1.03, "reindex_bulk_kernel": 0.978}
 
 
 def load_peaks():
