@@ -295,7 +295,8 @@ const double*  psmc_ess(psmc_ctx*);          /* [G] ESS of Eq. 5 before resampli
 const double*  psmc_log_z(psmc_ctx*);        /* [G] running log of the normaliser estimate               */
 const int32_t* psmc_mask_sizes(psmc_ctx*);    /* [R] size of the proposal's support at the last step (psmc_set_proposal_mask) */
 const int32_t* psmc_lens(psmc_ctx*);         /* [R] live KV length                                       */
-const uint8_t* psmc_done(psmc_ctx*);         /* [R]                                                      */
+const uint8_t* psmc_done(psmc_ctx*);         /* [R] finished flags (ask again after each step: steps read one array
+                                                    and write another, and the two alternate)                 */
 const int32_t* psmc_move_count(psmc_ctx*);   /* [1] slots rewritten by the last step's maps (ask again after each step:
                                                     the counter alternates between two words)                */
 

@@ -14,7 +14,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libpsmc.so")
 LIB_WORKLOAD = os.path.join(PKG, "libpsmc_workload.so")
 
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "--threads", "0", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 
 PRODUCT_SOURCES = ["context.cu", "logits_pass.cu", "step_fused.cu", "weights_resample.cu", "vocab_shard.cu",

@@ -41,7 +41,7 @@ struct psmc_ctx {
     PagedState paged;          // block table, reference counts and free list of the paged cache (zero until created)
     // particle state
     double *logW, *S;
-    uint8_t* done;
+    uint8_t* done2[2];  // finished flags after steps of even / odd index: step t reads [(t-1)&1] and writes [t&1]
     int32_t* len;
     // results of the last step
     int32_t *tok, *last_tok, *anc, *map, *resampled;
@@ -52,8 +52,9 @@ struct psmc_ctx {
     MoveSource* sources[2];
     int32_t* dst_rows[2];
     int32_t* counts[3];  // {n_sources, n_moves}: [0]/[1] steps of even/odd index (they alternate), [2] idx_override
-    int32_t* row_arrivals;    // [R] arrival counters of the fused step kernel (zero between launches)
+    int32_t* row_arrivals;    // [R] arrival counters of the one-kernel step (zero between launches)
     int32_t* group_arrivals;  // [G]
+    void* step_triples;       // its triples of rows shared between CTAs
     int32_t* status;
     int32_t* kv_work;    // [2] unit queue of the reindex kernels (kept at zero between launches by the kernels)
     void* scratch;       // span triples of the logit pass
@@ -74,6 +75,9 @@ struct psmc_ctx {
 
 namespace {
 
+// finished flags after the steps taken so far
+uint8_t* done_now(const psmc_ctx* c) { return c->done2[c->t & 1]; }
+
 template <typename T>
 cudaError_t dev_alloc(T** p, size_t count) {
     return cudaMalloc(reinterpret_cast<void**>(p), (count ? count : 1) * sizeof(T));
@@ -90,7 +94,7 @@ psmc_status reset_device_state(psmc_ctx* c) {
     const size_t R = (size_t)c->R, G = (size_t)c->G;
     cudaError_t e = cudaSuccess;
     auto z = [&](void* p, size_t bytes) { if (e == cudaSuccess) e = cudaMemset(p, 0, bytes); };
-    z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done, R);
+    z(c->logW, 8 * R); z(c->S, 8 * R); z(c->done2[0], R); z(c->done2[1], R);
     z(c->logp, 8 * R); z(c->loginc, 8 * R); z(c->logZ, 8 * G); z(c->resampled, 4 * G);
     z(c->counts[0], 8); z(c->counts[1], 8); z(c->counts[2], 8); z(c->status, 4); z(c->kv_work, 8);
     z(c->row_arrivals, 4 * R); z(c->group_arrivals, 4 * G); z(c->set_size, 4 * R);
@@ -152,10 +156,10 @@ void free_ctx(psmc_ctx* c) {
     for (auto e : c->event_pool) cudaEventDestroy(e);
     if (c->staged) cudaEventDestroy(c->staged);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
-    void* ptrs[] = {c->logW, c->S, c->done, c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
+    void* ptrs[] = {c->logW, c->S, c->done2[0], c->done2[1], c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
-                    c->group_arrivals, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev, c->set_size};
+                    c->group_arrivals, c->step_triples, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev, c->set_size};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     void* paged_ptrs[] = {c->paged.table, c->paged.refc, c->paged.free_list, c->paged.free_top};
@@ -190,7 +194,8 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     const size_t R = (size_t)c->R;
     cudaError_t e = cudaSuccess;
     auto ok = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
-    ok(dev_alloc(&c->logW, R)); ok(dev_alloc(&c->S, R)); ok(dev_alloc(&c->done, R)); ok(dev_alloc(&c->len, R));
+    ok(dev_alloc(&c->logW, R)); ok(dev_alloc(&c->S, R)); ok(dev_alloc(&c->done2[0], R)); ok(dev_alloc(&c->done2[1], R));
+    ok(dev_alloc(&c->len, R));
     ok(dev_alloc(&c->tok, R)); ok(dev_alloc(&c->last_tok, R));
     ok(dev_alloc(&c->anc, R)); ok(dev_alloc(&c->map, R)); ok(dev_alloc(&c->resampled, (size_t)G));
     ok(dev_alloc(&c->logp, R)); ok(dev_alloc(&c->loginc, R)); ok(dev_alloc(&c->ess, (size_t)G));
@@ -202,6 +207,7 @@ extern "C" psmc_status psmc_init_batched(psmc_ctx** out, int G, int N, int V, fl
     }
     for (int s = 0; s < 3; ++s) ok(dev_alloc(&c->counts[s], 2));
     ok(dev_alloc(&c->row_arrivals, R)); ok(dev_alloc(&c->group_arrivals, (size_t)G));
+    ok(cudaMalloc(&c->step_triples, step_fused_scratch_bytes()));
     ok(dev_alloc(&c->prompt_len_dev, (size_t)G));
     if (e == cudaSuccess) e = cudaMemcpy(c->prompt_len_dev, c->prompt_len_host, 4 * (size_t)G, cudaMemcpyHostToDevice);
     ok(dev_alloc(&c->status, 1));
@@ -271,7 +277,7 @@ WeightsArgs weights_args(psmc_ctx* c, int t, const StepExponents& x) {
     wa.alpha_t = x.alpha_t; wa.beta = x.beta_t; wa.delta = x.alpha_t - x.alpha_prev; wa.kappa = c->kappa;
     wa.seed = c->seed;
     wa.logp = c->logp; wa.loginc = c->loginc;
-    wa.logW = c->logW; wa.S = c->S; wa.done = c->done; wa.len = c->len;
+    wa.logW = c->logW; wa.S = c->S; wa.done = c->done2[(t - 1) & 1]; wa.done_out = c->done2[t & 1]; wa.len = c->len;
     wa.tok = c->tok; wa.last_tok = c->last_tok; wa.anc = c->anc; wa.map = c->map;
     wa.resampled = c->resampled; wa.ess = c->ess; wa.logZ = c->logZ;
     wa.hist_tok = c->hist_tok + (size_t)(t - 1) * c->R;
@@ -293,7 +299,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
 
     LogitsStreamArgs la{};
     la.logits = logits; la.dt = dt; la.R = c->R; la.V = c->V; la.ld = ld; la.beta = x.beta_t;
-    la.done = c->done; la.scratch = c->scratch;
+    la.done = done_now(c); la.scratch = c->scratch;
     la.status = c->status;
     la.zero_words = c->counts[(t + 1) & 1];  // each step clears the pair of move counters the next step will use
 
@@ -305,7 +311,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
         if (launch_step_masked(la, wa, c->top_k, c->top_p, c->set_size, s) != cudaSuccess) return PSMC_E_CUDA;
     } else if (step_can_fuse(la, c->N)) {  // the whole step as one kernel
         LaunchTimer lt(c, s, 0);
-        if (launch_step_fused(la, wa, c->row_arrivals, c->group_arrivals, s) != cudaSuccess) return PSMC_E_CUDA;
+        if (launch_step_fused(la, wa, c->step_triples, c->row_arrivals, c->group_arrivals, s) != cudaSuccess) return PSMC_E_CUDA;
     } else {
         {
             LaunchTimer lt(c, s, 0);
@@ -341,7 +347,7 @@ extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, p
     const StepExponents x = exponents_at(c, t);
     LogitsStreamArgs la{};
     la.logits = logits_local; la.dt = dt; la.R = c->R; la.V = V_local; la.ld = ld; la.beta = x.beta_t;
-    la.done = c->done; la.scratch = c->scratch;
+    la.done = done_now(c); la.scratch = c->scratch;
     la.status = c->status;
     la.zero_words = c->counts[(t + 1) & 1];
     LaunchTimer lt(c, s, 0);
@@ -508,7 +514,7 @@ extern "C" psmc_status psmc_kv_paged_create(psmc_ctx* c, int n_blocks, int block
 extern "C" psmc_status psmc_kv_paged_append(psmc_ctx* c, void* stream) {
     if (!c) return PSMC_E_INVAL;
     if (!c->paged.table) return PSMC_E_STATE;
-    return launch_paged_append(c->paged, c->len, c->done, c->status, static_cast<cudaStream_t>(stream)) == cudaSuccess
+    return launch_paged_append(c->paged, c->len, done_now(c), c->status, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? PSMC_OK : PSMC_E_CUDA;
 }
 
@@ -534,7 +540,7 @@ extern "C" psmc_status psmc_reindex_kv_paged(psmc_ctx* c, const psmc_kv_pools* p
     // unless this was the last step the context can take, the rows are also made ready for the next token
     const bool more = c->t < c->T_max;
     return launch_paged_reindex(c->paged, pp, c->sources[0], c->dst_rows[0], c->counts[c->t & 1], c->counts[c->t & 1] + 1,
-                                more ? c->len : nullptr, more ? c->done : nullptr, c->status, s) == cudaSuccess
+                                more ? c->len : nullptr, more ? done_now(c) : nullptr, c->status, s) == cudaSuccess
                ? PSMC_OK : PSMC_E_CUDA;
 }
 
@@ -560,7 +566,7 @@ extern "C" psmc_status psmc_set_state(psmc_ctx* c, const double* log_w, const do
     cudaError_t e = cudaSuccess;
     if (log_w) e = cudaMemcpy(c->logW, log_w, 8 * R, cudaMemcpyHostToDevice);
     if (e == cudaSuccess && cum_logp) e = cudaMemcpy(c->S, cum_logp, 8 * R, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess && done) e = cudaMemcpy(c->done, done, R, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && done) e = cudaMemcpy(done_now(c), done, R, cudaMemcpyHostToDevice);
     if (e == cudaSuccess && lens) e = cudaMemcpy(c->len, lens, 4 * R, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
@@ -592,7 +598,7 @@ int snapshot_pieces(psmc_ctx* c, int t, Piece* out) {
     add(c->len, 4 * R); add(c->tok, 4 * R); add(c->last_tok, 4 * R); add(c->anc, 4 * R); add(c->map, 4 * R);
     add(c->resampled, 4 * G); add(c->status, 4);
     add(c->hist_tok, 4 * R * (size_t)t); add(c->hist_map, 4 * R * (size_t)t);
-    add(c->done, R);
+    add(c->done2[t & 1], R);
     return n;
 }
 size_t snapshot_bytes(psmc_ctx* c, int t) {
@@ -713,7 +719,7 @@ extern "C" const double* psmc_ess(psmc_ctx* c) { return c ? c->ess : nullptr; }
 extern "C" const double* psmc_log_z(psmc_ctx* c) { return c ? c->logZ : nullptr; }
 extern "C" const int32_t* psmc_mask_sizes(psmc_ctx* c) { return c ? c->set_size : nullptr; }
 extern "C" const int32_t* psmc_lens(psmc_ctx* c) { return c ? c->len : nullptr; }
-extern "C" const uint8_t* psmc_done(psmc_ctx* c) { return c ? c->done : nullptr; }
+extern "C" const uint8_t* psmc_done(psmc_ctx* c) { return c ? done_now(c) : nullptr; }
 extern "C" const int32_t* psmc_move_count(psmc_ctx* c) { return c ? c->counts[c->t & 1] + 1 : nullptr; }
 extern "C" int psmc_step_index(const psmc_ctx* c) { return c ? c->t : -1; }
 extern "C" int psmc_rows(const psmc_ctx* c) { return c ? c->R : -1; }

@@ -80,7 +80,9 @@ struct WeightsArgs {
     // particle state, updated in place
     double* logW;
     double* S;
-    uint8_t* done;
+    const uint8_t* done;  // finished flags as the step finds them: read only, by any CTA at any time during the step
+    uint8_t* done_out;    // finished flags after the step (another array: a group may close while other CTAs still look
+                          // at the flags of its rows)
     int32_t* len;
     // per-step results
     int32_t* tok;       // [R] token of each slot this step (EOS for finished rows)
@@ -101,11 +103,13 @@ struct WeightsArgs {
 };
 cudaError_t launch_weights_resample(const WeightsArgs& a, cudaStream_t stream);
 
-// The logit pass and the per-group update as one kernel: possible for groups of up to 32 particles whose logit
-// rows start on 16-byte boundaries.  row_arrivals [R] and group_arrivals [G] are zero between launches.
+// The logit pass and the per-group update as one kernel (step_fused.cu): possible for groups of up to 32 particles
+// whose logit rows start on 16-byte boundaries.  shared_triples: step_fused_scratch_bytes() of device memory, contents
+// irrelevant; row_arrivals [R] and group_arrivals [G] are zero between launches (the kernel leaves them so).
 bool step_can_fuse(const LogitsStreamArgs& la, int N);
-cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, int32_t* row_arrivals,
-                              int32_t* group_arrivals, cudaStream_t stream);
+size_t step_fused_scratch_bytes();
+cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, void* shared_triples,
+                              int32_t* row_arrivals, int32_t* group_arrivals, cudaStream_t stream);
 
 // The step with the proposal restricted to the top_k tokens of each row, or to the nucleus of share top_p (exactly one
 // of the two > 0): one CTA per row for the logit pass, then the per-group update.  set_size: [R].

@@ -124,25 +124,25 @@ struct RowFrame {
     double target, base;
 };
 
+// Totals, target and selected span out of n triples handed out by fetch(j) (global memory, shared memory: the
+// arithmetic and its order are the same wherever the numbers come from); one warp, every lane gets the same result.
 // FRAMED: the triples are rescaled to fr->C instead of the row's own largest reference exponent, the prefix over the
 // spans starts at fr->base and looks for fr->target (U is not used).
-template <int MODE, bool FRAMED = false>
-__device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane,
-                                                   const RowFrame* fr = nullptr) {
+template <int MODE, bool FRAMED = false, class Fetch>
+__device__ __forceinline__ RowTotals combine_triples(Fetch fetch, int n, double beta, double U, int lane,
+                                                     const RowFrame* fr = nullptr) {
     constexpr int kKeep = 8;  // span masses a lane keeps in registers between the two sweeps (rows of <= 256 spans)
     RowTotals t;
     t.ok = false;
-    const int n = p.n_spans;
-    const float4* P = p.partials + (size_t)row * n;
 
     // the lane's first triple is fetched once and kept (rows of up to 32 spans need no second trip to L2)
-    const float4 f0 = lane < n ? __ldcg(&P[lane]) : make_float4(kRefFloor, 0.f, 0.f, 0.f);
+    const float4 f0 = lane < n ? fetch(lane) : make_float4(kRefFloor, 0.f, 0.f, 0.f);
     float cf = kRefFloor;
     if (FRAMED) {
         cf = fr->C;
     } else {
         cf = f0.x;
-        for (int j = lane + 32; j < n; j += 32) cf = fmaxf(cf, __ldcg(&P[j]).x);
+        for (int j = lane + 32; j < n; j += 32) cf = fmaxf(cf, fetch(j).x);
         cf = warp_max(cf);
     }
     t.C = cf;
@@ -153,9 +153,9 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
 #pragma unroll
     for (int i = 0; i < kKeep; ++i) keep[i] = 0.0;
     for (int j = lane, i = 0; j < n; j += 32, ++i) {
-        const float4 f = i == 0 ? f0 : __ldcg(&P[j]);
+        const float4 f = i == 0 ? f0 : fetch(j);
         double f1, fb;
-        span_scales<MODE>(f.x - cf, p.beta, f1, fb);
+        span_scales<MODE>(f.x - cf, beta, f1, fb);
         const double a = (double)f.y * f1;
         const double b = (MODE == kBeta1) ? a : (double)f.z * fb;
         a_sum += a;
@@ -180,9 +180,9 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
             for (int q = 0; q < kKeep; ++q)
                 if (q == i) b = keep[q];
         } else if (j < n) {
-            const float4 f = __ldcg(&P[j]);
+            const float4 f = fetch(j);
             double f1, fb;
-            span_scales<MODE>(f.x - cf, p.beta, f1, fb);
+            span_scales<MODE>(f.x - cf, beta, f1, fb);
             b = (MODE == kBeta1) ? (double)f.y * f1 : (double)f.z * fb;
         }
         const double incl = carry + warp_scan_incl(b, lane);
@@ -210,9 +210,17 @@ __device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int ro
     return t;
 }
 
+// the triples of row `row` as the streaming kernel left them in global memory
+template <int MODE, bool FRAMED = false>
+__device__ __forceinline__ RowTotals combine_spans(const FinishParams& p, int row, double U, int lane,
+                                                   const RowFrame* fr = nullptr) {
+    const float4* P = p.partials + (size_t)row * p.n_spans;
+    return combine_triples<MODE, FRAMED>([&](int j) { return __ldcg(&P[j]); }, p.n_spans, p.beta, U, lane, fr);
+}
+
 // One lane's share of the selected span: `E` consecutive logits from e0 (clipped to b0).  Returns their mass
 // (eight logits summed in fp32 at a time, then in fp64).
-template <int DT, int MODE>
+template <int DT, int MODE, int BATCH = 4>
 __device__ __forceinline__ double lane_share(const FinishParams& p, const void* rowp, int e0, int E, int b0, float neg_C) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;  // logits per 16 bytes
     double lm = 0.0;
@@ -220,13 +228,13 @@ __device__ __forceinline__ double lane_share(const FinishParams& p, const void* 
     if (p.vec && e0 + E <= b0) {
         const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)e0 * (16 / kPer));
         const int Q = E / kPer;
-        for (int q0 = 0; q0 < Q; q0 += 4) {  // four loads in flight
-            uint4 v[4];
+        for (int q0 = 0; q0 < Q; q0 += BATCH) {  // BATCH loads in flight
+            uint4 v[BATCH];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < BATCH; ++i)
                 if (q0 + i < Q) v[i] = q[q0 + i];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < BATCH; ++i) {
                 if (q0 + i >= Q) break;
                 const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
                 float g[4];

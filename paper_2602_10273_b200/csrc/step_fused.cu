@@ -1,19 +1,32 @@
 // The whole per-token step as ONE kernel (groups of up to 32 particles, 16-byte aligned rows): the loop body of
-// Algorithm 1 without the cache move.
+// Algorithm 1 without the cache move -- proposal sums (Corollary 1), token draw, Eq. 7, weight update, ESS (Eq. 5),
+// trigger, resampling and slot map.
 //
-// Every CTA (one per SM) runs up to kStreamers streaming warps (logits_stream.cuh) plus kFinishers finishing warps.
-// The streaming warps take the (row, span) tasks of the logit block in short runs dealt round-robin over the whole
-// grid, so the rows of the block complete one after the other while the sweep is still going on; after a span's
-// triple is stored its warp counts one arrival for the row.  Finishing warp f owns rows f, f + F, ... in that
-// order: it waits (bounded) until a row has all its arrivals, draws the row's token and Eq. 7 from the triples
-// (finish_row_warp), and counts one arrival for the row's group; finished rows (absorbing EOS) arrive at once.
-// The warp that brings a group to N arrivals runs the group's update (weights_core.cuh) on the spot.  Only the rows
-// of the last wave and the last groups are finished after the sweep has ended; everything else hides behind it.
-// The context uses this kernel for small logit blocks, where saving a launch matters most (step_can_fuse).
+// How the logit block is dealt out.  Every row is cut into granules of 512 bytes; the R * granules-per-row granules
+// of the block, in row-major order, are split into one contiguous share per CTA (one CTA per SM, shares differ by at
+// most one granule).  A share meets a few rows: its "segments".  A segment that covers a whole row is LOCAL to the
+// CTA; the first and the last segment of a share may be parts of rows shared with the neighbouring CTAs.  Each
+// segment is split evenly among the CTA's streaming warps (a "piece" per warp, a few KB), which stream their pieces
+// through private rings of bulk asynchronous copies exactly as the stand-alone logit pass does (logits_stream.cuh)
+// and leave one (c, s1, sb) triple per piece: in shared memory for local segments, in global memory for shared rows.
+// The shared parts are taken first, then the whole rows one after the other, so rows complete one after the other
+// while the sweep is still running.
 //
-// The arrival counters are left at zero by their last user, so consecutive launches need no clearing.  The two
-// counters of the move lists alternate between steps (the kernel clears the pair the next step will use), because
-// a group may close and append to the lists while other CTAs are only starting.
+// Who finishes a row.  One extra warp per CTA, the finisher, follows the segments in the same order.  It waits on a
+// shared-memory mbarrier that the streaming warps of ITS OWN CTA arrive on (so every wait is for warps that are
+// resident by construction), then: a local row it finishes at once from the triples in shared memory; for a shared
+// row it takes a ticket on the row's global counter and the CTA that draws the last ticket finishes the row from
+// the triples in global memory.  No CTA ever waits for another one.  Finishing = totals in fp64, the piece that
+// holds U * sum, a re-read of that piece (it is a few KB and still in L2), the token, log p(y) and log omega
+// (logits_common.cuh).  A finished row counts one arrival for its group, and the warp that brings a group to N
+// arrivals runs the group's update (weights_core.cuh) on the spot.  Only the last row of each CTA is finished after
+// the sweep has ended, and that one by all warps of the CTA together (one 16-byte chunk of the piece per thread).
+//
+// The finished flags are read from one array and written to another (they alternate from step to step): a group may
+// close, and rewrite its flags, while other CTAs have not looked at the flags of their rows yet.  Arrival counters
+// are put back to zero by the warp that draws the last ticket, on every path, so consecutive launches need no
+// clearing.  The two counters of the move lists alternate between steps (the kernel clears the pair the next step
+// will use), because a group may append to the lists while other CTAs are only starting.
 #include <mutex>
 
 #include "logits_stream.cuh"
@@ -22,112 +35,471 @@
 namespace psmc {
 namespace {
 
-constexpr int kFinishers = 2;            // finishing warps per CTA
-constexpr int kStreamers = 16;           // streaming warps per CTA at most (small blocks: more would only sit idle)
-constexpr int kRun = 2;                  // consecutive spans a streaming warp takes at a time
-constexpr uint32_t kPollLimit = 1u << 19;  // polls of ~0.25 us before a finishing warp gives up on a row
-constexpr int64_t kFuseMaxBytes = 8 << 20;  // logit blocks up to this size take the one-kernel step
+constexpr int kGranule = 512;      // bytes: one 16-byte chunk per lane
+constexpr int kStepWarps = 23;     // streaming warps per CTA at most (with the finisher: 6 warps per scheduler, 80 registers)
+constexpr int kMaxSegments = 48;   // rows one CTA's share may meet (shapes beyond that take the two-kernel step)
+constexpr int kMinGranulesPerWarp = 4;
 
-struct FusedParams {
-    StreamParams s;
-    FinishParams f;
-    WeightsArgs a;
-    int32_t* row_arrivals;    // [R] spans of the row whose triple is stored
-    int32_t* group_arrivals;  // [G] rows of the group that are finished
+// How a block is cut up; a pure function of (R, V, dtype), the same on host and device.
+struct StepGeom {
+    int gpr;          // granules per row
+    int base, extra;  // a CTA's share: `base` granules, one more for the first `extra` CTAs
+    int row_bytes16;  // bytes of a row that bulk copies can fetch (a multiple of 16)
+    int tail;         // ragged logits after them
+    int W;            // streaming warps per CTA
+    int seg_cap;      // rows of the shared-memory triple table
 };
 
-__device__ __forceinline__ int load_volatile(const int32_t* p) { return *reinterpret_cast<const volatile int32_t*>(p); }
+struct StepParams {
+    const void* logits;
+    int R, V;
+    int64_t ld;
+    StepGeom g;
+    FinishParams f;
+    WeightsArgs a;
+    float4* shared_triples;   // [grid][2][W]: triples of the parts of rows a CTA shares with its neighbours
+    int32_t* row_arrivals;    // [R] CTAs that have delivered their part of a shared row
+    int32_t* group_arrivals;  // [G] rows of the group that are finished
+    int32_t* zero_words;
+};
+
+__host__ __device__ __forceinline__ int share_first(const StepGeom& g, int b) { return b * g.base + (b < g.extra ? b : g.extra); }
+__host__ __device__ __forceinline__ int share_count(const StepGeom& g, int b) { return g.base + (b < g.extra ? 1 : 0); }
+__host__ __device__ __forceinline__ int share_of(const StepGeom& g, int q) {  // the CTA whose share holds granule q
+    const int big = g.extra * (g.base + 1);
+    return q < big ? q / (g.base + 1) : g.extra + (q - big) / g.base;
+}
+
+// One segment: the part of row `row` inside the share of CTA `b`.
+struct Segment {
+    int row;
+    int g0, g1;  // granules [g0, g1) of the row
+    int slot;    // which of the CTA's two global triple rows a shared part uses
+    __device__ __forceinline__ bool local(const StepGeom& g) const { return g0 == 0 && g1 == g.gpr; }
+};
+__device__ __forceinline__ Segment segment_of_row(const StepGeom& g, int b, int row) {
+    const int first = share_first(g, b), last = first + share_count(g, b);
+    const int lo = max(first, row * g.gpr), hi = min(last, (row + 1) * g.gpr);
+    Segment s;
+    s.row = row;
+    s.g0 = lo - row * g.gpr;
+    s.g1 = hi - row * g.gpr;
+    s.slot = (row == first / g.gpr) ? 0 : 1;
+    return s;
+}
+// The CTA's segments in the order they are taken: the shared parts at the two ends first, then the rows in between.
+__device__ __forceinline__ int segment_in_order(int k, int S) {
+    if (S < 2) return 0;
+    return k == 0 ? S - 1 : k - 1;
+}
+// A segment's granules are dealt to the W streaming warps in vocabulary order, `place` 0 first; which warp takes which
+// place rotates with the row so that the spare granules do not always fall to the same warps.
+__device__ __forceinline__ int place_of_warp(int warp, int row, int W) { return (warp + row) % W; }
+__device__ __forceinline__ void piece_granules(const Segment& s, int place, int W, int& p0, int& p1) {
+    const int n = s.g1 - s.g0, base = n / W, extra = n % W;
+    p0 = s.g0 + place * base + min(place, extra);
+    p1 = p0 + base + (place < extra ? 1 : 0);
+}
+// logits [a0, b0) of the row that a piece covers (the piece that holds a row's last granule also owns the ragged end)
+template <int DT>
+__device__ __forceinline__ void piece_logits(const StepGeom& g, int V, int p0, int p1, int& a0, int& b0) {
+    constexpr int kPerGranule = kGranule / (DT == PSMC_F32 ? 4 : 2);
+    a0 = p0 * kPerGranule;
+    b0 = p1 == g.gpr ? V : p1 * kPerGranule;
+    if (p1 <= p0) b0 = a0;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+struct StepShared {
+    uint64_t ring_bars[kStepWarps * kDepth];
+    uint64_t seg_bars[kMaxSegments];     // one per segment: all streaming warps have stored their triple
+    unsigned char seg_done[kMaxSegments];  // the segment's row is finished (absorbing EOS): nothing is read or summed
+    GroupScratch<32> sc;
+    // the CTA's last row, finished by all warps together
+    RowTotals end_t;
+    int end_row, end_a0, end_b0, end_go;
+    double end_tot[kStepWarps + 1];
+};
+
+// ---------------------------------------------------------------- streaming warps
+struct PieceDesc {
+    const char* src;   // first byte bulk copies fetch
+    int bytes;         // how many (a multiple of 16)
+    int tail;          // ragged logits after them, fetched with plain loads
+    int seg, place;
+    bool live;
+};
+template <int DT>
+__device__ __forceinline__ PieceDesc piece_at(const StepParams& sp, const StepShared& sh, int first_row, int S, int k,
+                                              int warp) {
+    constexpr int kEsize = DT == PSMC_F32 ? 4 : 2;
+    PieceDesc d;
+    d.seg = segment_in_order(k, S);
+    const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + d.seg);
+    d.place = place_of_warp(warp, s.row, sp.g.W);
+    d.live = !sh.seg_done[d.seg];
+    int p0, p1;
+    piece_granules(s, d.place, sp.g.W, p0, p1);
+    const char* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)s.row * sp.ld * kEsize;
+    d.src = rowp + (size_t)p0 * kGranule;
+    const int end = min(p1 * kGranule, sp.g.row_bytes16);
+    d.bytes = max(end - p0 * kGranule, 0);
+    d.tail = (p1 == sp.g.gpr && p1 > p0) ? sp.g.tail : 0;
+    return d;
+}
+
+// The streaming loop of one warp over its pieces; the bulk-copy pipeline of logits_stream.cuh with one triple per
+// piece.  Returns false when a bounded wait ran out (status raised, copies drained, every barrier still arrived on).
+template <int DT, int MODE>
+__device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& sh, float4* local_triples, int first_row,
+                                              int S, int warp, int lane, unsigned char* ring, uint64_t* full) {
+    const PackedConsts kc = packed_consts(sp.f.bf);
+    const int W = sp.g.W;
+
+    // producer cursor (the same in every lane; lane 0 issues)
+    int pk = 0, p_left = 0;
+    const char* p_src = nullptr;
+    auto prod_seek = [&]() {
+        for (; pk < S; ++pk) {
+            const PieceDesc d = piece_at<DT>(sp, sh, first_row, S, pk, warp);
+            if (d.live && d.bytes > 0) {
+                p_src = d.src;
+                p_left = d.bytes;
+                return;
+            }
+        }
+    };
+    int issued = 0;
+    auto issue = [&]() {
+        if (p_left == 0) return;
+        const int bytes = p_left < kStageBytes ? p_left : kStageBytes;
+        if (lane == 0) {
+            const int slot = issued & (kDepth - 1);
+            fence_async_smem();  // the stage's previous contents were read through the generic proxy
+            mbar_expect_tx(&full[slot], (uint32_t)bytes);
+            bulk_load(ring + (size_t)slot * kStageBytes, p_src, (uint32_t)bytes, &full[slot]);
+        }
+        ++issued;
+        p_src += bytes;
+        p_left -= bytes;
+        if (p_left == 0) {
+            ++pk;
+            prod_seek();
+        }
+    };
+    static_assert((kDepth & (kDepth - 1)) == 0, "the ring depth is a power of two");
+
+    prod_seek();
+    for (int d = 0; d < kDepth - 1; ++d) issue();
+
+    bool failed = false;
+    int consumed = 0;
+    for (int ck = 0; ck < S; ++ck) {
+        const PieceDesc d = piece_at<DT>(sp, sh, first_row, S, ck, warp);
+        if (!d.live) continue;  // finished row: no triple, no arrival (the finisher does not wait for it either)
+        LaneSums acc = lane_sums_init();
+        __nv_bfloat162 thr2 = __float2bfloat162_rn(acc.thr);
+        int left = failed ? 0 : d.bytes;
+        while (left > 0) {
+            __syncwarp();  // every lane is done with the stage that is about to be refilled
+            issue();
+            const int slot = consumed & (kDepth - 1);
+            if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // uniform verdict
+                failed = true;
+                break;
+            }
+            const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
+            const int bytes = left < kStageBytes ? left : kStageBytes;
+            const int chunks = bytes >> 4;
+            int c0 = 0;
+            for (; c0 + 128 <= chunks; c0 += 128) {  // 2 KB = four 16-byte chunks per lane at a time
+                const uint4 v0 = st[c0 + lane], v1 = st[c0 + 32 + lane], v2 = st[c0 + 64 + lane], v3 = st[c0 + 96 + lane];
+                const uint32_t w[16] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w,
+                                        v2.x, v2.y, v2.z, v2.w, v3.x, v3.y, v3.z, v3.w};
+                consume<DT, MODE, 16>(w, kc, acc, thr2);
+            }
+            constexpr uint32_t kNoLogit = DT == PSMC_BF16 ? 0xff80ff80u : 0xff800000u;  // -inf: no mass, never a maximum
+            for (; c0 < chunks; c0 += 32) {  // the same trip count in every lane
+                const bool in = c0 + lane < chunks;
+                const uint4 v0 = in ? st[c0 + lane] : make_uint4(kNoLogit, kNoLogit, kNoLogit, kNoLogit);
+                const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+                consume<DT, MODE, 4>(w, kc, acc, thr2);
+            }
+            ++consumed;
+            left -= bytes;
+        }
+        if (failed) {  // a triple without mass: the row gets flagged, the barrier still gets its arrival
+            acc = lane_sums_init();
+        } else if (d.tail > 0) {  // ragged end of the row
+            add_one<MODE>(lane < d.tail ? load_elem<DT>(d.src + d.bytes, lane) : -INFINITY, kc.bf1, kc.slack, acc);
+        }
+        const float s1 = warp_sum(pair_sum(add2(acc.s1a, acc.s1b)));
+        const float sb = (MODE == kBeta1) ? 0.f : warp_sum(pair_sum(add2(acc.sba, acc.sbb)));
+        if (lane == 0) {
+            const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + d.seg);
+            const float4 tr = make_float4(-acc.neg_c, s1, sb, 0.f);
+            if (s.local(sp.g)) local_triples[d.seg * W + d.place] = tr;
+            else __stcg(&sp.shared_triples[((size_t)blockIdx.x * 2 + s.slot) * W + d.place], tr);
+            mbar_arrive(&sh.seg_bars[d.seg]);  // release: the triple is visible to whoever sees the barrier complete
+        }
+    }
+    if (failed) {
+        if (lane == 0) raise_status(sp.a.status, PSMC_E_TIMEOUT);
+        // do not leave with copies still landing in this CTA's shared memory: bounded second wait
+        for (int j = consumed; j < issued; ++j) mbar_wait(&full[j & (kDepth - 1)], (uint32_t)((j / kDepth) & 1));
+    }
+    return !failed;
+}
+
+// ---------------------------------------------------------------- finishing a row
+// Row totals from the triples of a local row (shared memory, W of them) or of a shared row (global memory, W from each
+// CTA that holds a part, in CTA order = vocabulary order).  Every lane gets the same result.
+template <int MODE>
+__device__ __forceinline__ RowTotals row_totals(const StepParams& sp, const float4* local_triples, const Segment& s, int seg,
+                                                int c_first, int c_last, double U, int lane) {
+    const int W = sp.g.W;
+    if (s.local(sp.g)) {
+        const float4* P = local_triples + seg * W;
+        return combine_triples<MODE>([&](int j) { return P[j]; }, W, sp.f.beta, U, lane);
+    }
+    const int row = s.row;
+    return combine_triples<MODE>(
+        [&](int j) {
+            const int c = c_first + j / W, place = j - (j / W) * W;
+            const int slot = (row == share_first(sp.g, c) / sp.g.gpr) ? 0 : 1;
+            return __ldcg(&sp.shared_triples[((size_t)c * 2 + slot) * W + place]);
+        },
+        (c_last - c_first + 1) * W, sp.f.beta, U, lane);
+}
+// the logits the selected triple stands for
+template <int DT>
+__device__ __forceinline__ void selected_range(const StepParams& sp, const Segment& s, int c_first, int jsel, int& a0, int& b0) {
+    const int W = sp.g.W;
+    Segment part = s;
+    int place = jsel;
+    if (!s.local(sp.g)) {
+        part = segment_of_row(sp.g, c_first + jsel / W, s.row);
+        place = jsel % W;
+    }
+    int p0, p1;
+    piece_granules(part, place, W, p0, p1);
+    piece_logits<DT>(sp.g, sp.V, p0, p1, a0, b0);
+}
+
+// The token inside logits [a0, b0) by one warp: every lane sums a contiguous share (whole 16-byte chunks), the lane
+// whose share reaches the target is searched 32 logits at a time.  -1: nothing there has mass.
+template <int DT, int MODE>
+__device__ __forceinline__ int locate_in_range_warp(const FinishParams& p, const void* rowp, const RowTotals& t, int a0, int b0,
+                                                    int lane) {
+    constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
+    const float neg_C = -t.C;
+    const int chunks = (b0 - a0 + kPer - 1) / kPer;
+    const int E = ((chunks + 31) / 32) * kPer;  // logits per lane
+    const double lm = lane_share<DT, MODE, 8>(p, rowp, a0 + lane * E, E, b0, neg_C);
+    const double r_incl = t.base + warp_scan_incl(lm, lane);
+    const unsigned hit = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+    if (hit) {
+        const int owner = __ffs(hit) - 1;
+        const double run = __shfl_sync(kFull, r_incl - lm, owner);
+        const int o0 = a0 + owner * E;
+        return locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+    }
+    return last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);  // the re-read sums fall short of the target
+}
+
+// A row's result goes to memory and its group gets one arrival; the warp that completes the group updates it.
+// Called by all 32 lanes of one warp.  rr == nullptr: the row is finished (absorbing EOS) and has nothing to store.
+__device__ __forceinline__ void row_arrives(const StepParams& sp, StepShared& sh, int row, const RowResult* rr, bool timed_out,
+                                            int lane) {
+    const WeightsArgs& a = sp.a;
+    const int N = a.N, g = row / N;
+    if (rr && lane == 0) {
+        if (timed_out) raise_status(a.status, PSMC_E_TIMEOUT);
+        else if (rr->tok < 0) raise_status(a.status, PSMC_E_NUMERIC);
+        a.tok[row] = rr->tok;
+        a.logp[row] = rr->logp;
+        a.loginc[row] = rr->loginc;
+    }
+    int ticket = 0;
+    if (lane == 0) {
+        __threadfence();  // the row's result first, then the arrival
+        ticket = atomicAdd(&sp.group_arrivals[g], 1);
+    }
+    ticket = __shfl_sync(kFull, ticket, 0);
+    if (ticket != N - 1) return;
+    // the group is complete: this warp updates it
+    if (lane == 0) sp.group_arrivals[g] = 0;
+    __threadfence();
+    int tk = -1;
+    double lp = 0.0, inc = 0.0;
+    ParticleState st{};
+    if (lane < N) {
+        const int r = g * N + lane;
+        st = load_particle(a, r);
+        if (!st.done) {
+            tk = __ldcg(const_cast<const int32_t*>(a.tok) + r);
+            lp = __ldcg(const_cast<const double*>(a.logp) + r);
+            inc = __ldcg(const_cast<const double*>(a.loginc) + r);
+        }
+    }
+    group_update(a, g, lane, 1, sh.sc, tk, lp, inc, st);
+    __syncwarp();  // sh.sc is reused by the next group this CTA closes
+}
+
+// Waits for the streaming warps of this CTA to have delivered segment `seg`; for a shared row also takes the CTA's
+// ticket.  Returns true when this CTA is the one to finish the row.  Every lane gets the same answer.
+__device__ __forceinline__ bool segment_complete(const StepParams& sp, StepShared& sh, const Segment& s, int seg, int c_first,
+                                                 int c_last, bool& timed_out, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(&sh.seg_bars[seg], 0) ? 1 : 0;
+    ok = __shfl_sync(kFull, ok, 0);
+    if (!ok) timed_out = true;
+    if (s.local(sp.g)) return true;
+    int last = 0;
+    if (lane == 0) {
+        __threadfence();  // this CTA's triples first, then its ticket
+        const int ticket = atomicAdd(&sp.row_arrivals[s.row], 1);
+        last = ticket == c_last - c_first ? 1 : 0;
+        if (last) {
+            sp.row_arrivals[s.row] = 0;  // every part has arrived: ready for the next launch
+            __threadfence();             // the other CTAs' triples are visible from here on
+        }
+    }
+    return __shfl_sync(kFull, last, 0) != 0;
+}
 
 template <int DT, int MODE>
-__device__ __forceinline__ void finishing_warp(const FusedParams& fp, int fin_id, int n_fin, int lane, GroupScratch<32>& sc) {
-    const WeightsArgs& a = fp.a;
+__device__ __noinline__ void finisher_warp(const StepParams& sp, StepShared& sh, const float4* local_triples, int first_row,
+                                              int S, int lane) {
+    const WeightsArgs& a = sp.a;
     const int N = a.N;
-    for (int row = fin_id; row < a.R; row += n_fin) {
-        const int g = row / N, k = row - g * N;
-        if (!a.done[row]) {
-            int ok = 1;
-            if (lane == 0) {
-                uint32_t polls = 0;
-                while (load_volatile(&fp.row_arrivals[row]) < fp.s.n_spans) {
-                    if (++polls > kPollLimit) {
-                        ok = 0;
-                        break;
-                    }
-                    __nanosleep(256);
+    // every segment but the last one in order is finished by this warp alone, while the sweep goes on
+    for (int k = 0; k < S; ++k) {
+        const bool at_end = k == S - 1;
+        const int seg = segment_in_order(k, S);
+        const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + seg);
+        const int row = s.row, g = row / N;
+        if (at_end && lane == 0) sh.end_go = 0;
+        if (sh.seg_done[seg]) {
+            // a finished row is reported to its group by the CTA that holds the row's last granule
+            if (s.g1 == sp.g.gpr) row_arrives(sp, sh, row, nullptr, false, lane);
+            continue;
+        }
+        const int c_first = share_of(sp.g, row * sp.g.gpr), c_last = share_of(sp.g, (row + 1) * sp.g.gpr - 1);
+        bool timed_out = false;
+        if (!segment_complete(sp, sh, s, seg, c_first, c_last, timed_out, lane)) continue;
+        RowResult rr{-1, 0.0, 0.0};
+        RowTotals t;
+        t.ok = false;
+        if (!timed_out) {
+            const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)(row - g * N)));
+            t = row_totals<MODE>(sp, local_triples, s, seg, c_first, c_last, U, lane);
+        }
+        if (t.ok) {
+            int a0, b0;
+            selected_range<DT>(sp, s, c_first, t.jsel, a0, b0);
+            if (at_end) {  // hand the row to the whole CTA
+                if (lane == 0) {
+                    sh.end_t = t;
+                    sh.end_row = row;
+                    sh.end_a0 = a0;
+                    sh.end_b0 = b0;
+                    sh.end_go = 1;
                 }
-                if (ok) fp.row_arrivals[row] = 0;  // every producer of this row has arrived: ready for the next launch
+                return;
             }
-            ok = __shfl_sync(kFull, ok, 0);
-            __threadfence();  // the triples counted above are visible from here on
-            RowResult rr{-1, 0.0, 0.0};
-            if (ok) {
-                const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)k));
-                rr = finish_row_warp<DT, MODE>(fp.f, row, U, lane);
-            }
-            if (lane == 0) {
-                if (!ok) raise_status(a.status, PSMC_E_TIMEOUT);
-                else if (rr.tok < 0) raise_status(a.status, PSMC_E_NUMERIC);
-                a.tok[row] = rr.tok;
-                a.logp[row] = rr.logp;
-                a.loginc[row] = rr.loginc;
-                __threadfence();
-            }
+            const void* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * (DT == PSMC_F32 ? 4 : 2);
+            const int y = locate_in_range_warp<DT, MODE>(sp.f, rowp, t, a0, b0, lane);
+            if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
         }
-        int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&fp.group_arrivals[g], 1);
-        ticket = __shfl_sync(kFull, ticket, 0);
-        if (ticket == N - 1) {  // the group is complete: this warp updates it
-            if (lane == 0) fp.group_arrivals[g] = 0;
-            __threadfence();
-            int tk = -1;
-            double lp = 0.0, inc = 0.0;
-            ParticleState st{};
-            if (lane < N) {
-                const int r = g * N + lane;
-                st = load_particle(a, r);
-                tk = __ldcg(const_cast<const int32_t*>(a.tok) + r);
-                lp = __ldcg(const_cast<const double*>(a.logp) + r);
-                inc = __ldcg(const_cast<const double*>(a.loginc) + r);
-            }
-            group_update(a, g, lane, 1, sc, tk, lp, inc, st);
-            __syncwarp();  // sc is reused by the next group this warp closes
-        }
+        row_arrives(sp, sh, row, &rr, timed_out, lane);
+    }
+}
+
+// The CTA's last row by all of its warps: one contiguous run of 16-byte chunks per thread (one chunk each when the
+// piece has no more chunks than the CTA has threads), the warp whose threads reach the target names the token.
+// Every thread of the CTA calls this.
+template <int DT, int MODE>
+__device__ __noinline__ void finish_last_row(const StepParams& sp, StepShared& sh) {
+    constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const RowTotals t = sh.end_t;
+    const int row = sh.end_row, a0 = sh.end_a0, b0 = sh.end_b0;
+    const void* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * (DT == PSMC_F32 ? 4 : 2);
+    const float neg_C = -t.C;
+    const int chunks = (b0 - a0 + kPer - 1) / kPer;
+    const int E = ((chunks + (int)blockDim.x - 1) / (int)blockDim.x) * kPer;  // logits per thread
+    const int e0 = a0 + (int)threadIdx.x * E;
+    const double lm = lane_share<DT, MODE, 4>(sp.f, rowp, e0, E, b0, neg_C);
+    const double incl = warp_scan_incl(lm, lane);
+    if (lane == 31) sh.end_tot[warp] = incl;
+    __syncthreads();
+    // which warp's threads reach the target: the same additions, in the same order, in every warp
+    double cum = t.base, before = t.base;
+    int first_hit = -1;
+    for (int i = 0; i < n_warps; ++i) {
+        if (i == warp) before = cum;
+        const double ti = sh.end_tot[i];
+        cum += ti;
+        if (first_hit < 0 && ti > 0.0 && cum >= t.target) first_hit = i;
+    }
+    int y = -1;
+    bool mine = false;
+    if (first_hit == warp) {
+        mine = true;
+        const double r_incl = before + incl;
+        const unsigned hit = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+        const int owner = hit ? __ffs(hit) - 1 : 31;
+        const double run = __shfl_sync(kFull, r_incl - lm, owner);
+        const int o0 = a0 + (warp * 32 + owner) * E;
+        y = locate_in_lane<DT, MODE>(sp.f, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+    } else if (first_hit < 0 && warp == 0) {
+        mine = true;  // the re-read sums fall short of the target: last token with mass in the piece
+        y = last_with_mass<DT, MODE>(sp.f, rowp, a0, b0, neg_C, lane);
+    }
+    if (mine) {
+        RowResult rr{-1, 0.0, 0.0};
+        if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
+        row_arrives(sp, sh, row, &rr, false, lane);
     }
 }
 
 template <int DT, int MODE>
-__global__ void __launch_bounds__((kStreamers + kFinishers) * 32, 1) psmc_step_kernel(const __grid_constant__ FusedParams fp) {
+__global__ void __launch_bounds__((kStepWarps + 1) * 32, 1) psmc_step_kernel(const __grid_constant__ StepParams sp) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[kStreamers * kDepth];
-    __shared__ GroupScratch<32> sc[kFinishers];
+    __shared__ StepShared sh;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_stream = (blockDim.x >> 5) - kFinishers;  // streaming warps of this CTA
-    if (warp < n_stream) {
-        const StreamParams& p = fp.s;
-        const int warp_global = blockIdx.x * n_stream + warp;
-        const int n_warps = gridDim.x * n_stream;
-        const int n_tasks = p.R * p.n_spans;  // < 2^31, checked by the host
-        stream_init_barriers(bars + warp * kDepth, lane);
-        chain_begin();  // everything above is local set-up; global memory from here on
-        if (p.zero_words && blockIdx.x == 0 && threadIdx.x < 2) p.zero_words[threadIdx.x] = 0;
-        stream_tasks<DT, MODE>(p, smem + (size_t)warp * kDepth * kStageBytes, bars + warp * kDepth, lane,
-                               min(n_tasks, warp_global * kRun), n_tasks, kRun, (n_warps - 1) * kRun, [&](int row) {
-                                   if (lane == 0) {
-                                       __threadfence();  // the triple first, then the arrival
-                                       atomicAdd(&fp.row_arrivals[row], 1);
-                                   }
-                               });
+    const int W = sp.g.W;
+    float4* local_triples = reinterpret_cast<float4*>(smem + (size_t)W * kDepth * kStageBytes);
+    const int first = share_first(sp.g, (int)blockIdx.x), count = share_count(sp.g, (int)blockIdx.x);
+    const int first_row = first / sp.g.gpr;
+    const int S = (first + count - 1) / sp.g.gpr - first_row + 1;  // <= sp.g.seg_cap, checked by the host
+
+    if (warp < W) stream_init_barriers(sh.ring_bars + warp * kDepth, lane);
+    if ((int)threadIdx.x < S) mbar_init(&sh.seg_bars[threadIdx.x], (uint32_t)W);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    chain_begin();  // everything above is local set-up; global memory from here on
+    if (sp.zero_words && blockIdx.x == 0 && threadIdx.x < 2) sp.zero_words[threadIdx.x] = 0;
+    if ((int)threadIdx.x < S) sh.seg_done[threadIdx.x] = sp.a.done[first_row + threadIdx.x];
+    __syncthreads();
+
+    if (warp < W) {
+        stream_pieces<DT, MODE>(sp, sh, local_triples, first_row, S, warp, lane, smem + (size_t)warp * kDepth * kStageBytes,
+                                sh.ring_bars + warp * kDepth);
     } else {
-        chain_begin();
-        finishing_warp<DT, MODE>(fp, blockIdx.x * kFinishers + (warp - n_stream), gridDim.x * kFinishers, lane,
-                                 sc[warp - n_stream]);
+        finisher_warp<DT, MODE>(sp, sh, local_triples, first_row, S, lane);
     }
+    __syncthreads();  // the sweep is over; the finisher has left the CTA's last row (if it is this CTA's to finish) in sh
+    if (sh.end_go) finish_last_row<DT, MODE>(sp, sh);
 }
 
-typedef void (*FusedFn)(const FusedParams);
+typedef void (*StepFn)(const StepParams);
 template <int DT>
-FusedFn pick_fused(int mode) {
+StepFn pick_step(int mode) {
     switch (mode) {
         case kBeta1: return psmc_step_kernel<DT, kBeta1>;
         case kBeta2: return psmc_step_kernel<DT, kBeta2>;
@@ -137,46 +509,60 @@ FusedFn pick_fused(int mode) {
     }
 }
 
-}  // namespace
-
-// Measured on B200: with logit blocks of a few MB the step is bound by launch and dependency latency and one launch
-// beats two (20-22 us against 26-28 us for 8 x 32000 and 16 x 151936 bf16 logits); from about 10 MB on, the tail of
-// one-warp row finishes after the sweep costs more than the second kernel's 32 warps per group (58 us against 44 us
-// for 512 x 128256).
-bool step_can_fuse(const LogitsStreamArgs& la, int N) {
-    const LogitsGeometry g = logits_geometry(la.logits, la.dt, la.R, la.V, la.ld, la.beta);
-    const int64_t bytes = (int64_t)la.R * la.V * (la.dt == PSMC_F32 ? 4 : 2);
-    return N <= 32 && g.vec != 0 && bytes <= kFuseMaxBytes;
+// false: the shape does not fit the one-kernel step
+bool step_geometry(int R, int V, int dt, StepGeom& g, int& grid) {
+    const int esize = dt == PSMC_F32 ? 4 : 2, per16 = 16 / esize;
+    const int64_t row_bytes16 = (int64_t)(V / per16) * 16;
+    const int64_t gpr = row_bytes16 > 0 ? (row_bytes16 + kGranule - 1) / kGranule : 1;
+    const int64_t total = (int64_t)R * gpr;
+    if (total >= (int64_t)1 << 30) return false;
+    grid = (int)(total < kSMs ? total : kSMs);
+    g.gpr = (int)gpr;
+    g.base = (int)(total / grid);
+    g.extra = (int)(total % grid);
+    g.row_bytes16 = (int)row_bytes16;
+    g.tail = V % per16;
+    const int per_cta = g.base + (g.extra ? 1 : 0);
+    int W = (per_cta + kMinGranulesPerWarp - 1) / kMinGranulesPerWarp;
+    g.W = W < 1 ? 1 : (W > kStepWarps ? kStepWarps : W);
+    g.seg_cap = (int)((per_cta + gpr - 2) / gpr + 1);
+    return g.seg_cap <= kMaxSegments;
 }
 
-cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, int32_t* row_arrivals,
-                              int32_t* group_arrivals, cudaStream_t stream) {
-    const LogitsGeometry g = logits_geometry(la.logits, la.dt, la.R, la.V, la.ld, la.beta);
-    const int64_t n_tasks = (int64_t)la.R * g.n_spans;
-    if (n_tasks >= (int64_t)1 << 31) return cudaErrorInvalidValue;
-    FusedParams fp;
-    fp.s.logits = la.logits; fp.s.R = la.R; fp.s.V = la.V; fp.s.ld = la.ld; fp.s.span = g.span; fp.s.n_spans = g.n_spans;
-    fp.s.bf = g.bf; fp.s.done = la.done; fp.s.partials = reinterpret_cast<float4*>(la.scratch);
-    fp.s.zero_words = la.zero_words; fp.s.status = la.status;
-    fp.f.logits = la.logits; fp.f.V = la.V; fp.f.ld = la.ld; fp.f.span = g.span; fp.f.n_spans = g.n_spans;
-    fp.f.partials = reinterpret_cast<const float4*>(la.scratch); fp.f.beta = wa.beta; fp.f.alpha_t = wa.alpha_t;
-    fp.f.bf = g.bf; fp.f.vec = g.vec;
-    fp.a = wa;
-    fp.row_arrivals = row_arrivals;
-    fp.group_arrivals = group_arrivals;
+}  // namespace
 
-    // one CTA per SM; as many streaming warps per CTA as it takes to give every run of spans a warp, up to kStreamers
-    const int64_t units = (n_tasks + kRun - 1) / kRun;
-    int64_t warps = (units + kSMs - 1) / kSMs;
-    if (warps > kStreamers) warps = kStreamers;
-    if (warps < 1) warps = 1;
-    int64_t blocks = (units + warps - 1) / warps;
-    if (blocks > kSMs) blocks = kSMs;
-    const size_t smem = (size_t)warps * kDepth * kStageBytes;
-    FusedFn fn = la.dt == PSMC_F32 ? pick_fused<PSMC_F32>(g.mode) : pick_fused<PSMC_BF16>(g.mode);
-    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn), kStreamers * kDepth * kStageBytes);
+size_t step_fused_scratch_bytes() { return (size_t)kSMs * 2 * kStepWarps * sizeof(float4); }
+
+// The one-kernel step needs groups that one warp can update (N <= 32), rows that bulk copies can fetch (16-byte
+// aligned starts) and a share per CTA that meets at most kMaxSegments rows.  Everything else takes the step as two
+// kernels (logits_pass.cu, weights_resample.cu).
+bool step_can_fuse(const LogitsStreamArgs& la, int N) {
+    const LogitsGeometry lg = logits_geometry(la.logits, la.dt, la.R, la.V, la.ld, la.beta);
+    StepGeom g;
+    int grid;
+    return N <= 32 && lg.vec != 0 && step_geometry(la.R, la.V, la.dt, g, grid);
+}
+
+cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, void* shared_triples,
+                              int32_t* row_arrivals, int32_t* group_arrivals, cudaStream_t stream) {
+    const LogitsGeometry lg = logits_geometry(la.logits, la.dt, la.R, la.V, la.ld, la.beta);
+    StepParams sp;
+    int grid;
+    if (!step_geometry(la.R, la.V, la.dt, sp.g, grid)) return cudaErrorInvalidValue;
+    sp.logits = la.logits; sp.R = la.R; sp.V = la.V; sp.ld = la.ld;
+    sp.f.logits = la.logits; sp.f.V = la.V; sp.f.ld = la.ld; sp.f.span = 0; sp.f.n_spans = 0; sp.f.partials = nullptr;
+    sp.f.beta = wa.beta; sp.f.alpha_t = wa.alpha_t; sp.f.bf = lg.bf; sp.f.vec = lg.vec;
+    sp.a = wa;
+    sp.shared_triples = reinterpret_cast<float4*>(shared_triples);
+    sp.row_arrivals = row_arrivals;
+    sp.group_arrivals = group_arrivals;
+    sp.zero_words = la.zero_words;
+    const size_t smem = (size_t)sp.g.W * kDepth * kStageBytes + (size_t)sp.g.seg_cap * sp.g.W * sizeof(float4);
+    StepFn fn = la.dt == PSMC_F32 ? pick_step<PSMC_F32>(lg.mode) : pick_step<PSMC_BF16>(lg.mode);
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn),
+                                       kStepWarps * kDepth * kStageBytes + kMaxSegments * kStepWarps * (int)sizeof(float4));
     if (e != cudaSuccess) return e;
-    return launch_chained(fn, dim3((unsigned)blocks), dim3((unsigned)((warps + kFinishers) * 32)), smem, stream, fp);
+    return launch_chained(fn, dim3((unsigned)grid), dim3((unsigned)((sp.g.W + 1) * 32)), smem, stream, sp);
 }
 
 }  // namespace psmc

@@ -103,7 +103,7 @@ __device__ __forceinline__ void group_update(const WeightsArgs& a, int g, int i,
         if (on) {
             a.logW[r] = lw;
             a.S[r] = S;
-            a.done[r] = dn;
+            a.done_out[r] = dn;
             a.len[r] = ln;
             a.anc[r] = i;
             a.map[r] = i;
@@ -212,7 +212,7 @@ __device__ __forceinline__ void group_update(const WeightsArgs& a, int g, int i,
     if (on) {
         a.logW[r] = 0.0;
         a.S[r] = sc.S[mp];
-        a.done[r] = sc.done[mp];
+        a.done_out[r] = sc.done[mp];
         a.len[r] = sc.len[mp];
         a.anc[r] = anc;
         a.map[r] = mp;
