@@ -35,6 +35,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// The same for a warp that expects to wait long while others work: a failed try comes back at once, so polling flat
+// out would take issue slots from the warps that have work to do; a short sleep between tries costs at most that much
+// wake-up delay.  (A try with a suspend-time hint was measured to sleep for the whole hint.)
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t* bar, uint32_t parity) {
+    for (uint32_t k = 0; k < kWaitTries; ++k) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(100);
+    }
+    return false;
+}
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                      smem_u32(smem_dst)),

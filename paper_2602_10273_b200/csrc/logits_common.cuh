@@ -104,16 +104,20 @@ struct RowTotals {
     int jsel;       // span that holds the target
 };
 
+// 2^e for a whole number e <= 0, exactly, built from its bits; 0 below the normal range (such a term is less than
+// 2^-1022 of the row's largest and cannot change any sum)
+__device__ __forceinline__ double pow2_neg(int e) { return e >= -1022 ? __hiloint2double((1023 + e) << 20, 0) : 0.0; }
+
 // 2^{dc} and 2^{beta dc} for a span whose reference exponent lies dc <= 0 below the row's.  dc is a whole number,
-// so for whole beta both factors are exact powers of two (ldexp); other beta take one fp64 exp2.
+// so for whole beta both factors are exact powers of two; other beta take one fp64 exp2.
 template <int MODE>
 __device__ __forceinline__ void span_scales(float dcf, double beta, double& f1, double& fb) {
-    const int dc = (int)fmaxf(dcf, -4000.f);  // below -2100 or so every factor is 0 anyway
-    f1 = ldexp(1.0, dc);
+    const int dc = (int)fmaxf(dcf, -4000.f);  // below -1022 every factor is 0
+    f1 = pow2_neg(dc);
     if (MODE == kBeta1) fb = f1;
-    else if (MODE == kBeta2) fb = ldexp(1.0, 2 * dc);
-    else if (MODE == kBeta4) fb = ldexp(1.0, 4 * dc);
-    else if (MODE == kBeta8) fb = ldexp(1.0, 8 * dc);
+    else if (MODE == kBeta2) fb = pow2_neg(2 * dc);
+    else if (MODE == kBeta4) fb = pow2_neg(4 * dc);
+    else if (MODE == kBeta8) fb = pow2_neg(8 * dc);
     else fb = exp2(beta * (double)dc);
 }
 
@@ -206,6 +210,33 @@ __device__ __forceinline__ RowTotals combine_triples(Fetch fetch, int n, double 
     if (jsel < 0) return t;
     t.jsel = jsel;
     t.base = base;
+    t.ok = true;
+    return t;
+}
+
+// The same for up to 32 triples, one per lane, in straight-line code: lane j passes triple j (lanes from n on pass
+// any triple with zero sums).  The same additions in the same order as combine_triples.
+template <int MODE>
+__device__ __forceinline__ RowTotals combine_triples_32(float4 f, double beta, double U, int lane) {
+    RowTotals t;
+    t.ok = false;
+    const float cf = warp_max(f.x);
+    t.C = cf;
+    double f1, fb;
+    span_scales<MODE>(f.x - cf, beta, f1, fb);
+    const double a = (double)f.y * f1;
+    const double b = (MODE == kBeta1) ? a : (double)f.z * fb;
+    t.S1 = warp_sum(a);
+    t.Sb = warp_sum(b);
+    if (!(t.S1 > 0.0) || !(t.Sb > 0.0) || isinf(t.S1) || isinf(t.Sb)) return t;
+    t.target = U * t.Sb;
+    const double incl = warp_scan_incl(b, lane);
+    const unsigned hit = __ballot_sync(kFull, b > 0.0 && incl >= t.target);
+    const unsigned pos = __ballot_sync(kFull, b > 0.0);
+    if (!pos) return t;
+    const int src = hit ? __ffs(hit) - 1 : 31 - __clz(pos);  // the last span with mass if rounding leaves every prefix short
+    t.jsel = src;
+    t.base = __shfl_sync(kFull, incl - b, src);
     t.ok = true;
     return t;
 }

@@ -12,15 +12,17 @@
 // The shared parts are taken first, then the whole rows one after the other, so rows complete one after the other
 // while the sweep is still running.
 //
-// Who finishes a row.  One extra warp per CTA, the finisher, follows the segments in the same order.  It waits on a
-// shared-memory mbarrier that the streaming warps of ITS OWN CTA arrive on (so every wait is for warps that are
-// resident by construction), then: a local row it finishes at once from the triples in shared memory; for a shared
-// row it takes a ticket on the row's global counter and the CTA that draws the last ticket finishes the row from
-// the triples in global memory.  No CTA ever waits for another one.  Finishing = totals in fp64, the piece that
-// holds U * sum, a re-read of that piece (it is a few KB and still in L2), the token, log p(y) and log omega
-// (logits_common.cuh).  A finished row counts one arrival for its group, and the warp that brings a group to N
-// arrivals runs the group's update (weights_core.cuh) on the spot.  Only the last row of each CTA is finished after
-// the sweep has ended, and that one by all warps of the CTA together (one 16-byte chunk of the piece per thread).
+// Who finishes a row, and when.  Dependent trips to memory take several times longer while the sweep saturates HBM
+// than after it, so no row is finished during the sweep; what happens during the sweep is only what must happen
+// between CTAs.  One extra warp per CTA, the helper, waits on a shared-memory mbarrier that the streaming warps of
+// ITS OWN CTA arrive on (every wait is for warps that are resident by construction) until the CTA's part of a shared
+// row is complete, then takes a ticket on the row's global counter: the CTA that draws the last ticket owns the row.
+// No CTA ever waits for another one.  After the sweep all warps of the CTA finish the rows it owns (its local rows
+// and the shared rows it drew the last ticket for) together, a team of up to eight warps per row: totals in fp64 from
+// the triples (shared memory, or global memory for a shared row), the piece that holds U * sum, a re-read of that
+// piece split over the team (a few KB, still in L2), the token, log p(y) and log omega (logits_common.cuh).  A
+// finished row counts one arrival for its group, and the warp that brings a group to N arrivals runs the group's
+// update (weights_core.cuh) on the spot.
 //
 // The finished flags are read from one array and written to another (they alternate from step to step): a group may
 // close, and rewrite its flags, while other CTAs have not looked at the flags of their rows yet.  Arrival counters
@@ -39,6 +41,7 @@ constexpr int kGranule = 512;      // bytes: one 16-byte chunk per lane
 constexpr int kStepWarps = 23;     // streaming warps per CTA at most (with the finisher: 6 warps per scheduler, 80 registers)
 constexpr int kMaxSegments = 48;   // rows one CTA's share may meet (shapes beyond that take the two-kernel step)
 constexpr int kMinGranulesPerWarp = 4;
+static_assert(kStepWarps % 4 == 3, "the helper completes the last scheduler's set of warps");
 
 // How a block is cut up; a pure function of (R, V, dtype), the same on host and device.
 struct StepGeom {
@@ -92,13 +95,23 @@ __device__ __forceinline__ int segment_in_order(int k, int S) {
     if (S < 2) return 0;
     return k == 0 ? S - 1 : k - 1;
 }
-// A segment's granules are dealt to the W streaming warps in vocabulary order, `place` 0 first; which warp takes which
-// place rotates with the row so that the spare granules do not always fall to the same warps.
-__device__ __forceinline__ int place_of_warp(int warp, int row, int W) { return (warp + row) % W; }
+// A segment's granules are dealt to the W streaming warps in vocabulary order, warp 0 first, in proportion to the
+// warps' weights.  A full CTA has 23 streaming warps and the helper: the scheduler that hosts the helper (warp 23,
+// hence warps 3, 7, ... too) runs five streaming warps where the other three run six, the helper is parked on a
+// barrier for nearly all of the sweep, and the sweep is close to what a scheduler can issue.  Measured on B200: with
+// equal pieces those five warps end 3 us before the others, with 6/5 of a plain piece each 1 us after them, so they
+// take 7/6.  Smaller CTAs deal evenly.
+constexpr unsigned kFullWeight = 6 * kStepWarps + kStepWarps / 4;  // 18 warps of weight 6, 5 of weight 7
+__device__ __forceinline__ unsigned weight_before(int place) { return 6u * (unsigned)place + (unsigned)place / 4u; }
 __device__ __forceinline__ void piece_granules(const Segment& s, int place, int W, int& p0, int& p1) {
-    const int n = s.g1 - s.g0, base = n / W, extra = n % W;
-    p0 = s.g0 + place * base + min(place, extra);
-    p1 = p0 + base + (place < extra ? 1 : 0);
+    const unsigned n = (unsigned)(s.g1 - s.g0);  // n * kFullWeight < 2^32, checked by the host
+    if (W == kStepWarps) {  // division by a constant
+        p0 = s.g0 + (int)(n * weight_before(place) / kFullWeight);
+        p1 = s.g0 + (int)(n * weight_before(place + 1) / kFullWeight);
+    } else {
+        p0 = s.g0 + (int)(n * (unsigned)place / (unsigned)W);
+        p1 = s.g0 + (int)(n * (unsigned)(place + 1) / (unsigned)W);
+    }
 }
 // logits [a0, b0) of the row that a piece covers (the piece that holds a row's last granule also owns the ragged end)
 template <int DT>
@@ -109,19 +122,38 @@ __device__ __forceinline__ void piece_logits(const StepGeom& g, int V, int p0, i
     if (p1 <= p0) b0 = a0;
 }
 
+// One arrival on a global counter.  Release: what this thread wrote, and what it has observed of other threads' writes,
+// is visible to whoever reads the new count; acquire: the writes of the earlier arrivals are visible to this thread
+// (and, after a warp barrier, to its warp) once it holds the returned count.
+__device__ __forceinline__ int arrive_acq_rel(int32_t* counter) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+    return old;
+}
+// Named CTA barriers 1..15 as producer/consumer signals: the streaming warps arrive (and run on), the helper waits.
+// The hardware parks the waiting warp, so it takes no issue slots while it waits and resumes with the last arrival.
+constexpr int kNamedBarriers = 15;
+__device__ __forceinline__ void named_arrive(int id, int threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 struct StepShared {
     uint64_t ring_bars[kStepWarps * kDepth];
-    uint64_t seg_bars[kMaxSegments];     // one per segment: all streaming warps have stored their triple
+    uint64_t seg_bars[kMaxSegments];       // one per segment: all streaming warps have stored their triple
     unsigned char seg_done[kMaxSegments];  // the segment's row is finished (absorbing EOS): nothing is read or summed
-    GroupScratch<32> sc;
-    // the CTA's last row, finished by all warps together
-    RowTotals end_t;
-    int end_row, end_a0, end_b0, end_go;
-    double end_tot[kStepWarps + 1];
+    double seg_u[kMaxSegments];            // the uniform of the segment's row (token stream of the counter hash)
+    GroupScratch<32> sc;                   // the helper's; a streaming warp that closes a group uses its idle ring
+    // rows this CTA finishes after the sweep, listed by the helper with their totals and the piece to re-read
+    int n_pend, timed_out;
+    RowTotals pend_t[kMaxSegments];
+    int pend_row[kMaxSegments], pend_a0[kMaxSegments], pend_b0[kMaxSegments];
+    double end_tot[kStepWarps + 1];        // per warp: mass of its part of the selected piece
 };
 
 // ---------------------------------------------------------------- streaming warps
@@ -139,7 +171,7 @@ __device__ __forceinline__ PieceDesc piece_at(const StepParams& sp, const StepSh
     PieceDesc d;
     d.seg = segment_in_order(k, S);
     const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + d.seg);
-    d.place = place_of_warp(warp, s.row, sp.g.W);
+    d.place = warp;
     d.live = !sh.seg_done[d.seg];
     int p0, p1;
     piece_granules(s, d.place, sp.g.W, p0, p1);
@@ -233,6 +265,7 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
         }
         if (failed) {  // a triple without mass: the row gets flagged, the barrier still gets its arrival
             acc = lane_sums_init();
+            if (lane == 0) sh.timed_out = 1;
         } else if (d.tail > 0) {  // ragged end of the row
             add_one<MODE>(lane < d.tail ? load_elem<DT>(d.src + d.bytes, lane) : -INFINITY, kc.bf1, kc.slack, acc);
         }
@@ -243,8 +276,10 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
             const float4 tr = make_float4(-acc.neg_c, s1, sb, 0.f);
             if (s.local(sp.g)) local_triples[d.seg * W + d.place] = tr;
             else __stcg(&sp.shared_triples[((size_t)blockIdx.x * 2 + s.slot) * W + d.place], tr);
-            mbar_arrive(&sh.seg_bars[d.seg]);  // release: the triple is visible to whoever sees the barrier complete
+            // release: the triple is visible to whoever sees the barrier complete
+            if (S > kNamedBarriers) mbar_arrive(&sh.seg_bars[d.seg]);
         }
+        if (S <= kNamedBarriers) named_arrive(1 + ck, (W + 1) * 32);  // the triple is stored: tell the helper, do not wait
     }
     if (failed) {
         if (lane == 0) raise_status(sp.a.status, PSMC_E_TIMEOUT);
@@ -261,9 +296,9 @@ template <int MODE>
 __device__ __forceinline__ RowTotals row_totals(const StepParams& sp, const float4* local_triples, const Segment& s, int seg,
                                                 int c_first, int c_last, double U, int lane) {
     const int W = sp.g.W;
-    if (s.local(sp.g)) {
-        const float4* P = local_triples + seg * W;
-        return combine_triples<MODE>([&](int j) { return P[j]; }, W, sp.f.beta, U, lane);
+    if (s.local(sp.g)) {  // at most kStepWarps <= 32 triples: one per lane
+        const float4 f = lane < W ? local_triples[seg * W + lane] : make_float4(kRefFloor, 0.f, 0.f, 0.f);
+        return combine_triples_32<MODE>(f, sp.f.beta, U, lane);
     }
     const int row = s.row;
     return combine_triples<MODE>(
@@ -289,31 +324,10 @@ __device__ __forceinline__ void selected_range(const StepParams& sp, const Segme
     piece_logits<DT>(sp.g, sp.V, p0, p1, a0, b0);
 }
 
-// The token inside logits [a0, b0) by one warp: every lane sums a contiguous share (whole 16-byte chunks), the lane
-// whose share reaches the target is searched 32 logits at a time.  -1: nothing there has mass.
-template <int DT, int MODE>
-__device__ __forceinline__ int locate_in_range_warp(const FinishParams& p, const void* rowp, const RowTotals& t, int a0, int b0,
-                                                    int lane) {
-    constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
-    const float neg_C = -t.C;
-    const int chunks = (b0 - a0 + kPer - 1) / kPer;
-    const int E = ((chunks + 31) / 32) * kPer;  // logits per lane
-    const double lm = lane_share<DT, MODE, 8>(p, rowp, a0 + lane * E, E, b0, neg_C);
-    const double r_incl = t.base + warp_scan_incl(lm, lane);
-    const unsigned hit = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
-    if (hit) {
-        const int owner = __ffs(hit) - 1;
-        const double run = __shfl_sync(kFull, r_incl - lm, owner);
-        const int o0 = a0 + owner * E;
-        return locate_in_lane<DT, MODE>(p, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
-    }
-    return last_with_mass<DT, MODE>(p, rowp, a0, b0, neg_C, lane);  // the re-read sums fall short of the target
-}
-
 // A row's result goes to memory and its group gets one arrival; the warp that completes the group updates it.
 // Called by all 32 lanes of one warp.  rr == nullptr: the row is finished (absorbing EOS) and has nothing to store.
-__device__ __forceinline__ void row_arrives(const StepParams& sp, StepShared& sh, int row, const RowResult* rr, bool timed_out,
-                                            int lane) {
+__device__ __forceinline__ void row_arrives(const StepParams& sp, StepShared& sh, GroupScratch<32>& sc, int row,
+                                            const RowResult* rr, bool timed_out, int lane) {
     const WeightsArgs& a = sp.a;
     const int N = a.N, g = row / N;
     if (rr && lane == 0) {
@@ -323,147 +337,166 @@ __device__ __forceinline__ void row_arrives(const StepParams& sp, StepShared& sh
         a.logp[row] = rr->logp;
         a.loginc[row] = rr->loginc;
     }
+    // The group's state as the step found it (nobody writes it before the group is complete) is asked for now: should
+    // this warp turn out to be the one that completes the group, the loads have overlapped the trip of the ticket.
+    ParticleState st{};
+    if (lane < N) st = load_particle(a, g * N + lane);
     int ticket = 0;
-    if (lane == 0) {
-        __threadfence();  // the row's result first, then the arrival
-        ticket = atomicAdd(&sp.group_arrivals[g], 1);
-    }
+    if (lane == 0) ticket = arrive_acq_rel(&sp.group_arrivals[g]);  // the row's result first, then the arrival
     ticket = __shfl_sync(kFull, ticket, 0);
     if (ticket != N - 1) return;
     // the group is complete: this warp updates it
     if (lane == 0) sp.group_arrivals[g] = 0;
-    __threadfence();
+    __syncwarp();
     int tk = -1;
     double lp = 0.0, inc = 0.0;
-    ParticleState st{};
-    if (lane < N) {
+    if (lane < N) {  // one trip to memory for the rows' results (what a finished row has there is not used)
         const int r = g * N + lane;
-        st = load_particle(a, r);
-        if (!st.done) {
-            tk = __ldcg(const_cast<const int32_t*>(a.tok) + r);
-            lp = __ldcg(const_cast<const double*>(a.logp) + r);
-            inc = __ldcg(const_cast<const double*>(a.loginc) + r);
-        }
+        tk = __ldcg(const_cast<const int32_t*>(a.tok) + r);
+        lp = __ldcg(const_cast<const double*>(a.logp) + r);
+        inc = __ldcg(const_cast<const double*>(a.loginc) + r);
     }
-    group_update(a, g, lane, 1, sh.sc, tk, lp, inc, st);
-    __syncwarp();  // sh.sc is reused by the next group this CTA closes
+    group_update(a, g, lane, 1, sc, tk, lp, inc, st);
+    __syncwarp();  // sc is reused by the next group this warp closes
 }
 
-// Waits for the streaming warps of this CTA to have delivered segment `seg`; for a shared row also takes the CTA's
-// ticket.  Returns true when this CTA is the one to finish the row.  Every lane gets the same answer.
-__device__ __forceinline__ bool segment_complete(const StepParams& sp, StepShared& sh, const Segment& s, int seg, int c_first,
-                                                 int c_last, bool& timed_out, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(&sh.seg_bars[seg], 0) ? 1 : 0;
-    ok = __shfl_sync(kFull, ok, 0);
-    if (!ok) timed_out = true;
-    if (s.local(sp.g)) return true;
-    int last = 0;
-    if (lane == 0) {
-        __threadfence();  // this CTA's triples first, then its ticket
-        const int ticket = atomicAdd(&sp.row_arrivals[s.row], 1);
-        last = ticket == c_last - c_first ? 1 : 0;
-        if (last) {
-            sp.row_arrivals[s.row] = 0;  // every part has arrived: ready for the next launch
-            __threadfence();             // the other CTAs' triples are visible from here on
-        }
-    }
-    return __shfl_sync(kFull, last, 0) != 0;
-}
-
+// The helper warp, during the sweep: lists the rows this CTA will finish, each with its totals (fp64, from the
+// triples) and the piece that holds the target.  It follows the segments in the order they are streamed and waits for
+// each on the segment's mbarrier, so all of this hides behind the sweep except for the segment streamed last.  For the
+// CTA's part of a shared row it takes the CTA's ticket first and goes on only with the last ticket.  A finished row
+// (absorbing EOS) is reported to its group by the CTA that holds the row's last granule.
 template <int DT, int MODE>
-__device__ __noinline__ void finisher_warp(const StepParams& sp, StepShared& sh, const float4* local_triples, int first_row,
-                                              int S, int lane) {
+__device__ __noinline__ void helper_warp(const StepParams& sp, StepShared& sh, const float4* local_triples, int first_row,
+                                         int S, int lane) {
     const WeightsArgs& a = sp.a;
     const int N = a.N;
-    // every segment but the last one in order is finished by this warp alone, while the sweep goes on
+    for (int seg = lane; seg < S; seg += 32) {  // everything that does not depend on the sweep, ahead of it
+        const int row = first_row + seg, g = row / N;
+        sh.seg_u[seg] = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)(row - g * N)));
+    }
+    __syncwarp();
     for (int k = 0; k < S; ++k) {
-        const bool at_end = k == S - 1;
         const int seg = segment_in_order(k, S);
         const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + seg);
-        const int row = s.row, g = row / N;
-        if (at_end && lane == 0) sh.end_go = 0;
+        const int row = s.row;
         if (sh.seg_done[seg]) {
-            // a finished row is reported to its group by the CTA that holds the row's last granule
-            if (s.g1 == sp.g.gpr) row_arrives(sp, sh, row, nullptr, false, lane);
+            if (s.g1 == sp.g.gpr) row_arrives(sp, sh, sh.sc, row, nullptr, false, lane);
             continue;
         }
-        const int c_first = share_of(sp.g, row * sp.g.gpr), c_last = share_of(sp.g, (row + 1) * sp.g.gpr - 1);
-        bool timed_out = false;
-        if (!segment_complete(sp, sh, s, seg, c_first, c_last, timed_out, lane)) continue;
-        RowResult rr{-1, 0.0, 0.0};
-        RowTotals t;
-        t.ok = false;
-        if (!timed_out) {
-            const double U = hash_uniform(hash5(a.seed, kStreamToken, (uint64_t)g, (uint64_t)a.t, (uint64_t)(row - g * N)));
-            t = row_totals<MODE>(sp, local_triples, s, seg, c_first, c_last, U, lane);
+        int c_first = (int)blockIdx.x, c_last = (int)blockIdx.x;
+        if (!s.local(sp.g)) {
+            c_first = share_of(sp.g, row * sp.g.gpr);
+            c_last = share_of(sp.g, (row + 1) * sp.g.gpr - 1);
         }
-        if (t.ok) {
-            int a0, b0;
-            selected_range<DT>(sp, s, c_first, t.jsel, a0, b0);
-            if (at_end) {  // hand the row to the whole CTA
-                if (lane == 0) {
-                    sh.end_t = t;
-                    sh.end_row = row;
-                    sh.end_a0 = a0;
-                    sh.end_b0 = b0;
-                    sh.end_go = 1;
-                }
-                return;
+        // Every streaming warp of this CTA has stored its triple of the segment.  Each of them gets there in bounded
+        // time (its own waits are bounded and it arrives whatever happens), so this wait ends.
+        if (S <= kNamedBarriers) named_sync(1 + k, (sp.g.W + 1) * 32);
+        int mine = 1;
+        if (lane == 0) {
+            if (S > kNamedBarriers && !mbar_wait_idle(&sh.seg_bars[seg], 0)) sh.timed_out = 1;
+            if (c_last > c_first) {  // this CTA's triples first, then its ticket
+                mine = arrive_acq_rel(&sp.row_arrivals[row]) == c_last - c_first ? 1 : 0;
+                if (mine) sp.row_arrivals[row] = 0;  // every part has arrived: ready for the next launch
             }
-            const void* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * (DT == PSMC_F32 ? 4 : 2);
-            const int y = locate_in_range_warp<DT, MODE>(sp.f, rowp, t, a0, b0, lane);
-            if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
         }
-        row_arrives(sp, sh, row, &rr, timed_out, lane);
+        mine = __shfl_sync(kFull, mine, 0);
+        if (!mine) continue;
+        RowTotals t = row_totals<MODE>(sp, local_triples, s, seg, c_first, c_last, sh.seg_u[seg], lane);
+        int a0 = 0, b0 = 0;
+        if (t.ok) selected_range<DT>(sp, s, c_first, t.jsel, a0, b0);
+        if (lane == 0) {
+            const int i = sh.n_pend++;
+            sh.pend_t[i] = t;
+            sh.pend_row[i] = row;
+            sh.pend_a0[i] = a0;
+            sh.pend_b0[i] = b0;
+        }
+        __syncwarp();
     }
 }
 
-// The CTA's last row by all of its warps: one contiguous run of 16-byte chunks per thread (one chunk each when the
-// piece has no more chunks than the CTA has threads), the warp whose threads reach the target names the token.
-// Every thread of the CTA calls this.
+// After the sweep, every thread of the CTA: the pending rows, (warps / wpr) at a time.  The wpr warps of a row's team
+// share the re-read of the piece that holds the target (contiguous 16-byte chunks per thread); the warp whose threads
+// reach the target names the token and reports the row.
 template <int DT, int MODE>
-__device__ __noinline__ void finish_last_row(const StepParams& sp, StepShared& sh) {
+__device__ __noinline__ void finish_pending(const StepParams& sp, StepShared& sh, unsigned char* rings) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    const RowTotals t = sh.end_t;
-    const int row = sh.end_row, a0 = sh.end_a0, b0 = sh.end_b0;
-    const void* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * (DT == PSMC_F32 ? 4 : 2);
-    const float neg_C = -t.C;
-    const int chunks = (b0 - a0 + kPer - 1) / kPer;
-    const int E = ((chunks + (int)blockDim.x - 1) / (int)blockDim.x) * kPer;  // logits per thread
-    const int e0 = a0 + (int)threadIdx.x * E;
-    const double lm = lane_share<DT, MODE, 4>(sp.f, rowp, e0, E, b0, neg_C);
-    const double incl = warp_scan_incl(lm, lane);
-    if (lane == 31) sh.end_tot[warp] = incl;
-    __syncthreads();
-    // which warp's threads reach the target: the same additions, in the same order, in every warp
-    double cum = t.base, before = t.base;
-    int first_hit = -1;
-    for (int i = 0; i < n_warps; ++i) {
-        if (i == warp) before = cum;
-        const double ti = sh.end_tot[i];
-        cum += ti;
-        if (first_hit < 0 && ti > 0.0 && cum >= t.target) first_hit = i;
-    }
-    int y = -1;
-    bool mine = false;
-    if (first_hit == warp) {
-        mine = true;
-        const double r_incl = before + incl;
-        const unsigned hit = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
-        const int owner = hit ? __ffs(hit) - 1 : 31;
-        const double run = __shfl_sync(kFull, r_incl - lm, owner);
-        const int o0 = a0 + (warp * 32 + owner) * E;
-        y = locate_in_lane<DT, MODE>(sp.f, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
-    } else if (first_hit < 0 && warp == 0) {
-        mine = true;  // the re-read sums fall short of the target: last token with mass in the piece
-        y = last_with_mass<DT, MODE>(sp.f, rowp, a0, b0, neg_C, lane);
-    }
-    if (mine) {
-        RowResult rr{-1, 0.0, 0.0};
-        if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
-        row_arrives(sp, sh, row, &rr, false, lane);
+    const int n = sh.n_pend;
+    const bool timed_out = sh.timed_out != 0;
+    int wpr = 1;
+    while (wpr * 2 * n <= n_warps && wpr * 2 <= 8) wpr *= 2;
+    const int rows_per_pass = n_warps / wpr;
+    const int q = warp & (wpr - 1), kk = warp / wpr;
+    // a streaming warp's ring is idle by now: room for the group update's scratch
+    GroupScratch<32>& sc = warp < sp.g.W ? *reinterpret_cast<GroupScratch<32>*>(rings + (size_t)warp * kDepth * kStageBytes)
+                                         : sh.sc;
+    for (int k0 = 0; k0 < n; k0 += rows_per_pass) {
+        // ---- wpr warps per row: mass of each part of the selected piece ----
+        const bool active = kk < rows_per_pass && k0 + kk < n;
+        RowTotals t;
+        t.ok = false;
+        int row = 0, a0 = 0, b0 = 0, E = 0;
+        const void* rowp = nullptr;
+        float neg_C = 0.f;
+        double lm = 0.0, incl = 0.0;
+        if (active) {
+            t = sh.pend_t[k0 + kk];
+            if (timed_out) t.ok = false;
+            row = sh.pend_row[k0 + kk];
+            rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * (DT == PSMC_F32 ? 4 : 2);
+            if (t.ok) {
+                a0 = sh.pend_a0[k0 + kk];
+                b0 = sh.pend_b0[k0 + kk];
+                neg_C = -t.C;
+                const int chunks = (b0 - a0 + kPer - 1) / kPer, team = wpr * 32;
+                E = ((chunks + team - 1) / team) * kPer;  // logits per thread
+                lm = lane_share<DT, MODE, 8>(sp.f, rowp, a0 + (q * 32 + lane) * E, E, b0, neg_C);
+                incl = warp_scan_incl(lm, lane);
+            }
+            if (lane == 31) sh.end_tot[warp] = incl;
+        }
+        __syncthreads();
+        // ---- the warp whose threads reach the target: the token ----
+        if (active) {
+            const int w0 = warp - q;  // first warp of this row's team
+            if (!t.ok) {
+                if (q == 0) {
+                    const RowResult bad{-1, 0.0, 0.0};
+                    row_arrives(sp, sh, sc, row, &bad, timed_out, lane);
+                }
+            } else {
+                // which part of the piece reaches the target: the same additions, in the same order, in every warp
+                double cum = t.base, before = t.base;
+                int first_hit = -1;
+                for (int i = 0; i < wpr; ++i) {
+                    if (i == q) before = cum;
+                    const double ti = sh.end_tot[w0 + i];
+                    cum += ti;
+                    if (first_hit < 0 && ti > 0.0 && cum >= t.target) first_hit = i;
+                }
+                int y = -1;
+                bool mine = false;
+                if (first_hit == q) {
+                    mine = true;
+                    const double r_incl = before + incl;
+                    const unsigned hit = __ballot_sync(kFull, lm > 0.0 && r_incl >= t.target);
+                    const int owner = hit ? __ffs(hit) - 1 : 31;
+                    const double run = __shfl_sync(kFull, r_incl - lm, owner);
+                    const int o0 = a0 + (q * 32 + owner) * E;
+                    y = locate_in_lane<DT, MODE>(sp.f, rowp, o0, min(b0, o0 + E), run, t.target, neg_C, lane);
+                } else if (first_hit < 0 && q == 0) {
+                    mine = true;  // the re-read sums fall short of the target: last token with mass in the piece
+                    y = last_with_mass<DT, MODE>(sp.f, rowp, a0, b0, neg_C, lane);
+                }
+                if (mine) {
+                    RowResult rr{-1, 0.0, 0.0};
+                    if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
+                    row_arrives(sp, sh, sc, row, &rr, false, lane);
+                }
+            }
+        }
+        if (k0 + rows_per_pass < n) __syncthreads();  // sh.end_tot is reused by the next pass
     }
 }
 
@@ -485,16 +518,17 @@ __global__ void __launch_bounds__((kStepWarps + 1) * 32, 1) psmc_step_kernel(con
     chain_begin();  // everything above is local set-up; global memory from here on
     if (sp.zero_words && blockIdx.x == 0 && threadIdx.x < 2) sp.zero_words[threadIdx.x] = 0;
     if ((int)threadIdx.x < S) sh.seg_done[threadIdx.x] = sp.a.done[first_row + threadIdx.x];
+    if (threadIdx.x == 0) sh.n_pend = sh.timed_out = 0;
     __syncthreads();
 
     if (warp < W) {
         stream_pieces<DT, MODE>(sp, sh, local_triples, first_row, S, warp, lane, smem + (size_t)warp * kDepth * kStageBytes,
                                 sh.ring_bars + warp * kDepth);
     } else {
-        finisher_warp<DT, MODE>(sp, sh, local_triples, first_row, S, lane);
+        helper_warp<DT, MODE>(sp, sh, local_triples, first_row, S, lane);
     }
-    __syncthreads();  // the sweep is over; the finisher has left the CTA's last row (if it is this CTA's to finish) in sh
-    if (sh.end_go) finish_last_row<DT, MODE>(sp, sh);
+    __syncthreads();  // the sweep is over, every bulk copy has landed and been summed; sh lists this CTA's rows
+    if (sh.n_pend > 0) finish_pending<DT, MODE>(sp, sh, smem);
 }
 
 typedef void (*StepFn)(const StepParams);
@@ -515,7 +549,7 @@ bool step_geometry(int R, int V, int dt, StepGeom& g, int& grid) {
     const int64_t row_bytes16 = (int64_t)(V / per16) * 16;
     const int64_t gpr = row_bytes16 > 0 ? (row_bytes16 + kGranule - 1) / kGranule : 1;
     const int64_t total = (int64_t)R * gpr;
-    if (total >= (int64_t)1 << 30) return false;
+    if (total >= (int64_t)1 << 30 || gpr * 256 >= (int64_t)1 << 32) return false;
     grid = (int)(total < kSMs ? total : kSMs);
     g.gpr = (int)gpr;
     g.base = (int)(total / grid);

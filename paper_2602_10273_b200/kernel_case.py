@@ -103,7 +103,7 @@ def case_step(a):
     G = cfg.G if a.groups is None else a.groups
     wl = WC.DeviceWorkload(cfg, 1, G=G)
     n_buf = min(64, max(2, -(-2 * L2_BYTES // (wl.R * cfg.logit_bytes_per_row))))
-    T = 2 * a.iters + 4
+    T = 3 * a.iters + 8
     ps = B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
                 T_max=T, prompt_len=wl.prompt_len)
     if a.top_k or a.top_p:
@@ -118,7 +118,21 @@ def case_step(a):
 
     us = _time(run, a.iters)
     assert ps.sync_status() == B.OK
-    # the two kernels of the step, each bracketed by events on the stream
+    # the same launches back to back between ONE pair of events: what a step costs in a run of steps, where the next
+    # launch is already queued when a kernel ends
+    ps.reset(1)
+    for i in range(2):
+        run(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(a.iters):
+        run(2 + i)
+    e1.record()
+    torch.cuda.synchronize()
+    back_to_back = e0.elapsed_time(e1) * 1e3 / a.iters
+    assert ps.sync_status() == B.OK
+    # the kernels of the step, each bracketed by events on the stream
     ps.reset(1)
     ps.timing_enable(True)
     for i in range(a.iters):
@@ -127,7 +141,7 @@ def case_step(a):
     ps.timing_enable(False)
     ps.destroy()
     return {"case": "step", "workload": cfg.name, "rows": wl.R, "vocab": cfg.V, "buffers": n_buf, "us": us,
-            "top_k": a.top_k, "top_p": a.top_p,
+            "top_k": a.top_k, "top_p": a.top_p, "back_to_back_us": back_to_back,
             "logits_stream_us": 1e3 * kms[0] / max(kn[0], 1), "finish_weights_us": 1e3 * kms[1] / max(kn[1], 1),
             "us_median": float(np.median(us)), "bytes": wl.R * cfg.logit_bytes_per_row,
             "gb_per_s": wl.R * cfg.logit_bytes_per_row / (np.median(us) * 1e-6) / 1e9}
