@@ -354,7 +354,7 @@ psmc_status psmc_shard_finish(psmc_ctx*, const double* all_triples, const psmc_s
  * up to the current step; caches (dense or paged, with their tables) are the caller's to save, and the move list
  * of a step does not travel: take the snapshot after the step's cache move.  psmc_state_save
  * writes psmc_state_bytes() bytes to HOST memory; psmc_state_load needs a context created with the same G, N, V,
- * T_max (PSMC_E_INVAL otherwise, nothing loaded) and takes over alpha, tau, kappa, ramp, eos, seed, resampler and
+ * T_max and per-group prompt lengths (PSMC_E_INVAL otherwise, nothing loaded) and takes over alpha, tau, kappa, ramp, eos, seed, resampler and
  * the step counter from the snapshot.  Both synchronise the device. */
 size_t psmc_state_bytes(const psmc_ctx*);
 psmc_status psmc_state_save(psmc_ctx*, void* host_buf, size_t bytes);

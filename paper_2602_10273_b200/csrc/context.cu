@@ -582,7 +582,7 @@ struct SnapshotHeader {
     double top_p;
     int32_t top_k, reserved;
 };
-constexpr uint64_t kSnapshotMagic = 0x32434d5350ull;  // "PSMC2"
+constexpr uint64_t kSnapshotMagic = 0x33434d5350ull;  // "PSMC3"
 
 // the device arrays of a snapshot, in file order; hist arrays only up to step t
 struct Piece {
@@ -604,7 +604,7 @@ int snapshot_pieces(psmc_ctx* c, int t, Piece* out) {
 size_t snapshot_bytes(psmc_ctx* c, int t) {
     Piece ps[20];
     const int n = snapshot_pieces(c, t, ps);
-    size_t total = sizeof(SnapshotHeader);
+    size_t total = sizeof(SnapshotHeader) + 4 * (size_t)c->G;  // header, the G prompt lengths, the device arrays
     for (int i = 0; i < n; ++i) total += ps[i].bytes;
     return total;
 }
@@ -627,6 +627,8 @@ extern "C" psmc_status psmc_state_save(psmc_ctx* c, void* host_buf, size_t bytes
     char* out = static_cast<char*>(host_buf);
     memcpy(out, &h, sizeof(h));
     out += sizeof(h);
+    memcpy(out, c->prompt_len_host, 4 * (size_t)c->G);
+    out += 4 * (size_t)c->G;
     Piece ps[20];
     const int n = snapshot_pieces(c, c->t, ps);
     for (int i = 0; i < n; ++i) {
@@ -644,10 +646,13 @@ extern "C" psmc_status psmc_state_load(psmc_ctx* c, const void* host_buf, size_t
         h.t > c->T_max || h.resampler < 0 || h.resampler > 3)
         return PSMC_E_INVAL;
     if (bytes < snapshot_bytes(c, h.t)) return PSMC_E_INVAL;
+    // the prompt lengths decide which cache positions the shared-prompt reindex and the paged cache leave alone:
+    // a context created with other lengths would go on silently with the wrong ones
+    if (memcmp(static_cast<const char*>(host_buf) + sizeof(h), c->prompt_len_host, 4 * (size_t)c->G) != 0) return PSMC_E_INVAL;
     if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
     psmc_status st = reset_device_state(c);  // counters, arrival words and the rest of the scratch state start clean
     if (st != PSMC_OK) return st;
-    const char* in = static_cast<const char*>(host_buf) + sizeof(h);
+    const char* in = static_cast<const char*>(host_buf) + sizeof(h) + 4 * (size_t)c->G;
     Piece ps[20];
     const int n = snapshot_pieces(c, h.t, ps);
     for (int i = 0; i < n; ++i) {

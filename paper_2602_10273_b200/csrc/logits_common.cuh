@@ -9,7 +9,11 @@
 // All exponentials are taken in base 2 (the hardware's ex2): with x_v = l_v * log2(e),
 //   exp(l_v) = 2^{x_v}.  x_v - c is formed as fma(l, k_lo, fma(l, k_hi, -c)) with log2(e) = k_hi + k_lo split
 // over two floats, so the product carries no representation error of log2(e) and the big parts cancel
-// before the small one is added.  The streaming kernel cuts a row into spans and writes one triple (c, s1, sb)
+// before the small one is added.  k_hi has 16 significant bits: l k_hi - c is then exact for the terms that matter
+// (bf16 logits, c close to l k_hi), and l k_lo is far larger than the spacing of floats near x - c, so the one
+// rounding that is left is unbiased.  (With k_hi = float(log2 e) the small part, 2e-8 l, was below half that
+// spacing for most terms and simply dropped out of the sum: every x low by 2e-8 l, the dominant terms of a row low
+// by about 3e-8 of their value, always in the same direction.)  The streaming kernel cuts a row into spans and writes one triple (c, s1, sb)
 // per span:   c = a reference exponent (close to the span's largest x),  s1 = sum 2^{x - c},
 //   sb = sum 2^{beta (x - c)}.  Reference exponents are whole numbers.
 // The finish rescales the triples to the row's largest c in fp64, in span order, finds the span
@@ -24,8 +28,8 @@ namespace psmc {
 
 constexpr float kNegBig = -3.3895313892515355e38f;  // most negative finite bf16; start value of a running maximum
 constexpr float kRefFloor = -3.0e38f;               // reference exponent of a lane or span that saw no finite logit
-constexpr float kLog2eHi = 1.4426950216293335f;     // float(log2 e)
-constexpr float kLog2eLo = 1.925963033500011e-8f;   // float(log2 e - kLog2eHi)
+constexpr float kLog2eHi = 1.44268798828125f;       // log2 e to 16 significant bits: its product with a bf16 logit is exact
+constexpr float kLog2eLo = 7.052607543300837e-6f;   // float(log2 e - kLog2eHi); what is left is 1.7e-13
 constexpr double kLn2 = 0.6931471805599453;
 
 enum BetaMode { kBeta1 = 0, kBeta2 = 1, kBeta4 = 2, kBeta8 = 3, kBetaAny = 4 };
@@ -48,9 +52,33 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ float rel_exponent(float l, float neg_c) {
     return fmaf(l, kLog2eLo, fmaf(l, kLog2eHi, neg_c));
 }
-// reference exponent for a logit value m: m * log2(e) rounded up to a whole number (so that rescaling between
-// reference points is an exact power of two), kept finite
-__device__ __forceinline__ float ref_exponent(float m) { return fmaxf(ceilf(m * kLog2eHi), kRefFloor); }
+// Reference exponent for logits bounded by m: m * log2(e) rounded up to a whole number (so that rescaling between
+// reference points is an exact power of two) plus `shift`, kept finite.  shift = 1 (ref_shift) puts every exponent
+// x - c at or below -1, where the hardware's 2^x has one known mean error (kEx2Low, below); between -1 and 0 and above
+// 0 its mean error is a different one, and sums that mix the ranges cannot be corrected.
+__device__ __forceinline__ float ref_exponent(float m, float shift) { return fmaxf(ceilf(m * kLog2eHi) + shift, kRefFloor); }
+// The shift costs range at the bottom: the largest term of a sum may then be as small as 2^{-2 - slack log2 e}, its
+// beta-th power 2^{-4.9 beta} with the slack of the streaming kernel.  Up to beta = 16 that stays far above the
+// smallest normal float; beyond, the reference is left where it is and the sums are not corrected.
+constexpr float kMaxShiftBeta = 16.f;
+__host__ __device__ __forceinline__ float ref_shift(float bf) { return bf <= kMaxShiftBeta ? 1.f : 0.f; }
+
+// ex2.approx.ftz.f32 returns 2^x low by this fraction of the value on average for x <= -1 (B200, 2^26 arguments per
+// range against exp2 in fp64: -4.95e-8 ... -5.08e-8 for every range [-k-1, -k), k = 1 ... 59; -2.2e-8 on [-1, 0),
+// +0.6e-8 on [0, 1), +3.3e-8 above).  A sum of such terms is low by the same fraction whatever the terms are, and a
+// sum of their beta-th powers formed by squaring (exactly rounded multiplications) by beta times that.  Left in, the
+// error is the same at every token and adds up in log p(y_{1:t}): 3.4e-8 per token, 1e-4 after 2900 tokens.
+constexpr double kEx2Low = 4.99e-8;
+// what to add to ln(sum 2^{x-c}) and ln(sum 2^{beta (x-c)}) as the kernels form them
+template <int MODE>
+__device__ __forceinline__ void ln_sum_corrections(double beta, double& add_s1, double& add_sb) {
+    if (ref_shift((float)beta) == 0.f) {
+        add_s1 = add_sb = 0.0;
+        return;
+    }
+    add_s1 = kEx2Low;
+    add_sb = (MODE == kBeta1 || MODE == kBetaAny) ? kEx2Low : beta * kEx2Low;  // one ex2 per term, or one squared up
+}
 
 // 2^{beta d} for d = x - c.  One MUFU: for beta in {1,2,4,8} 2^d is squared up; bf = (float)beta otherwise.
 template <int MODE>
@@ -327,13 +355,15 @@ __device__ __forceinline__ int locate_in_lane(const FinishParams& p, const void*
 
 // Called by all 32 lanes; every lane returns the same RowResult.  The two logarithms are taken side by side
 // (lane 0 and lane 1 of one call) rather than one after the other.
-template <int DT>
+template <int DT, int MODE>
 __device__ __forceinline__ RowResult row_result(const FinishParams& p, const void* rowp, const RowTotals& t, int y, int lane) {
     RowResult r;
     // l_y - C ln 2: the token's logit relative to the row's reference, in natural units
     const double dl = (double)load_elem<DT>(rowp, y) - (double)t.C * kLn2;
     const double lg = log((lane & 1) ? t.Sb : t.S1);
-    const double ln_s1 = __shfl_sync(kFull, lg, 0), ln_sb = __shfl_sync(kFull, lg, 1);
+    double add_s1, add_sb;
+    ln_sum_corrections<MODE>(p.beta, add_s1, add_sb);
+    const double ln_s1 = __shfl_sync(kFull, lg, 0) + add_s1, ln_sb = __shfl_sync(kFull, lg, 1) + add_sb;
     r.tok = y;
     r.logp = dl - ln_s1;  // log p(y) = l_y - L1
     // alpha_t log p(y) - log q(y), log q(y) = beta l_y - Lb, grouped so that the token's own logit drops out
@@ -371,7 +401,7 @@ __device__ __forceinline__ RowResult finish_row_warp(const FinishParams& p, int 
     const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
     const int y = locate_token_warp<DT, MODE>(p, rowp, t, lane);
     if (y < 0) return bad;
-    return row_result<DT>(p, rowp, t, y, lane);
+    return row_result<DT, MODE>(p, rowp, t, y, lane);
 }
 
 // ---- the finish at CTA level: several warps share a row ----
@@ -468,7 +498,7 @@ __device__ __forceinline__ void finish_rows(const FinishParams& p, FinishShared&
                 }
                 if (mine) {
                     RowResult rr{-1, 0.0, 0.0};
-                    if (y >= 0) rr = row_result<DT>(p, rowp, t, y, lane);
+                    if (y >= 0) rr = row_result<DT, MODE>(p, rowp, t, y, lane);
                     if (lane == 0) emit(k, rr);
                 }
             }

@@ -100,7 +100,8 @@ __device__ __forceinline__ f32x2 pair_scale(f32x2 v, float f) { return mul2(v, p
 struct PackedConsts {
     f32x2 k_hi, k_lo, bf;
     float bf1;
-    float slack;  // min(kRefSlack, 62 / beta): keeps 2^{beta slack log2 e} below 2^90
+    float slack;  // how far a logit may exceed the largest one seen before the reference moves (natural units)
+    float shift;  // ref_shift(beta)
 };
 __device__ __forceinline__ PackedConsts packed_consts(float bf) {
     PackedConsts k;
@@ -108,7 +109,11 @@ __device__ __forceinline__ PackedConsts packed_consts(float bf) {
     k.k_lo = pack2(kLog2eLo, kLog2eLo);
     k.bf = pack2(bf, bf);
     k.bf1 = bf;
-    k.slack = fminf(kRefSlack, 62.f / fmaxf(bf, 1.f));
+    k.shift = ref_shift(bf);
+    // With the shift the largest term of a sum has an exponent between -2 - slack log2(e) and -1, and what limits the
+    // accuracy of a term is the fp32 rounding of beta (x - c): the slack shrinks as beta grows so that beta |x - c|
+    // of the largest terms stays below about 20.  Without the shift (large beta) the slack keeps 2^{beta (x - c)} in range.
+    k.slack = k.shift != 0.f ? fminf(kRefSlack, 4.f / fmaxf(bf, 1.f)) : fminf(kRefSlack, 62.f / bf);
     // hide the values from constant propagation so that they are not rebuilt at every use
     asm volatile("" : "+l"(k.k_hi), "+l"(k.k_lo), "+l"(k.bf));
     return k;
@@ -135,13 +140,15 @@ __device__ __forceinline__ void add_pair(f32x2 d, const PackedConsts& k, f32x2& 
     }
 }
 // Some lane met a logit above the threshold; cm is this lane's largest candidate.  The warp moves its reference
-// exponent to the largest of them and shrinks the sums accordingly.  Called by all 32 lanes together.
-// Logits up to the new maximum + slack then pass without another move: a term stays below
-// 2^{beta slack log2 e} <= 2^90 and whatever underflows is smaller than 2^-126 against a largest term of about 1.
+// exponent beyond the largest of them plus the slack and shrinks the sums accordingly.  Called by all 32 lanes
+// together.  Logits up to the new maximum + slack then pass without another move; every term stays at or below 1/2,
+// the largest ones lie between 2^{-2 - slack log2 e} and 1/2, and whatever underflows is smaller than 2^-120 of them.
 template <int MODE>
-__device__ __forceinline__ void move_reference(float cm, float bf, float slack, LaneSums& a) {
+__device__ __forceinline__ void move_reference(float cm, const PackedConsts& k, LaneSums& a) {
+    const float bf = k.bf1, slack = k.slack;
     cm = warp_max(cm);
-    const float new_neg_c = -ref_exponent(cm);
+    // with the shift, logits up to the new threshold keep their exponents at or below -1
+    const float new_neg_c = -(k.shift != 0.f ? ref_exponent(cm + slack, 1.f) : ref_exponent(cm, 0.f));
     const float d0 = new_neg_c - a.neg_c;  // c_old - c_new < 0; hugely negative the first time, when the sums are empty
     const float f1 = ex2(d0);
     a.s1a = pair_scale(a.s1a, f1);
@@ -156,8 +163,9 @@ __device__ __forceinline__ void move_reference(float cm, float bf, float slack, 
 }
 // one logit per lane (ragged ends, unaligned rows); all 32 lanes call it, lanes without a logit pass -inf
 template <int MODE>
-__device__ __forceinline__ void add_one(float l, float bf, float slack, LaneSums& a) {
-    if (__any_sync(kFull, l > a.thr)) move_reference<MODE>(l, bf, slack, a);
+__device__ __forceinline__ void add_one(float l, const PackedConsts& k, LaneSums& a) {
+    const float bf = k.bf1;
+    if (__any_sync(kFull, l > a.thr)) move_reference<MODE>(l, k, a);
     const float d = rel_exponent(l, a.neg_c);  // -inf for a lane without a logit: mass 0
     a.s1a = add2(a.s1a, pack2(ex2(d), 0.f));
     if (MODE != kBeta1) a.sba = add2(a.sba, pack2(mass_beta<MODE>(d, bf), 0.f));
@@ -171,7 +179,7 @@ __device__ __forceinline__ void consume_bf16(const uint32_t (&w)[NW], const Pack
 #pragma unroll
     for (int i = 1; i < NW; ++i) pm = __hmax2(pm, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
     if (__any_sync(kFull, !__hble2(pm, thr2))) {  // some logit of the warp is above the threshold
-        move_reference<MODE>(fmaxf(__low2float(pm), __high2float(pm)), k.bf1, k.slack, a);
+        move_reference<MODE>(fmaxf(__low2float(pm), __high2float(pm)), k, a);
         thr2 = __float2bfloat162_rn(a.thr);
     }
     const f32x2 nc = pack2(a.neg_c, a.neg_c);
@@ -188,7 +196,7 @@ __device__ __forceinline__ void consume_f32(const uint32_t (&w)[NW], const Packe
     float cm = __uint_as_float(w[0]);
 #pragma unroll
     for (int i = 1; i < NW; ++i) cm = fmaxf(cm, __uint_as_float(w[i]));
-    if (__any_sync(kFull, cm > a.thr)) move_reference<MODE>(cm, k.bf1, k.slack, a);
+    if (__any_sync(kFull, cm > a.thr)) move_reference<MODE>(cm, k, a);
     const f32x2 nc = pack2(a.neg_c, a.neg_c);
 #pragma unroll
     for (int i = 0; i < NW; i += 2) {
@@ -209,7 +217,7 @@ template <int DT, int MODE>
 __device__ __forceinline__ void span_scalar(const void* rowp, int a0, int b0, const PackedConsts& k, int lane,
                                             LaneSums& acc) {
     for (int i0 = a0; i0 < b0; i0 += 32)  // the same trip count in every lane
-        add_one<MODE>(i0 + lane < b0 ? load_elem<DT>(rowp, i0 + lane) : -INFINITY, k.bf1, k.slack, acc);
+        add_one<MODE>(i0 + lane < b0 ? load_elem<DT>(rowp, i0 + lane) : -INFINITY, k, acc);
 }
 
 struct StreamParams {
@@ -342,7 +350,7 @@ __device__ __forceinline__ bool stream_tasks(const StreamParams& p, unsigned cha
     __nv_bfloat162 thr2 = __float2bfloat162_rn(acc.thr);
     auto finish_task = [&]() {
         if (c_d.tail > 0)  // ragged end of the row
-            add_one<MODE>(lane < c_d.tail ? load_elem<DT>(c_d.base + c_d.bytes16, lane) : -INFINITY, kc.bf1, kc.slack, acc);
+            add_one<MODE>(lane < c_d.tail ? load_elem<DT>(c_d.base + c_d.bytes16, lane) : -INFINITY, kc, acc);
         store_triple<MODE>(p, c_d.row, c_d.sp, acc, lane);
         stored(c_d.row);
     };

@@ -441,7 +441,7 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         }
         return;
     }
-    const float C = ref_exponent(mx), neg_C = -C;
+    const float C = ref_exponent(mx, ref_shift(p.bf)), neg_C = -C;
 
     bool have_list = false;
     int first_list_level = 2;
@@ -937,7 +937,9 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
             p.loginc[row] = 0.0;
         } else {
             const double dl = (double)load_elem<DT>(rowp, y) - (double)C * kLn2;
-            const double ln_s1 = log(S1), ln_sb = log(Sb);
+            double add_s1, add_sb;
+            ln_sum_corrections<MODE>(p.beta, add_s1, add_sb);
+            const double ln_s1 = log(S1) + add_s1, ln_sb = log(Sb) + add_sb;
             p.tok[row] = y;
             p.logp[row] = dl - ln_s1;
             p.loginc[row] = (p.alpha_t - p.beta) * dl - p.alpha_t * ln_s1 + ln_sb;

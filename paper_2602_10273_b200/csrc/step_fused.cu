@@ -267,7 +267,7 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
             acc = lane_sums_init();
             if (lane == 0) sh.timed_out = 1;
         } else if (d.tail > 0) {  // ragged end of the row
-            add_one<MODE>(lane < d.tail ? load_elem<DT>(d.src + d.bytes, lane) : -INFINITY, kc.bf1, kc.slack, acc);
+            add_one<MODE>(lane < d.tail ? load_elem<DT>(d.src + d.bytes, lane) : -INFINITY, kc, acc);
         }
         const float s1 = warp_sum(pair_sum(add2(acc.s1a, acc.s1b)));
         const float sb = (MODE == kBeta1) ? 0.f : warp_sum(pair_sum(add2(acc.sba, acc.sbb)));
@@ -491,7 +491,7 @@ __device__ __noinline__ void finish_pending(const StepParams& sp, StepShared& sh
                 }
                 if (mine) {
                     RowResult rr{-1, 0.0, 0.0};
-                    if (y >= 0) rr = row_result<DT>(sp.f, rowp, t, y, lane);
+                    if (y >= 0) rr = row_result<DT, MODE>(sp.f, rowp, t, y, lane);
                     row_arrives(sp, sh, sc, row, &rr, false, lane);
                 }
             }

@@ -228,7 +228,9 @@ __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_consta
                 if (pk.tok >= 0) {
                     // same grouping as the unsharded finish: the token's own logit drops out when beta = alpha_t
                     const double dl = (double)pk.logit - (double)tot.C * kLn2;
-                    const double ln_s1 = log(tot.S1), ln_sb = log(tot.Sb);
+                    double add_s1, add_sb;
+                    ln_sum_corrections<MODE>(a.beta, add_s1, add_sb);
+                    const double ln_s1 = log(tot.S1) + add_s1, ln_sb = log(tot.Sb) + add_sb;
                     tk = pk.tok;
                     lp = dl - ln_s1;
                     inc = (a.alpha_t - a.beta) * dl - a.alpha_t * ln_s1 + ln_sb;

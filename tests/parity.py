@@ -37,6 +37,7 @@ class LoopStats:
     resample_events: int = 0
     slots_moved: int = 0
     max_logw_err: float = 0.0
+    max_s_err: float = 0.0        # cumulative log p(y_{1:t}), never reset by resampling
     max_loginc_err: float = 0.0
     min_tok_margin: float = 1.0
 
@@ -46,6 +47,27 @@ def logits_to_numpy(t: torch.Tensor) -> np.ndarray:
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).cpu().numpy().view(np.uint16)
     return t.cpu().numpy()
+
+
+def logits_to_double(t: torch.Tensor) -> np.ndarray:
+    """Device logits as the doubles they stand for (bf16 and fp32 are both exact in a double)."""
+    if t.dtype == torch.bfloat16:
+        return W.bf16_bits_to_f32(t.view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+    return t.cpu().numpy().astype(np.float64)
+
+
+def check_rows_against_oracle(logits, beta, alpha_t, u, tok, logp, loginc, rows=None):
+    lg = logits_to_double(logits)
+    flagged = 0
+    for r in (range(lg.shape[0]) if rows is None else rows):
+        o = O.row(lg[r], beta, alpha_t, float(u[r]))
+        if o["y"] != tok[r]:
+            assert o["margin"] <= TOK_MARGIN, "row %d: %d vs %d margin %.3e" % (r, tok[r], o["y"], o["margin"])
+            flagged += 1
+            o = O.row(lg[r], beta, alpha_t, float(u[r]), force=int(tok[r]))
+        assert abs(o["log_omega"] - loginc[r]) <= TOL_LOGINC, (r, o["log_omega"], loginc[r])
+        assert abs(o["logp_y"] - logp[r]) <= TOL_LOGINC
+    return flagged
 
 
 def make_pair(cfg: W.Workload, seed: int, G: int = None, T_max: int = None, ramp: int = None, kappa: float = None,
@@ -125,7 +147,9 @@ def compare_step(ps: B.Psmc, orc: O.Oracle, lg_host: np.ndarray, st: LoopStats, 
     e = np.abs(ps.log_weights.numpy() - orc.log_weights).max()
     st.max_logw_err = max(st.max_logw_err, float(e))
     assert e <= TOL_LOGW, "log W differs by %.3e at step %d" % (e, orc.t)
-    assert np.abs(ps.cum_logp.numpy() - orc.cum_logp).max() <= TOL_LOGW
+    e = np.abs(ps.cum_logp.numpy() - orc.cum_logp).max()
+    st.max_s_err = max(st.max_s_err, float(e))
+    assert e <= TOL_LOGW, "S differs by %.3e at step %d" % (e, orc.t)
     assert np.abs(ps.log_z.numpy() - orc.log_z).max() <= TOL_LOGW * max(1, orc.t)
     st.steps += 1
 

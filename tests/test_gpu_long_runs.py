@@ -1,0 +1,59 @@
+"""The named configurations at their stated length (Algorithm 1 runs to T_max), CUDA path against the oracle at every
+token: the tolerance on log W and on S = log p(y_{1:t}) (1e-4 absolute) has to hold over the whole horizon, not just
+over the first tokens, and the final draw walks an ancestry log of the full length (several batches of the
+back-trace).  Caches keep the stated heads, head size and maximum length but one layer, to bound the host mirror.
+
+With PSMC_TEST_REPORT=<file> every run appends one JSON line with its counts (steps, resampling events, slots
+rewritten, choices the oracle adopted) and largest differences.
+"""
+import dataclasses
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import parity as P
+from paper_2602_10273_b200.workload import gen as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _report(label, st):
+    path = os.environ.get("PSMC_TEST_REPORT")
+    print(label, st)
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps({"run": label, **dataclasses.asdict(st)}) + "\n")
+
+
+@pytest.mark.parametrize("name", ["llama2_7b", "qwen25_7b", "resample_stress"])
+def test_closed_loop_at_the_stated_length(name):
+    c = W.CONFIGS[name]
+    st = P.closed_loop(c, seed=1, T=c.T, kv_shape=(1, c.n_kv_heads, c.max_len, c.head_dim))
+    assert st.steps == c.T and st.resample_events > 0 and st.slots_moved > 0
+    _report("%s, T = %d" % (name, c.T), st)
+
+
+def test_batched_prompts_eight_prompts_at_the_stated_length():
+    c = W.CONFIGS["batched_prompts"]
+    st = P.closed_loop(c, seed=1, T=c.T, G=8, kv_shape=(1, c.n_kv_heads, c.max_len, c.head_dim))
+    assert st.steps == c.T and st.resample_events > 0
+    _report("batched_prompts, 8 of 64 prompts, T = %d" % c.T, st)
+
+
+def test_batched_prompts_full_width_sixty_four_tokens():
+    c = W.CONFIGS["batched_prompts"]
+    st = P.closed_loop(c, seed=2, T=64, kv_shape=(1, c.n_kv_heads, c.max_len, c.head_dim))
+    assert st.live_rows == 64 * 512 and st.resample_events > 0
+    _report("batched_prompts, 64 prompts, T = 64", st)
+
+
+@pytest.mark.parametrize("N,V,T,kappa", [(33, 64, 300, 0.9), (1024, 32, 9, 1.0), (8, 50, 1200, 0.7)])
+def test_back_trace_over_several_batches(N, V, T, kappa):
+    """The output step stages its ancestry log in batches of 4096 integers; T * N beyond that takes several batches.
+    Frequent resampling and early EOS make the walk non-trivial (V is small, so EOS is drawn often)."""
+    c = W.Workload("trace", 1, N, V, "f32", 2.0, 1.5, T, 3, 3, 2.0, 0.5, kappa, 0, 1, 1, 8, T + 8)
+    st = P.closed_loop(c, seed=7, T=T)
+    assert st.steps == T and T * N > 4096 and st.resample_events > 0

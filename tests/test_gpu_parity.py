@@ -43,18 +43,7 @@ def run_logits_pass(logits, beta, alpha_t, u, done=None):
     return tok.cpu().numpy(), logp.cpu().numpy(), loginc.cpu().numpy(), int(status.item())
 
 
-def check_rows_against_oracle(logits, beta, alpha_t, u, tok, logp, loginc, rows=None):
-    lg = _to_double(logits)
-    flagged = 0
-    for r in (range(lg.shape[0]) if rows is None else rows):
-        o = O.row(lg[r], beta, alpha_t, float(u[r]))
-        if o["y"] != tok[r]:
-            assert o["margin"] <= P.TOK_MARGIN, "row %d: %d vs %d margin %.3e" % (r, tok[r], o["y"], o["margin"])
-            flagged += 1
-            o = O.row(lg[r], beta, alpha_t, float(u[r]), force=int(tok[r]))
-        assert abs(o["log_omega"] - loginc[r]) <= P.TOL_LOGINC, (r, o["log_omega"], loginc[r])
-        assert abs(o["logp_y"] - logp[r]) <= P.TOL_LOGINC
-    return flagged
+check_rows_against_oracle = P.check_rows_against_oracle
 
 
 # ------------------------------------------------------------------ the logit pass alone
@@ -321,6 +310,10 @@ def test_snapshot_resumes_bit_for_bit():
             with pytest.raises(B.PsmcError):
                 other.state_load(blob)                       # a different vocabulary: refused, nothing loaded
             other.destroy()
+            other = B.Psmc(c.N, c.V, c.alpha, c.tau, c.kappa, 0, 6, c.eos_id, G=1, T_max=T, prompt_len=wl.prompt_len + 1)
+            with pytest.raises(B.PsmcError):
+                other.state_load(blob)                       # other prompt lengths: the cache calls would skip wrongly
+            other.destroy()
     assert st.resample_events > 0
     toks, ln, ix = ps.select()
     o_toks, o_ln, o_ix = orc.select()
@@ -338,6 +331,41 @@ def test_eos_rows_freeze_and_are_not_read():
 
     st = P.closed_loop(c, seed=5, T=20, kappa=0.05, logit_bias_fn=push_eos)
     assert st.steps == 20
+
+
+def test_finished_slots_are_rewritten_by_live_ancestors_at_every_step():
+    """Finished flags that flip back to live while the step kernel is still reading flags elsewhere.  Every other
+    token two live slots per group are declared finished with a low weight (on both sides); kappa = 1 resamples at
+    once, so at the next token those slots are overwritten by live ancestors: a flag goes from 1 to 0 in a group that
+    closes early, while CTAs that hold other parts of the block have not looked at their rows' flags yet.  Rows span
+    several CTAs (5000 logits = 20 granules, 6.5 granules per CTA).  Every token is compared, the status stays clean."""
+    c = W.Workload("flip", 6, 8, 5000, "bf16", 3.0, 1.5, 300, 5, 9, 4.0, 0.25, 1.0, 0, 1, 2, 16, 320)
+    T = 300
+    wl, ps, orc = P.make_pair(c, seed=11, T_max=T)
+    st = P.LoopStats()
+    lg = wl.new_logits()
+    prev = wl.first_prev.clone()
+    flips = 0
+    for t in range(1, T + 1):
+        before = ps.done.numpy().copy()
+        wl.fill(lg, t, prev)
+        ps.step(lg)
+        P.compare_step(ps, orc, P.logits_to_numpy(lg), st, 1.0)
+        after = ps.done.numpy()
+        flips += int(((before == 1) & (after == 0)).sum())
+        prev.copy_(ps.device_view("psmc_last_tokens", ps.R))
+        if t % 2 == 0:
+            lw, dn = ps.log_weights.numpy().copy(), after.copy()
+            for g in range(c.G):
+                live = [r for r in range(g * c.N, (g + 1) * c.N) if not dn[r]]
+                for r in live[:2] if len(live) > 3 else []:
+                    dn[r] = 1
+                    lw[r] -= 40.0
+            ps.set_state(log_w=lw, done=dn)
+            orc.set_state(logW=lw, done=dn)
+    assert ps.sync_status() == B.OK
+    assert st.steps == T and st.resample_events > 100 and flips > 100
+    ps.destroy()
 
 
 def test_done_rows_logits_are_never_read():

@@ -5,7 +5,8 @@ may not call cudaMalloc because it would stall the device, a loop with a no-allo
 rule) passes only inputs and outputs; the span partials live in a fixed array inside the library.
 The test calls the entry point through the C-ABI twice in a row, on different shapes so that the
 second call finds the first call's leftovers in the shared array, and checks each result against
-psmc_logits_pass (caller-provided scratch) on the same inputs.  It is collected last on purpose.
+psmc_logits_pass (caller-provided scratch) on the same inputs and, row by row, against the CPU oracle.
+It is collected last on purpose.
 """
 import ctypes as C
 
@@ -61,6 +62,10 @@ def test_static_scratch_entry_point_matches_the_scratch_taking_one_twice_in_a_ro
         assert (r_tok[live] >= 0).all() and (r_tok[~live] == -7).all()       # finished rows are left untouched
         assert np.abs(logp.cpu().numpy() - r_logp).max() <= TOL
         assert np.abs(loginc.cpu().numpy() - r_loginc).max() <= TOL
+        # and the oracle's row function on the same bits (tokens equal unless the uniform sits on a CDF boundary)
+        import parity as P
+        P.check_rows_against_oracle(logits, beta, alpha_t, u.cpu().numpy(), tok.cpu().numpy(), logp.cpu().numpy(),
+                                  loginc.cpu().numpy(), rows=np.nonzero(live)[0])
 
 
 def test_static_scratch_entry_point_refuses_what_does_not_fit():
