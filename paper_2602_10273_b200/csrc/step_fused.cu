@@ -417,17 +417,16 @@ __device__ __noinline__ void helper_warp(const StepParams& sp, StepShared& sh, c
 
 // After the sweep, every thread of the CTA: the pending rows, (warps / wpr) at a time.  The wpr warps of a row's team
 // share the re-read of the piece that holds the target (contiguous 16-byte chunks per thread); the warp whose threads
-// reach the target names the token and reports the row.
+// reach the target names the token and reports the row.  (A team need not be a power of two of warps.)
 template <int DT, int MODE>
 __device__ __noinline__ void finish_pending(const StepParams& sp, StepShared& sh, unsigned char* rings) {
     constexpr int kPer = DT == PSMC_BF16 ? 8 : 4;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     const int n = sh.n_pend;
     const bool timed_out = sh.timed_out != 0;
-    int wpr = 1;
-    while (wpr * 2 * n <= n_warps && wpr * 2 <= 8) wpr *= 2;
+    const int wpr = max(1, min(8, n_warps / n));  // warps per row: all of the CTA's warps shared out, eight at most
     const int rows_per_pass = n_warps / wpr;
-    const int q = warp & (wpr - 1), kk = warp / wpr;
+    const int kk = warp / wpr, q = warp - kk * wpr;
     // a streaming warp's ring is idle by now: room for the group update's scratch
     GroupScratch<32>& sc = warp < sp.g.W ? *reinterpret_cast<GroupScratch<32>*>(rings + (size_t)warp * kDepth * kStageBytes)
                                          : sh.sc;
