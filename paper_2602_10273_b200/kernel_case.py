@@ -7,6 +7,7 @@ what-does-this-shape-cost questions:
   python -m paper_2602_10273_b200.kernel_case reindex --rows 64 --layers 8 --heads 8 --len 1024 --iters 3
   python -m paper_2602_10273_b200.kernel_case step --workload qwen25_7b --iters 20
   python -m paper_2602_10273_b200.kernel_case shard_step --workload batched_prompts --ranks 8 --iters 20
+  python -m paper_2602_10273_b200.kernel_case select --workload batched_prompts --groups 8 --steps 1024 --iters 3
 
 Each case rotates through enough distinct input buffers to exceed the L2 cache, so that the
 device-time and DRAM counters describe HBM-bound behaviour.
@@ -147,6 +148,33 @@ def case_step(a):
             "gb_per_s": wl.R * cfg.logit_bytes_per_row / (np.median(us) * 1e-6) / 1e9}
 
 
+def case_select(a):
+    """psmc_select (final draw + back-trace of the ancestry log) after --steps tokens of a named workload."""
+    cfg = gen.CONFIGS[a.workload]
+    G = cfg.G if a.groups is None else a.groups
+    wl = WC.DeviceWorkload(cfg, 1, G=G)
+    T = a.steps
+    ps = B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
+                T_max=T, prompt_len=wl.prompt_len)
+    lg = wl.new_logits()
+    prev = wl.first_prev.clone()
+    last = ps.device_view("psmc_last_tokens", wl.R)
+    for t in range(1, T + 1):
+        wl.fill(lg, t, prev)
+        ps.step(lg)
+        prev.copy_(last)
+    out = ps.select()
+
+    def run(i):
+        ps.select(*out)
+
+    us = _time(run, a.iters)
+    assert ps.sync_status() == B.OK
+    ps.destroy()
+    return {"case": "select", "workload": cfg.name, "groups": G, "particles": cfg.N, "steps": T, "us": us,
+            "us_median": float(np.median(us)), "log_bytes": 2 * 4 * wl.R * T}
+
+
 def case_shard_step(a):
     """One rank's share of the step on a vocabulary split over --ranks ranks (this GPU plays every rank in turn; the
     all-gathers are a stack on the device and are not timed).  Reports rank 0's three calls."""
@@ -207,7 +235,8 @@ def case_shard_step(a):
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("case", choices=["logits", "reindex", "step", "shard_step"])
+    ap.add_argument("case", choices=["logits", "reindex", "step", "shard_step", "select"])
+    ap.add_argument("--steps", type=int, default=1024, help="select: tokens decoded before the final draw")
     ap.add_argument("--ranks", type=int, default=8)
     ap.add_argument("--top-k", type=int, default=0, help="step: proposal restricted to the top-k tokens")
     ap.add_argument("--top-p", type=float, default=0.0, help="step: proposal restricted to the nucleus of this share")
@@ -225,7 +254,8 @@ def main():
     ap.add_argument("--no-ramp", action="store_true")
     ap.add_argument("--iters", type=int, default=5)
     a = ap.parse_args()
-    out = {"logits": case_logits, "reindex": case_reindex, "step": case_step, "shard_step": case_shard_step}[a.case](a)
+    out = {"logits": case_logits, "reindex": case_reindex, "step": case_step, "shard_step": case_shard_step,
+           "select": case_select}[a.case](a)
     print(json.dumps(out))
 
 
