@@ -13,16 +13,17 @@
 // while the sweep is still running.
 //
 // Who finishes a row, and when.  Dependent trips to memory take several times longer while the sweep saturates HBM
-// than after it, so no row is finished during the sweep; what happens during the sweep is only what must happen
-// between CTAs.  One extra warp per CTA, the helper, waits on a shared-memory mbarrier that the streaming warps of
-// ITS OWN CTA arrive on (every wait is for warps that are resident by construction) until the CTA's part of a shared
-// row is complete, then takes a ticket on the row's global counter: the CTA that draws the last ticket owns the row.
-// No CTA ever waits for another one.  After the sweep all warps of the CTA finish the rows it owns (its local rows
-// and the shared rows it drew the last ticket for) together, a team of up to eight warps per row: totals in fp64 from
-// the triples (shared memory, or global memory for a shared row), the piece that holds U * sum, a re-read of that
-// piece split over the team (a few KB, still in L2), the token, log p(y) and log omega (logits_common.cuh).  A
-// finished row counts one arrival for its group, and the warp that brings a group to N arrivals runs the group's
-// update (weights_core.cuh) on the spot.
+// than after it, and a warp that polls takes issue slots from the warps that stream, so during the sweep only what
+// must happen between CTAs happens, plus arithmetic on shared memory.  One extra warp per CTA, the helper, is parked
+// on a named CTA barrier that the streaming warps of ITS OWN CTA arrive on (every wait is for warps that are resident
+// by construction and whose own waits are bounded) until a segment is complete.  For the CTA's part of a shared row
+// it then takes a ticket on the row's global counter: the CTA that draws the last ticket owns the row.  No CTA ever
+// waits for another one.  For every row the CTA owns the helper forms the totals in fp64 from the triples (shared
+// memory, or global memory for a shared row) and names the piece that holds U * sum; all of that hides behind the
+// sweep except for the row streamed last.  After the sweep all warps of the CTA finish the rows it owns together, a
+// team of up to eight warps per row: a re-read of the selected piece split over the team (a few KB, still in L2), the
+// token, log p(y) and log omega (logits_common.cuh).  A finished row counts one arrival for its group, and the warp
+// that brings a group to N arrivals runs the group's update (weights_core.cuh) on the spot.
 //
 // The finished flags are read from one array and written to another (they alternate from step to step): a group may
 // close, and rewrite its flags, while other CTAs have not looked at the flags of their rows yet.  Arrival counters
@@ -38,7 +39,7 @@ namespace psmc {
 namespace {
 
 constexpr int kGranule = 512;      // bytes: one 16-byte chunk per lane
-constexpr int kStepWarps = 23;     // streaming warps per CTA at most (with the finisher: 6 warps per scheduler, 80 registers)
+constexpr int kStepWarps = 23;     // streaming warps per CTA at most (with the helper: 6 warps per scheduler, 80 registers)
 constexpr int kMaxSegments = 48;   // rows one CTA's share may meet (shapes beyond that take the two-kernel step)
 constexpr int kMinGranulesPerWarp = 4;
 static_assert(kStepWarps % 4 == 3, "the helper completes the last scheduler's set of warps");
