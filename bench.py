@@ -223,6 +223,9 @@ def run_ours(args):
         raise SystemExit("steps + warmup exceed the cache length of the workload")
     # shrink the number of prompts only if the cache does not fit this GPU (never the shapes)
     G = cfg.G if args.groups is None else args.groups
+    if args.split_prompts:  # strong scaling: the workload's prompts are split over the ranks instead of multiplied
+        lo, hi = replicas.shard_groups(G, world, rank)
+        G = max(1, hi - lo)
     free_b, _ = torch.cuda.mem_get_info(dev)
     per_group = cfg.N * cfg.max_len * cfg.kv_bytes_per_pos_per_row
     fixed = N_BLOCKS * cfg.N * cfg.logit_bytes_per_row  # per group
@@ -467,7 +470,7 @@ def run_ours(args):
     live_k = float(np.sum(live_rows[Wm:]))
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "strong" if args.split_prompts else "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "%s: %d prompts x %d particles, V=%d, KV %dx%dx%d max_len %d (%s)" % (
                        cfg.name, G, N, cfg.V, cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, cfg.max_len, cfg.dtype),
@@ -617,6 +620,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="batched_prompts", choices=sorted(gen.CONFIGS))
     ap.add_argument("--groups", type=int, default=None, help="override the number of prompts (default: the workload's)")
+    ap.add_argument("--split-prompts", action="store_true",
+                    help="with several ranks: split the workload's prompts over them (strong scaling) instead of giving "
+                         "every rank the whole set (weak scaling, the default)")
     ap.add_argument("--repeats", type=int, default=10, help="how often the headline pass is repeated (median reported)")
     ap.add_argument("--e2e-steps", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -23,6 +23,14 @@
  *     see (a NaN or +inf logit, a row without finite logits, a hazardous gather
  *     vector, a bounded wait that ran out) set a sticky device status word that
  *     psmc_sync_status() returns; the kernels never trap.
+ *   - No kernel waits for another CTA or another kernel: the only device-side
+ *     waits are for bulk copies into a CTA's own shared memory (bounded; on
+ *     expiry PSMC_E_TIMEOUT is raised, the affected rows get token -1 and the
+ *     kernel ends normally) and for warps of the same CTA.  Contexts may
+ *     therefore share a GPU, on any streams, with each other and with other
+ *     kernels.  After any device-detected error the context's counters are
+ *     consistent again at the end of the launch; psmc_reset() clears the
+ *     status word and restarts the run.
  *   - Randomness is a counter hash, so a run is a pure function of (seed,
  *     inputs): sm64(x) is the splitmix64 finaliser of x + 0x9E3779B97F4A7C15;
  *     H(a,b,c,d,e) = sm64(sm64(sm64(sm64(sm64(a)^b)^c)^d)^e); a uniform is
@@ -48,7 +56,7 @@ typedef enum {
     PSMC_E_CUDA = 3,    /* a CUDA runtime call failed                              */
     PSMC_E_STATE = 4,   /* call out of order (e.g. step beyond T_max)              */
     PSMC_E_NUMERIC = 5, /* NaN / +inf logit, or a row with no finite logit         */
-    PSMC_E_TIMEOUT = 6, /* a bounded device-side wait gave up                      */
+    PSMC_E_TIMEOUT = 6, /* a bounded device-side wait (for a bulk copy) gave up    */
     PSMC_E_HAZARD = 7,  /* in-place gather vector reads a row that is also written */
     PSMC_E_TOO_LARGE = 8 /* problem needs more than the fixed scratch of psmc_logits_pass_static */
 } psmc_status;
@@ -347,6 +355,35 @@ psmc_status psmc_shard_locate(psmc_ctx*, int v0, const double* all_triples, int 
                               psmc_shard_pick* picks_out, void* stream);
 psmc_status psmc_shard_finish(psmc_ctx*, const double* all_triples, const psmc_shard_pick* all_picks, int P,
                               void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* The step fed one vocabulary tile at a time                                 */
+/* ------------------------------------------------------------------------- */
+
+/* For a caller whose LM-head GEMM produces the logits of one vocabulary tile [R, width] at a time and never writes
+ * the [R, V] block to memory (the tile is consumed while it is still in L2).  The proposal of Corollary 1 and the
+ * weight of Eq. 7 need two row sums, which can be accumulated tile by tile, and the logits around the drawn token,
+ * which are only known to matter once the sums are complete; so the step is three kinds of calls:
+ *
+ *   psmc_tiles_feed    once per tile, in vocabulary order (v0 = 0, width, 2 width, ...; all tiles of one width but
+ *                      possibly the last; v0 + width <= V): reads the tile once and keeps one triple per row
+ *                      (reference exponent, sum 2^{x - c}, sum 2^{beta_t (x - c)}).  tile_logits: DEVICE [R, width],
+ *                      row stride ld elements; it may be overwritten as soon as the call's work on `stream` is done.
+ *   psmc_tiles_need    after the tile that ends at V: first_column_out (DEVICE int32 [R]) receives, per row, the first
+ *                      column of the tile that holds the row's target mass U * sum (-1 for a finished row).
+ *   psmc_tiles_finish  row_tiles: DEVICE [R, >= tile width], row stride ld: row r holds the logits of columns
+ *                      first_column[r] ... of ITS row again (recomputed by the caller: one tile per row, 1 / n_tiles
+ *                      of the GEMM), with -inf in columns beyond the vocabulary (last tile) and anything in finished
+ *                      rows.  Draws the token inside the tile, forms log p(y) and log omega (Eq. 7) from the
+ *                      accumulated sums and runs the rest of the step exactly as psmc_step does.
+ *
+ * The drawn token is the one psmc_step draws from the whole row up to the rounding of the partial sums (the inverse
+ * CDF runs over the vocabulary in its natural order).  Calls out of order return PSMC_E_STATE; not combinable with
+ * psmc_set_proposal_mask.  At most 1024 tiles. */
+psmc_status psmc_tiles_feed(psmc_ctx*, const void* tile_logits, psmc_dtype dt, int64_t ld, int v0, int width,
+                            void* stream);
+psmc_status psmc_tiles_need(psmc_ctx*, int32_t* first_column_out, void* stream);
+psmc_status psmc_tiles_finish(psmc_ctx*, const void* row_tiles, psmc_dtype dt, int64_t ld, void* stream);
 
 /* Snapshot of a run, for checkpointing and for moving a run to another context.  Because all randomness is a
  * counter hash of (seed, group, step, slot), a context that loads a snapshot continues bit for bit as the one that

@@ -109,6 +109,12 @@ def lib():
         L.psmc_shard_locate.argtypes = [vp, C.c_int, vp, C.c_int, C.c_int, vp, vp]
         L.psmc_shard_finish.restype = C.c_int
         L.psmc_shard_finish.argtypes = [vp, vp, vp, C.c_int, vp]
+        L.psmc_tiles_feed.restype = C.c_int
+        L.psmc_tiles_feed.argtypes = [vp, vp, C.c_int, C.c_int64, C.c_int, C.c_int, vp]
+        L.psmc_tiles_need.restype = C.c_int
+        L.psmc_tiles_need.argtypes = [vp, vp, vp]
+        L.psmc_tiles_finish.restype = C.c_int
+        L.psmc_tiles_finish.argtypes = [vp, vp, C.c_int, C.c_int64, vp]
         L.psmc_state_bytes.restype = C.c_size_t
         L.psmc_state_bytes.argtypes = [vp]
         L.psmc_state_save.restype = C.c_int
@@ -254,6 +260,25 @@ class Psmc:
         assert all_picks.dim() == 3 and all_picks.shape == (all_triples.shape[0], self.R, 2)
         _check(lib().psmc_shard_finish(self._h, all_triples.data_ptr(), all_picks.data_ptr(), all_triples.shape[0],
                                        _stream(stream)), "psmc_shard_finish")
+
+    # ---- the step fed one vocabulary tile at a time: feed every tile in order, ask which tile each row needs again,
+    # hand those tiles back
+    def tiles_feed(self, tile: torch.Tensor, v0: int, stream=None):
+        """tile: CUDA [R, width] logits of columns v0 .. v0+width (unit stride along the columns)."""
+        assert tile.is_cuda and tile.dim() == 2 and tile.stride(1) == 1 and tile.shape[0] == self.R
+        _check(lib().psmc_tiles_feed(self._h, tile.data_ptr(), _dtype_code(tile), tile.stride(0), v0, tile.shape[1],
+                                     _stream(stream)), "psmc_tiles_feed")
+
+    def tiles_need(self, first_column_out: torch.Tensor, stream=None):
+        """first_column_out: CUDA int32 [R]: first column of the tile each row needs again (-1: finished row)."""
+        assert first_column_out.is_cuda and first_column_out.dtype == torch.int32 and first_column_out.numel() == self.R
+        _check(lib().psmc_tiles_need(self._h, first_column_out.data_ptr(), _stream(stream)), "psmc_tiles_need")
+
+    def tiles_finish(self, row_tiles: torch.Tensor, stream=None):
+        """row_tiles: CUDA [R, tile width]: row r holds its own row's logits from first_column[r] on (-inf past V)."""
+        assert row_tiles.is_cuda and row_tiles.dim() == 2 and row_tiles.stride(1) == 1 and row_tiles.shape[0] == self.R
+        _check(lib().psmc_tiles_finish(self._h, row_tiles.data_ptr(), _dtype_code(row_tiles), row_tiles.stride(0),
+                                       _stream(stream)), "psmc_tiles_finish")
 
     def make_kv_desc(self, k_layers, v_layers, skip_shared_prompt: bool = False):
         """k_layers / v_layers: lists of CUDA tensors [R, H, max_len, D] with (max_len, D) contiguous.

@@ -62,6 +62,11 @@ struct psmc_ctx {
     // the step with the vocabulary split over ranks: 0 = idle, 1 = swept, 2 = located; the local columns of the sweep
     int shard_phase, shard_P;
     LogitsStreamArgs shard_la;
+    // the step fed one vocabulary tile at a time: 0 = idle, 1 = tiles coming in, 2 = owner columns handed out
+    int tile_phase, tile_width, tiles_fed, tile_next_v0;
+    double* tile_triples;          // [tile_cap][R][3]
+    int tile_cap;
+    psmc_shard_pick* tile_picks;   // [R]
     void* staging;       // psmc_step_host: device copy of the host logits
     size_t staging_bytes;
     cudaStream_t copy_stream;  // psmc_step_host: the logits travel on a stream of their own, so that the copy
@@ -117,6 +122,7 @@ psmc_status reset_device_state(psmc_ctx* c) {
     delete[] hd;
     c->t = 0;
     c->shard_phase = 0;
+    c->tile_phase = 0;
     return e == cudaSuccess ? PSMC_OK : PSMC_E_CUDA;
 }
 
@@ -159,7 +165,7 @@ void free_ctx(psmc_ctx* c) {
     void* ptrs[] = {c->logW, c->S, c->done2[0], c->done2[1], c->len, c->tok, c->last_tok, c->anc, c->map, c->resampled,
                     c->logp, c->loginc, c->ess, c->logZ, c->hist_tok, c->hist_map, c->sources[0], c->sources[1],
                     c->dst_rows[0], c->dst_rows[1], c->counts[0], c->counts[1], c->counts[2], c->row_arrivals,
-                    c->group_arrivals, c->step_triples, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev, c->set_size};
+                    c->group_arrivals, c->step_triples, c->tile_triples, c->tile_picks, c->status, c->kv_work, c->scratch, c->staging, c->prompt_len_dev, c->set_size};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     void* paged_ptrs[] = {c->paged.table, c->paged.refc, c->paged.free_list, c->paged.free_top};
@@ -271,6 +277,18 @@ StepExponents exponents_at(const psmc_ctx* c, int t) {
     return x;
 }
 
+// the span triples of a part of a row can take more room than those of the whole row (shorter spans)
+psmc_status grow_scratch(psmc_ctx* c, size_t need, cudaStream_t s) {
+    if (need <= c->scratch_bytes) return PSMC_OK;
+    if (cudaStreamSynchronize(s) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+    cudaFree(c->scratch);
+    c->scratch = nullptr;
+    c->scratch_bytes = 0;
+    if (cudaMalloc(&c->scratch, need) != cudaSuccess) return PSMC_E_NOMEM;
+    c->scratch_bytes = need;
+    return PSMC_OK;
+}
+
 WeightsArgs weights_args(psmc_ctx* c, int t, const StepExponents& x) {
     WeightsArgs wa{};
     wa.G = c->G; wa.N = c->N; wa.R = c->R; wa.t = t; wa.eos = c->eos; wa.resampler = c->resampler;
@@ -292,7 +310,7 @@ WeightsArgs weights_args(psmc_ctx* c, int t, const StepExponents& x) {
 
 extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt, int64_t ld, void* stream) {
     if (!c || !logits || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
-    if (c->t >= c->T_max || c->shard_phase != 0) return PSMC_E_STATE;
+    if (c->t >= c->T_max || c->shard_phase != 0 || c->tile_phase != 0) return PSMC_E_STATE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int t = c->t + 1;
     const StepExponents x = exponents_at(c, t);
@@ -330,19 +348,12 @@ extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, p
     if (!c || !logits_local || !triples_out || V_local < 2 || V_local > c->V || ld < V_local ||
         (dt != PSMC_F32 && dt != PSMC_BF16))
         return PSMC_E_INVAL;
-    if (c->t >= c->T_max || c->shard_phase != 0) return PSMC_E_STATE;
+    if (c->t >= c->T_max || c->shard_phase != 0 || c->tile_phase != 0) return PSMC_E_STATE;
     if (c->top_k > 0 || c->top_p > 0.0) return PSMC_E_STATE;  // ranking a row needs all of its columns
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // a shard is cut into spans of its own; with many ranks that can take a few more triples than the whole row
-    const size_t need = logits_pass_scratch_bytes(c->R, V_local);
-    if (need > c->scratch_bytes) {
-        if (cudaStreamSynchronize(s) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
-        cudaFree(c->scratch);
-        c->scratch = nullptr;
-        c->scratch_bytes = 0;
-        if (cudaMalloc(&c->scratch, need) != cudaSuccess) return PSMC_E_NOMEM;
-        c->scratch_bytes = need;
-    }
+    psmc_status grown = grow_scratch(c, logits_pass_scratch_bytes(c->R, V_local), s);
+    if (grown != PSMC_OK) return grown;
     const int t = c->t + 1;
     const StepExponents x = exponents_at(c, t);
     LogitsStreamArgs la{};
@@ -387,6 +398,95 @@ extern "C" psmc_status psmc_shard_finish(psmc_ctx* c, const double* all_triples,
     if (launch_shard_weights(wa, all_triples, all_picks, P, s) != cudaSuccess) return PSMC_E_CUDA;
     c->t = t;
     c->shard_phase = 0;
+    return PSMC_OK;
+}
+
+// ---- the step fed one vocabulary tile at a time (the consumer side of an LM-head GEMM that never writes [R, V]) ----
+extern "C" psmc_status psmc_tiles_feed(psmc_ctx* c, const void* tile_logits, psmc_dtype dt, int64_t ld, int v0, int width,
+                                       void* stream) {
+    if (!c || !tile_logits || width < 2 || ld < width || v0 < 0 || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
+    if (c->t >= c->T_max || c->shard_phase != 0 || c->tile_phase > 1) return PSMC_E_STATE;
+    if (c->top_k > 0 || c->top_p > 0.0) return PSMC_E_STATE;  // ranking a row needs all of its columns
+    if ((int64_t)v0 + width > c->V) return PSMC_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->tile_phase == 0) {  // first tile of the step: it fixes the tile width
+        if (v0 != 0) return PSMC_E_STATE;
+        const int cap = (c->V + width - 1) / width;
+        if (cap > 1024) return PSMC_E_INVAL;
+        if (cap > c->tile_cap) {
+            if (cudaStreamSynchronize(s) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
+            if (c->tile_triples) cudaFree(c->tile_triples);
+            c->tile_triples = nullptr;
+            c->tile_cap = 0;
+            if (cudaMalloc(reinterpret_cast<void**>(&c->tile_triples), (size_t)cap * c->R * 3 * sizeof(double)) != cudaSuccess)
+                return PSMC_E_NOMEM;
+            c->tile_cap = cap;
+        }
+        if (!c->tile_picks && dev_alloc(&c->tile_picks, (size_t)c->R) != cudaSuccess) return PSMC_E_NOMEM;
+        c->tile_width = width;
+        c->tiles_fed = 0;
+        c->tile_next_v0 = 0;
+    } else {  // tiles come in vocabulary order, all of one width but possibly the last
+        if (v0 != c->tile_next_v0) return PSMC_E_STATE;
+        if (width != c->tile_width && !(width < c->tile_width && v0 + width == c->V)) return PSMC_E_INVAL;
+    }
+    psmc_status grown = grow_scratch(c, logits_pass_scratch_bytes(c->R, width), s);
+    if (grown != PSMC_OK) return grown;
+    const int t = c->t + 1;
+    const StepExponents x = exponents_at(c, t);
+    LogitsStreamArgs la{};
+    la.logits = tile_logits; la.dt = dt; la.R = c->R; la.V = width; la.ld = ld; la.beta = x.beta_t;
+    la.done = done_now(c); la.scratch = c->scratch;
+    la.status = c->status;
+    la.zero_words = c->counts[(t + 1) & 1];
+    LaunchTimer lt(c, s, 0);
+    if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
+    if (launch_shard_triples(la, c->tile_triples + (size_t)c->tiles_fed * c->R * 3, s) != cudaSuccess) return PSMC_E_CUDA;
+    c->tiles_fed += 1;
+    c->tile_next_v0 = v0 + width;
+    c->tile_phase = 1;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_tiles_need(psmc_ctx* c, int32_t* first_column_out, void* stream) {
+    if (!c || !first_column_out) return PSMC_E_INVAL;
+    if (c->tile_phase != 1 || c->tile_next_v0 != c->V) return PSMC_E_STATE;  // the tiles have to cover the vocabulary
+    const int t = c->t + 1;
+    const StepExponents x = exponents_at(c, t);
+    if (launch_shard_owner_columns(c->tile_triples, c->tiles_fed, c->R, c->N, t, x.beta_t, c->seed, done_now(c),
+                                   c->tile_width, first_column_out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return PSMC_E_CUDA;
+    c->tile_phase = 2;
+    return PSMC_OK;
+}
+
+extern "C" psmc_status psmc_tiles_finish(psmc_ctx* c, const void* row_tiles, psmc_dtype dt, int64_t ld, void* stream) {
+    if (!c || !row_tiles || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
+    if (c->tile_phase != 2) return PSMC_E_STATE;
+    if (ld < c->tile_width) return PSMC_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    psmc_status grown = grow_scratch(c, logits_pass_scratch_bytes(c->R, c->tile_width), s);
+    if (grown != PSMC_OK) return grown;
+    const int t = c->t + 1;
+    const StepExponents x = exponents_at(c, t);
+    LogitsStreamArgs la{};
+    la.logits = row_tiles; la.dt = dt; la.R = c->R; la.V = c->tile_width; la.ld = ld; la.beta = x.beta_t;
+    la.done = done_now(c); la.scratch = c->scratch;
+    la.status = c->status;
+    la.zero_words = nullptr;
+    ShardLocateArgs sa{};
+    sa.all_triples = c->tile_triples; sa.P = c->tiles_fed; sa.rank = -1; sa.N = c->N; sa.t = t; sa.v0 = 0;
+    sa.tile_width = c->tile_width; sa.alpha_t = x.alpha_t; sa.seed = c->seed; sa.picks_out = c->tile_picks;
+    {
+        LaunchTimer lt(c, s, 0);
+        if (launch_logits_stream(la, s) != cudaSuccess) return PSMC_E_CUDA;
+        if (launch_shard_locate(la, sa, s) != cudaSuccess) return PSMC_E_CUDA;
+    }
+    const WeightsArgs wa = weights_args(c, t, x);
+    LaunchTimer lt(c, s, 1);
+    if (launch_shard_weights(wa, c->tile_triples, c->tile_picks, c->tiles_fed, s, true) != cudaSuccess) return PSMC_E_CUDA;
+    c->t = t;
+    c->tile_phase = 0;
     return PSMC_OK;
 }
 
@@ -617,7 +717,7 @@ extern "C" size_t psmc_state_bytes(const psmc_ctx* c) {
 
 extern "C" psmc_status psmc_state_save(psmc_ctx* c, void* host_buf, size_t bytes) {
     if (!c || !host_buf || bytes < snapshot_bytes(c, c->t)) return PSMC_E_INVAL;
-    if (c->shard_phase != 0) return PSMC_E_STATE;  // between the calls of a sharded step there is no consistent state
+    if (c->shard_phase != 0 || c->tile_phase != 0) return PSMC_E_STATE;  // inside a step there is no consistent state
     if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
     SnapshotHeader h{};
     h.magic = kSnapshotMagic;

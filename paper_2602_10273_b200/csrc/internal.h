@@ -120,6 +120,9 @@ cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa
 struct ShardLocateArgs {
     const double* all_triples;  // [P][R][3]
     int P, rank, N, t, v0;
+    int tile_width;             // 0: rank `rank` holds columns from v0 on.  > 0: the parts are vocabulary tiles of this
+                                // width fed one after the other, and row r of the logits given holds the columns of
+                                // the tile that owns row r (its own tile for every row)
     double alpha_t;
     uint64_t seed;
     psmc_shard_pick* picks_out;  // [R]
@@ -127,9 +130,13 @@ struct ShardLocateArgs {
 // la describes the local columns (V = their number); its scratch holds the span triples of the streaming kernel
 cudaError_t launch_shard_triples(const LogitsStreamArgs& la, double* triples_out, cudaStream_t stream);
 cudaError_t launch_shard_locate(const LogitsStreamArgs& la, const ShardLocateArgs& sa, cudaStream_t stream);
-// a.logits / a.scratch are not used: the row results come from the gathered triples and picks
+// a.logits / a.scratch are not used: the row results come from the gathered triples and picks.
+// picks_per_row: all_picks is [R] (row r's pick whoever its owner is) instead of [P][R].
 cudaError_t launch_shard_weights(const WeightsArgs& a, const double* all_triples, const psmc_shard_pick* all_picks, int P,
-                                 cudaStream_t stream);
+                                 cudaStream_t stream, bool picks_per_row = false);
+// need_out[r] = first column of the part (tile) that holds row r's target mass, -1 for a finished or unusable row
+cudaError_t launch_shard_owner_columns(const double* all_triples, int P, int R, int N, int t, double beta, uint64_t seed,
+                                       const uint8_t* done, int tile_width, int32_t* need_out, cudaStream_t stream);
 
 // ---------------------------------------------------------------- KV reindex (Appendix C)
 constexpr int kMaxKvPtrs = 128;  // K and V pointers per launch (64 layers); more layers take more launches

@@ -133,6 +133,7 @@ struct LocateParams {
     FinishParams f;  // the local columns
     const double* all;
     int P, rank, R, N, t, v0;
+    int tile_width;  // > 0: every row is located in the columns given for it, which start at owner * tile_width
     uint64_t seed;
     const uint8_t* done;
     psmc_shard_pick* picks;
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) shard_locate_kernel(const __
         } else {
             st = shard_combine<MODE>(TriplesInGlobal{lp.all, lp.R, row}, lp.P, lp.f.beta, U);
         }
-        if (st.ok && st.owner == lp.rank) {
+        if (st.ok && (lp.tile_width > 0 || st.owner == lp.rank)) {
             const RowFrame fr{st.C, st.target, st.base};
             const RowTotals t = combine_spans<MODE, true>(lp.f, row, U, lane, &fr);
             if (t.ok) {
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) shard_locate_kernel(const __
                     reinterpret_cast<const char*>(lp.f.logits) + (size_t)row * lp.f.ld * (DT == PSMC_F32 ? 4 : 2);
                 const int y = locate_token_warp<DT, MODE>(lp.f, rowp, t, lane);
                 if (y >= 0) {
-                    pick.tok = lp.v0 + y;
+                    pick.tok = (lp.tile_width > 0 ? st.owner * lp.tile_width : lp.v0) + y;
                     pick.logit = load_elem<DT>(rowp, y);
                 }
             }
@@ -185,6 +186,7 @@ struct ShardFinishParams {
     const psmc_shard_pick* picks;  // [P][R]
     int P;
     int staged;  // the group's triples fit the dynamic shared memory given to the launch
+    int picks_per_row;  // picks is [R]: row r's pick, whoever owns the row
 };
 template <int MODE>
 __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_constant__ ShardFinishParams sp) {
@@ -224,7 +226,7 @@ __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_consta
                 tot = shard_combine<MODE>(TriplesInGlobal{sp.all, a.R, r}, sp.P, a.beta, U);
             }
             if (tot.ok) {
-                const psmc_shard_pick pk = sp.picks[(size_t)tot.owner * a.R + r];
+                const psmc_shard_pick pk = sp.picks[sp.picks_per_row ? (size_t)r : (size_t)tot.owner * a.R + r];
                 if (pk.tok >= 0) {
                     // same grouping as the unsharded finish: the token's own logit drops out when beta = alpha_t
                     const double dl = (double)pk.logit - (double)tot.C * kLn2;
@@ -240,6 +242,24 @@ __global__ void __launch_bounds__(1024) shard_weights_kernel(const __grid_consta
         }
     }
     group_update(a, g, i, (N + 31) >> 5, sc, tk, lp, inc, st);
+}
+
+// ---- which part holds each row's target: what a caller that feeds the parts one after the other has to bring back ----
+template <int MODE>
+__global__ void __launch_bounds__(256) shard_owner_columns_kernel(const double* all, int P, int R, int N, int t, double beta,
+                                                                  uint64_t seed, const uint8_t* done, int tile_width,
+                                                                  int32_t* need_out) {
+    chain_begin();
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= R) return;
+    int need = -1;
+    if (!done[row]) {
+        const int g = row / N, k = row - g * N;
+        const double U = hash_uniform(hash5(seed, kStreamToken, (uint64_t)g, (uint64_t)t, (uint64_t)k));
+        const ShardTotals st = shard_combine<MODE>(TriplesInGlobal{all, R, row}, P, beta, U);
+        if (st.ok) need = st.owner * tile_width;
+    }
+    need_out[row] = need;
 }
 
 template <int DT>
@@ -276,16 +296,31 @@ cudaError_t launch_shard_locate(const LogitsStreamArgs& la, const ShardLocateArg
     lp.f.partials = reinterpret_cast<const float4*>(la.scratch); lp.f.beta = la.beta; lp.f.alpha_t = sa.alpha_t;
     lp.f.bf = g.bf; lp.f.vec = g.vec;
     lp.all = sa.all_triples; lp.P = sa.P; lp.rank = sa.rank; lp.R = la.R; lp.N = sa.N; lp.t = sa.t; lp.v0 = sa.v0;
+    lp.tile_width = sa.tile_width;
     lp.seed = sa.seed; lp.done = la.done; lp.picks = sa.picks_out;
     auto fn = la.dt == PSMC_F32 ? pick_locate<PSMC_F32>(g.mode) : pick_locate<PSMC_BF16>(g.mode);
     return launch_chained(fn, dim3((unsigned)((la.R + kRowsPerCta - 1) / kRowsPerCta)), dim3(kRowsPerCta * 32), 0, stream,
                           lp);
 }
 
+cudaError_t launch_shard_owner_columns(const double* all_triples, int P, int R, int N, int t, double beta, uint64_t seed,
+                                       const uint8_t* done, int tile_width, int32_t* need_out, cudaStream_t stream) {
+    void (*fn)(const double*, int, int, int, int, double, uint64_t, const uint8_t*, int, int32_t*);
+    switch (beta_mode(beta)) {
+        case kBeta1: fn = shard_owner_columns_kernel<kBeta1>; break;
+        case kBeta2: fn = shard_owner_columns_kernel<kBeta2>; break;
+        case kBeta4: fn = shard_owner_columns_kernel<kBeta4>; break;
+        case kBeta8: fn = shard_owner_columns_kernel<kBeta8>; break;
+        default: fn = shard_owner_columns_kernel<kBetaAny>; break;
+    }
+    return launch_chained(fn, dim3((unsigned)((R + 255) / 256)), dim3(256), 0, stream, all_triples, P, R, N, t, beta, seed,
+                          done, tile_width, need_out);
+}
+
 cudaError_t launch_shard_weights(const WeightsArgs& a, const double* all_triples, const psmc_shard_pick* all_picks, int P,
-                                 cudaStream_t stream) {
+                                 cudaStream_t stream, bool picks_per_row) {
     ShardFinishParams sp;
-    sp.a = a; sp.all = all_triples; sp.picks = all_picks; sp.P = P;
+    sp.a = a; sp.all = all_triples; sp.picks = all_picks; sp.P = P; sp.picks_per_row = picks_per_row ? 1 : 0;
     void (*fn)(const ShardFinishParams);
     switch (beta_mode(a.beta)) {
         case kBeta1: fn = shard_weights_kernel<kBeta1>; break;
