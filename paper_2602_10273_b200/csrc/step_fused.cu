@@ -194,6 +194,12 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
     const PackedConsts kc = packed_consts(sp.f.bf);
     const int W = sp.g.W;
 
+    // The block is read once: its lines go into L2 marked evict-first, so that the sweep recycles its own lines instead
+    // of pushing out what the kernel before left there (the dirty lines of a cache move would otherwise be written back
+    // under this sweep: measured 48.8 -> 46.1 us per step inside the decoding loop, and 2 us per step less overall).
+    // The segment streamed last keeps the normal priority: one piece of it is read again when the row is finished.
+    const uint64_t policy = l2_policy_evict_first();
+    const int hint_until = S - 1;
     // producer cursor (the same in every lane; lane 0 issues)
     int pk = 0, p_left = 0;
     const char* p_src = nullptr;
@@ -215,7 +221,8 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
             const int slot = issued & (kDepth - 1);
             fence_async_smem();  // the stage's previous contents were read through the generic proxy
             mbar_expect_tx(&full[slot], (uint32_t)bytes);
-            bulk_load(ring + (size_t)slot * kStageBytes, p_src, (uint32_t)bytes, &full[slot]);
+            if (pk < hint_until) bulk_load_hint(ring + (size_t)slot * kStageBytes, p_src, (uint32_t)bytes, &full[slot], policy);
+            else bulk_load(ring + (size_t)slot * kStageBytes, p_src, (uint32_t)bytes, &full[slot]);
         }
         ++issued;
         p_src += bytes;
