@@ -235,6 +235,16 @@ def test_closed_loop_random_settings():
         assert st.steps == 12
 
 
+@pytest.mark.parametrize("G,N,V,dtype", [(300, 8, 104, "bf16"), (330, 8, 2048, "bf16"), (1000, 8, 16, "f32"), (40, 32, 1000, "f32")])
+def test_closed_loop_many_rows_per_cta(G, N, V, dtype):
+    """Shapes whose logit block gives every CTA of the one-kernel step many short rows: 16-18 segments per CTA (beyond
+    the fifteen named barriers: the helper polls mbarriers instead), rows of a few granules split over two CTAs, and
+    54 rows per CTA (beyond the segment table: the step runs as two kernels)."""
+    c = W.Workload("many", G, N, V, dtype, 3.0, 1.5, 6, 2, 5, 4.0, 0.25, 0.7, 0, 1, 1, 8, 16)
+    st = P.closed_loop(c, seed=5, T=6, kv_shape=(1, 1, 16, 8))
+    assert st.steps == 6 and st.resample_events > 0
+
+
 def test_closed_loop_llama_shape():
     c = W.CONFIGS["llama2_7b"]
     st = P.closed_loop(c, seed=1, T=96, kv_shape=(2, 4, 512 + 96 + 8, c.head_dim))
