@@ -543,6 +543,9 @@ extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, con
         if (dst->stride_head < min_head || dst->stride_row < (int64_t)dst->n_kv_heads * dst->stride_head)
             return PSMC_E_INVAL;
     }
+    // the copy kernels number their work units in an int
+    const int ptrs_per_launch = 2 * (src->n_layers < kMaxKvPtrs / 2 ? src->n_layers : kMaxKvPtrs / 2);
+    if ((int64_t)c->R * ptrs_per_launch * src->n_kv_heads * reindex_unit_parts() >= ((int64_t)1 << 31)) return PSMC_E_INVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int set = idx_override ? 1 : 0;
     if (idx_override) {

@@ -159,6 +159,7 @@ struct KvLaunch {
     int bulk_ok;     // 16-byte alignment holds everywhere
 };
 cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream);
+int reindex_unit_parts();  // work units per (source row, tensor, head): rows * pointers * heads * this must stay below 2^31
 // turn an arbitrary gather vector into move records (and check in-place hazards)
 cudaError_t launch_build_moves(const int32_t* idx, int R, int max_len, int in_place, MoveSource* sources,
                                int32_t* dst_rows, int32_t* n_sources, int32_t* n_moves, int32_t* status,

@@ -383,7 +383,7 @@ __device__ __forceinline__ bool stream_tasks(const StreamParams& p, unsigned cha
         __syncwarp();  // every lane is done with the stage that is about to be refilled
         issue();
         const int slot = consumed % kDepth;
-        if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // uniform verdict
+        if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // the same answer in every lane
             failed = true;
             break;
         }

@@ -22,10 +22,13 @@ namespace {
 constexpr int kChunk = 16384;   // bytes per stage
 constexpr int kStages = 4;
 constexpr int kBulkCtasPerSm = 3;
-// Work is handed out in units of one (source record, pointer/head segment): the live prefix of one head of one
-// K or V tensor of one surviving row.  Lengths differ from row to row, so a static deal of fixed-size pieces
-// leaves CTAs with unequal loads; instead every CTA takes the next unit from a global counter when it runs
-// out (the fetch of the unit after that is already in flight, so its latency stays off the copy pipeline).
+constexpr int kUnitParts = 4;   // a (source, tensor, head) segment is handed out in this many parts (whole chunks each)
+// Work is handed out in units of a quarter of one (source record, pointer/head segment): the live prefix of one head
+// of one K or V tensor of one surviving row, cut at chunk boundaries.  Lengths differ from row to row, so a static
+// deal of fixed-size pieces leaves CTAs with unequal loads; instead every CTA takes the next unit from a global
+// counter when it runs out (the fetch of the unit after that is already in flight, so its latency stays off the copy
+// pipeline).  The last unit a CTA draws is what the others wait for at the end of the kernel: with whole segments
+// (180 KB at 700 positions, read once and written 2-3 times) that tail was 4-5 % of the kernel.
 // A unit is streamed in chunks of kChunk bytes.
 struct Item {
     const char* src;
@@ -41,7 +44,8 @@ struct UnitCursor {
     int64_t off;         // next byte to hand out
 };
 __device__ __forceinline__ void open_unit(const KvLaunch& k, int u, int n_seg, UnitCursor& c) {
-    const int s = u / n_seg, seg = u - s * n_seg;
+    const int part = u % kUnitParts, us = u / kUnitParts;
+    const int s = us / n_seg, seg = us - s * n_seg;
     const MoveSource ms = k.sources[s];
     const int len = ms.len < k.max_len ? ms.len : k.max_len;
     int skip = k.skip_pos ? k.skip_pos[ms.src_row / k.N] : 0;  // a prompt shared by the group stays where it is
@@ -51,8 +55,12 @@ __device__ __forceinline__ void open_unit(const KvLaunch& k, int u, int n_seg, U
     c.dst_begin = ms.dst_begin;
     c.n_dst = ms.n_dst;
     c.src = k.src[c.seg_ptr] + (int64_t)ms.src_row * k.row_bytes_stride + (int64_t)c.seg_head * k.head_bytes_stride;
-    c.seg_bytes = (int64_t)(len > 0 ? len : 0) * k.pos_bytes;
-    c.off = (int64_t)skip * k.pos_bytes;
+    // the part's share of [skip, len): whole chunks, the last part takes the ragged end
+    const int64_t lo = (int64_t)skip * k.pos_bytes, hi = (int64_t)(len > 0 ? len : 0) * k.pos_bytes;
+    const int64_t chunks = (hi - lo + kChunk - 1) / kChunk, per_part = (chunks + kUnitParts - 1) / kUnitParts;
+    const int64_t p_lo = lo + (int64_t)part * per_part * kChunk, p_hi = p_lo + per_part * kChunk;
+    c.off = p_lo < hi ? p_lo : hi;
+    c.seg_bytes = p_hi < hi ? p_hi : hi;  // the cursor runs from off to seg_bytes
 }
 __device__ __forceinline__ void take_chunk(UnitCursor& c, Item& it) {
     it.src = c.src + c.off;
@@ -94,7 +102,7 @@ __global__ void __launch_bounds__(32) reindex_bulk_kernel(const __grid_constant_
     fence_async_smem();
 
     const int n_seg = k.n_ptrs * k.H;
-    const int n_units = n_src * n_seg;   // < 2^31: rows <= 2^24 is checked at init, and segments per launch <= 128 * H
+    const int n_units = n_src * n_seg * kUnitParts;   // < 2^31: checked by the host (rows, pointers and heads per launch)
 
     // unit queue: `next_u` is always one fetch ahead of the unit being streamed
     UnitCursor cur;
@@ -159,7 +167,7 @@ __global__ void __launch_bounds__(256) reindex_plain_kernel(const __grid_constan
     const int n_src = *reinterpret_cast<const volatile int32_t*>(k.n_sources);
     if (n_src <= 0) return;
     const int n_seg = k.n_ptrs * k.H;
-    const int n_units = n_src * n_seg;
+    const int n_units = n_src * n_seg * kUnitParts;
     for (;;) {
         __syncthreads();  // everyone has read the previous sh_u
         if (threadIdx.x == 0) sh_u = atomicAdd(k.work, 1);
@@ -227,6 +235,8 @@ __global__ void __launch_bounds__(1024) build_moves_kernel(const int32_t* idx, i
 }
 
 }  // namespace
+
+int reindex_unit_parts() { return kUnitParts; }
 
 cudaError_t launch_reindex_kv(const KvLaunch& k, cudaStream_t stream) {
     if (k.bulk_ok) {

@@ -249,7 +249,7 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
             __syncwarp();  // every lane is done with the stage that is about to be refilled
             issue();
             const int slot = consumed & (kDepth - 1);
-            if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // uniform verdict
+            if (!__all_sync(kFull, mbar_wait(&full[slot], (uint32_t)((consumed / kDepth) & 1)))) {  // the same answer in every lane
                 failed = true;
                 break;
             }
