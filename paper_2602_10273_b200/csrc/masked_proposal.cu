@@ -96,10 +96,27 @@ __device__ __forceinline__ uint32_t load_bits(const void* rowp, int i) {
     return __ldg(reinterpret_cast<const unsigned short*>(rowp) + i);
 }
 
-// Two bf16 logits in one word -> their two keys in one word (the -0 adjustment of key_of left out: such a key is one
-// too low, which the callers allow for).
-__device__ __forceinline__ uint32_t keys_of_pair(uint32_t w) {
-    return w ^ ((((w >> 15) & 0x00010001u) * 0xffffu) | 0x80008000u);
+// Two bf16 logits in one word, handled by the packed bf16 instructions.  The maximum is the NaN-propagating one (a
+// NaN of either sign anywhere in a share makes the share's maximum a NaN, whose key ranks above +inf's); +0 and -0
+// compare equal, as their keys do.
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) {
+    __nv_bfloat162 r;
+    *reinterpret_cast<uint32_t*>(&r) = w;
+    return r;
+}
+__device__ __forceinline__ uint32_t max_nan_pair(uint32_t a, uint32_t b) {
+    const __nv_bfloat162 m = __hmax2_nan(as_bf162(a), as_bf162(b));
+    return *reinterpret_cast<const uint32_t*>(&m);
+}
+// 0xffff in each half of the word whose logit is >= the threshold's (no NaN on either side)
+__device__ __forceinline__ uint32_t ge_pair(uint32_t w, uint32_t th2) { return __hge2_mask(as_bf162(w), as_bf162(th2)); }
+// the bf16 pattern (in both halves of a word) that compares like `key`: every logit with a key >= key is >= it
+__device__ __forceinline__ uint32_t pair_threshold(uint32_t key) {
+    constexpr uint32_t kNegInfKey = 0x007fu;
+    const uint32_t k = key < kNegInfKey ? kNegInfKey : key;  // below -inf's key: everything passes
+    const uint32_t sign = 0x8000u;
+    const uint32_t b = (k & sign) ? (k ^ sign) : (~k & 0xffffu);
+    return b | (b << 16);
 }
 
 // The row in no particular order: fv(v, id of its first logit) for every aligned 16 bytes between the first and the
@@ -360,30 +377,27 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
 #pragma unroll
     for (int j = 0; j < kSub; ++j) sub[j] = 0u;
     if (DT == PSMC_BF16 && (by_threshold || by_floor)) {  // nothing to count: two keys at a time, packed maxima and minima
-        uint32_t mx2[4] = {0u, 0u, 0u, 0u}, mn2 = 0xffffffffu;
+        constexpr uint32_t kNegInf2 = 0xff80ff80u;
+        uint32_t mx2[4] = {kNegInf2, kNegInf2, kNegInf2, kNegInf2};
         for_each_vector<DT>(
             rowp, V,
             [&](const uint4& v, int) {
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t k2 = keys_of_pair(w[c]);
-                    mx2[c] = __vmaxu2(mx2[c], k2);
-                    mn2 = __vminu2(mn2, k2);
-                }
+                mx2[0] = max_nan_pair(mx2[0], v.x);
+                mx2[1] = max_nan_pair(mx2[1], v.y);
+                mx2[2] = max_nan_pair(mx2[2], v.z);
+                mx2[3] = max_nan_pair(mx2[3], v.w);
             },
             [&](uint32_t b, int) {
-                const uint32_t key = keys_of_pair(b) & 0xffffu;
+                const uint32_t key = key_of<DT>(b);
                 kmax = max(kmax, key);
                 kmin = min(kmin, key);
             });
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            sub[(2 * c) % kSub] = mx2[c] & 0xffffu;
-            sub[(2 * c + 1) % kSub] = mx2[c] >> 16;
+        for (int c = 0; c < 4; ++c) {  // (a NaN maximum has the sign bit clear: its key ranks above +inf's)
+            sub[(2 * c) % kSub] = key_of<DT>(mx2[c] & 0xffffu);
+            sub[(2 * c + 1) % kSub] = key_of<DT>(mx2[c] >> 16);
         }
         sub[0] = max(sub[0], kmax);  // the ragged ends join the first sub-share
-        kmin = min(kmin, min(mn2 & 0xffffu, mn2 >> 16));
     } else if (by_threshold) {
         for_each_vector<DT>(
             rowp, V,
@@ -452,6 +466,19 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         if (pos < kListCap) list[pos] = ((unsigned long long)(uint32_t)i << 32) | b;
     };
 
+    // the logits of one 16-byte vector (bf16) that are >= the threshold's go to the list: one test for all eight first
+    auto collect8 = [&](const uint32_t (&w)[4], int i0, uint32_t th2) {
+        const uint32_t g0 = ge_pair(w[0], th2), g1 = ge_pair(w[1], th2), g2 = ge_pair(w[2], th2), g3 = ge_pair(w[3], th2);
+        if ((g0 | g1) | (g2 | g3)) {
+            const uint32_t ge[4] = {g0, g1, g2, g3};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (ge[c] & 0xffffu) append(w[c] & 0xffffu, i0 + 2 * c);
+                if (ge[c] >> 16) append(w[c] >> 16, i0 + 2 * c + 1);
+            }
+        }
+    };
+
     if (by_threshold) {
         // ---- the threshold: the k-th largest of the threads' maxima, by the same digit search on a plain histogram ----
         if (threadIdx.x == 0) {
@@ -474,30 +501,22 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         const uint32_t theta = thr.prefix;
         // ---- sweep 2: the normaliser of p, and every logit at or above the threshold into the list ----
         if (DT == PSMC_BF16) {
-            // packed keys lack the -0 adjustment (one too low for -0), and so may the threshold: compare against one
-            // below +0's key when the threshold is +0's, so that either zero passes
-            constexpr uint32_t kZero = 0x8000u;
-            const uint32_t th = theta == kZero ? kZero - 1u : theta, th2 = th | (th << 16);
+            const uint32_t th2 = pair_threshold(theta);
             for_each_vector<DT>(
                 rowp, V,
                 [&](const uint4& v, int i0) {
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
                     float part = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 4; ++c)
                         part += ex2(rel_exponent(__uint_as_float(w[c] << 16), neg_C)) +
                                 ex2(rel_exponent(__uint_as_float(w[c] & 0xffff0000u), neg_C));
-                        const uint32_t ge = __vcmpgeu2(keys_of_pair(w[c]), th2);
-                        if (ge) {
-                            if (ge & 0xffffu) append(w[c] & 0xffffu, i0 + 2 * c);
-                            if (ge >> 16) append(w[c] >> 16, i0 + 2 * c + 1);
-                        }
-                    }
                     s1 += (double)part;
+                    collect8(w, i0, th2);
                 },
                 [&](uint32_t b, int i) {
                     s1 += (double)ex2(rel_exponent(value_of<DT>(b), neg_C));
-                    if ((keys_of_pair(b) & 0xffffu) >= th) append(b, i);
+                    if (key_of<DT>(b) >= theta) append(b, i);
                 });
         } else {
             float part = 0.f;
@@ -554,22 +573,15 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
                                    : (DT == PSMC_BF16 ? key32 >> 16 : key32);
         // ---- sweep 3: the tokens at or above the floor into the list ----
         if (DT == PSMC_BF16) {
-            const uint32_t th = floor_key > 0u ? floor_key - 1u : 0u, th2 = th | (th << 16);  // packed keys may be one low
+            const uint32_t th2 = pair_threshold(floor_key);
             for_each_vector<DT>(
                 rowp, V,
                 [&](const uint4& v, int i0) {
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const uint32_t ge = __vcmpgeu2(keys_of_pair(w[c]), th2);
-                        if (ge) {
-                            if (ge & 0xffffu) append(w[c] & 0xffffu, i0 + 2 * c);
-                            if (ge >> 16) append(w[c] >> 16, i0 + 2 * c + 1);
-                        }
-                    }
+                    collect8(w, i0, th2);
                 },
                 [&](uint32_t b, int i) {
-                    if ((keys_of_pair(b) & 0xffffu) >= th) append(b, i);
+                    if (key_of<DT>(b) >= floor_key) append(b, i);
                 });
         } else {
             for_each_logit<DT>(rowp, V, [&](uint32_t b, int i) {
