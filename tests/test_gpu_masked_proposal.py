@@ -90,6 +90,39 @@ def test_signed_zeros_and_masked_columns():
         assert st.steps == 6
 
 
+@pytest.mark.parametrize("rule", [dict(top_k=5), dict(top_k=3000), dict(top_p=0.9), dict(top_p=1.0)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_rows_with_nan_or_inf_are_flagged(rule, dtype):
+    """A NaN of either sign or a +inf anywhere in a row (inside the 16-byte vectors or at the ragged ends; the bf16
+    sweeps take maxima two logits at a time) makes the row unusable: token -1, PSMC_E_NUMERIC, the other rows as usual.
+    A row of -inf only has nothing to draw from either."""
+    V, N = 4099, 8
+    as_int = torch.int16 if dtype == torch.bfloat16 else torch.int32
+    bads = [(1, 0, float("nan")), (2, 1001, "-nan"), (3, 2222, float("inf")), (4, V - 1, float("nan")),
+            (5, V - 2, "-nan"), (6, 7, float("inf"))]
+    for row, col, val in bads:
+        ps = B.Psmc(N, V, 4.0, 0.25, 0.5, 0, 11, V - 1, T_max=2)
+        ps.set_proposal_mask(**rule)
+        lg = (torch.randn(N, V + 3, device="cuda") * 2.0).to(dtype)[:, 1:V + 1]   # rows start off a 16-byte boundary
+        if val == "-nan":
+            lg.view(as_int)[row, col] = -1                                         # all bits set: a NaN with the sign bit
+            assert bool(torch.isnan(lg[row, col]))
+        else:
+            lg[row, col] = val
+        ps.step(lg)
+        assert ps.sync_status() == B.E_NUMERIC
+        tok = ps.tokens.numpy()
+        assert tok[row] == -1 or tok[row] == V - 1    # (the group update maps a flagged row's token to a valid id)
+        ps.destroy()
+    ps = B.Psmc(N, V, 4.0, 0.25, 0.5, 0, 11, V - 1, T_max=2)
+    ps.set_proposal_mask(**rule)
+    lg = (torch.randn(N, V, device="cuda") * 2.0).to(dtype)
+    lg[3] = float("-inf")
+    ps.step(lg)
+    assert ps.sync_status() == B.E_NUMERIC
+    ps.destroy()
+
+
 def test_support_sizes_and_the_tokens_outside_it():
     """Every drawn token is among the row's top_k; the reported size is min(top_k, V)."""
     cfg = W.CONFIGS["llama2_7b"]
