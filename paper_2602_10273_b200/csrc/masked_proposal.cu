@@ -762,7 +762,9 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         }
         if (y < 0) y = last;
         const double dl = (double)load_elem<DT>(rowp, y) - (double)C * kLn2;
-        const double ln_s1 = log(S1), ln_sb = log(Sb);
+        double add_s1, add_sb;
+        ln_sum_corrections<MODE>(p.beta, add_s1, add_sb);  // both sums are made of ex2 terms, on the list as on the row
+        const double ln_s1 = log(S1) + add_s1, ln_sb = log(Sb) + add_sb;
         p.tok[row] = y;
         p.logp[row] = dl - ln_s1;
         p.loginc[row] = (p.alpha_t - p.beta) * dl - p.alpha_t * ln_s1 + ln_sb;

@@ -50,6 +50,21 @@ def test_batched_prompts_full_width_sixty_four_tokens():
     _report("batched_prompts, 64 prompts, T = 64", st)
 
 
+@pytest.mark.parametrize("rule", [dict(top_k=50), dict(top_p=0.9)])
+def test_restricted_proposals_over_three_thousand_tokens(rule):
+    """The fast exponential returns its values low by 5e-8 of the value on average, every sum of such terms is low by
+    that fraction, and log p(y_{1:t}) adds the same error at every token: 1.5e-4 after 3000 tokens unless the kernels
+    take it out.  The restricted proposals form their sums in a kernel of their own."""
+    c = W.Workload("restricted_long", 1, 8, 4096, "bf16", 3.0, 1.5, 3000, 4, 4, 4.0, 0.25, 0.5, 0, 1, 1, 8, 3008)
+
+    def no_eos(t, lg):          # keep the particles alive to the end
+        lg[:, c.eos_id] = -40.0
+
+    st = P.closed_loop(c, seed=3, T=c.T, logit_bias_fn=no_eos, **rule)
+    assert st.steps == c.T and st.live_rows == c.T * c.N and st.resample_events > 0
+    _report("restricted_long %r, T = %d" % (rule, c.T), st)
+
+
 @pytest.mark.parametrize("N,V,T,kappa", [(33, 64, 300, 0.9), (1024, 32, 9, 1.0), (8, 50, 1200, 0.7)])
 def test_back_trace_over_several_batches(N, V, T, kappa):
     """The output step stages its ancestry log in batches of 4096 integers; T * N beyond that takes several batches.
