@@ -65,6 +65,45 @@ def test_restricted_proposals_over_three_thousand_tokens(rule):
     _report("restricted_long %r, T = %d" % (rule, c.T), st)
 
 
+def _long_small(name, N=8, dtype="bf16", alpha=4.0, tau=0.25, T=3000):
+    return W.Workload(name, 1, N, 4096, dtype, 3.0, 1.5, T, 4, 4, alpha, tau, 0.5, 0, 1, 1, 8, T + 8)
+
+
+def _no_eos(c):
+    def edit(t, lg):            # keep the particles alive to the end
+        lg[:, c.eos_id] = -40.0
+    return edit
+
+
+@pytest.mark.parametrize("label,kw", [("fp32 logits", dict(dtype="f32")),
+                                      ("beta = 3 (no squaring)", dict(alpha=3.0, tau=1.0 / 3.0)),
+                                      ("beta = 2", dict(alpha=2.0, tau=0.5)),
+                                      ("33 particles (the step as two kernels)", dict(N=33, T=2000))])
+def test_other_forms_of_the_step_over_thousands_of_tokens(label, kw):
+    """The same horizon for the forms of the logit pass the named configurations do not reach: fp32 logits, an
+    exponent that is not a power of two, groups too large for the one-kernel step."""
+    c = _long_small("long_small", **kw)
+    st = P.closed_loop(c, seed=5, T=c.T, logit_bias_fn=_no_eos(c))
+    assert st.steps == c.T and st.live_rows == c.T * c.N and st.resample_events > 0
+    _report("long_small, %s, T = %d" % (label, c.T), st)
+
+
+def test_vocabulary_sharded_step_over_three_thousand_tokens():
+    from test_gpu_vocab_shard import sharded_loop
+    c = _long_small("long_sharded")
+    st, owners = sharded_loop(c, 6, c.T, [(0, 1500), (1500, 2596)], logit_edit=_no_eos(c))
+    assert st.steps == c.T and (owners > 0).all()
+    _report("long_sharded, 2 ranks, T = %d" % c.T, st)
+
+
+def test_tile_fed_step_over_three_thousand_tokens():
+    from test_gpu_tile_fed import tile_fed_loop
+    c = _long_small("long_tiles")
+    st = tile_fed_loop(c, 7, c.T, 1024, logit_edit=_no_eos(c))
+    assert st.steps == c.T
+    _report("long_tiles, width 1024, T = %d" % c.T, st)
+
+
 @pytest.mark.parametrize("N,V,T,kappa", [(33, 64, 300, 0.9), (1024, 32, 9, 1.0), (8, 50, 1200, 0.7)])
 def test_back_trace_over_several_batches(N, V, T, kappa):
     """The output step stages its ancestry log in batches of 4096 integers; T * N beyond that takes several batches.
