@@ -94,6 +94,14 @@ __device__ __forceinline__ float pair_sum(f32x2 v) {
     const float2 f = unpack2(v);
     return f.x + f.y;
 }
+// The warp's total of one sum, from the lanes' four partial sums each: added up in fp64 and rounded to fp32 once.
+// (A partner below half an ulp of the partial sum that holds the row's dominant term would vanish in an fp32 tree,
+// the remainders of compensated sums among them.)
+__device__ __forceinline__ float warp_total(f32x2 a, f32x2 b) {
+    const float2 fa = unpack2(a), fb = unpack2(b);
+    const double t = ((double)fa.x + (double)fb.x) + ((double)fa.y + (double)fb.y);
+    return (float)warp_sum(t);
+}
 __device__ __forceinline__ f32x2 pair_scale(f32x2 v, float f) { return mul2(v, pack2(f, f)); }
 
 // The packed operations take no immediates; the constants they need live in registers for the whole kernel.
@@ -214,12 +222,27 @@ __device__ __forceinline__ void consume(const uint32_t (&w)[NW], const PackedCon
     else consume_f32<MODE, NW>(w, k, a);
 }
 
-// any alignment: one logit per lane per load
+// any alignment: one logit per lane per load.  A lane has one running sum here, not four, and the sum that holds a
+// row's dominant term swallows every later term below half an ulp of it, always downwards (measured on rows with one
+// token far above the rest: ln(sum) low by 2e-8 to 4e-8, the same at every token, which adds up in log p(y_{1:t})).
+// So the sum of the 2^{x-c} is compensated: what each addition rounds away is collected in the second accumulator,
+// which the warp's total adds back.
 template <int DT, int MODE>
 __device__ __forceinline__ void span_scalar(const void* rowp, int a0, int b0, const PackedConsts& k, int lane,
                                             LaneSums& acc) {
-    for (int i0 = a0; i0 < b0; i0 += 32)  // the same trip count in every lane
-        add_one<MODE>(i0 + lane < b0 ? load_elem<DT>(rowp, i0 + lane) : -INFINITY, k, acc);
+    for (int i0 = a0; i0 < b0; i0 += 32) {  // the same trip count in every lane
+        const float l = i0 + lane < b0 ? load_elem<DT>(rowp, i0 + lane) : -INFINITY;
+        if (__any_sync(kFull, l > acc.thr)) move_reference<MODE>(l, k, acc);  // (scales sum and remainder alike)
+        const float d = rel_exponent(l, acc.neg_c);  // -inf for a lane without a logit: mass 0
+        const float e = ex2(d);
+        float2 s = unpack2(acc.s1a), r = unpack2(acc.s1b);
+        const float t = s.x + e, virt = t - s.x;
+        r.x += (s.x - (t - virt)) + (e - virt);  // exactly what the addition lost
+        s.x = t;
+        acc.s1a = pack2(s.x, s.y);
+        acc.s1b = pack2(r.x, r.y);
+        if (MODE != kBeta1) acc.sba = add2(acc.sba, pack2(mass_beta<MODE>(d, k.bf1), 0.f));
+    }
 }
 
 struct StreamParams {
@@ -296,8 +319,8 @@ struct TaskWalker {
 // one triple per span: the lanes share the reference exponent, so their sums add up as they are
 template <int MODE>
 __device__ __forceinline__ void store_triple(const StreamParams& p, int row, int sp, const LaneSums& acc, int lane) {
-    const float s1 = warp_sum(pair_sum(add2(acc.s1a, acc.s1b)));
-    const float sb = (MODE == kBeta1) ? 0.f : warp_sum(pair_sum(add2(acc.sba, acc.sbb)));
+    const float s1 = warp_total(acc.s1a, acc.s1b);
+    const float sb = (MODE == kBeta1) ? 0.f : warp_total(acc.sba, acc.sbb);
     if (lane == 0) __stcg(&p.partials[(size_t)row * p.n_spans + sp], make_float4(-acc.neg_c, s1, sb, 0.f));
 }
 // The streaming loop of one warp (rows that start on 16-byte boundaries): the bulk-copy pipeline described at the top
