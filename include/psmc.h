@@ -402,7 +402,10 @@ psmc_status psmc_state_load(psmc_ctx*, const void* host_buf, size_t bytes);
  * their chained launches) and one around every reindex kernel.  on = 0: off.  psmc_timing_read waits for the
  * recorded events, adds up the device time per bracket kind (HOST arrays of 3: [0] logit pass, or with on = 2 the
  * whole step; [1] weights/ESS/resampling when it is a kernel of its own; [2] KV reindex; milliseconds and
- * bracket counts) and clears the record. */
+ * bracket counts) and clears the record.
+ * Independently of this, every call that launches kernels (psmc_step, psmc_step_host, psmc_reindex_kv, the paged,
+ * sharded and tile-fed calls, psmc_select, psmc_reset) opens an NVTX range named after itself on the calling
+ * thread for the duration of the call, so that timelines of NVTX-aware tools show which call a kernel belongs to. */
 psmc_status psmc_timing_enable(psmc_ctx*, int on);
 psmc_status psmc_timing_read(psmc_ctx*, double* ms_out, int64_t* launches_out);
 

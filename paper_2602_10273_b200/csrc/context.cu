@@ -8,6 +8,8 @@
 #include <string.h>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "internal.h"
 
 using namespace psmc;
@@ -79,6 +81,15 @@ struct psmc_ctx {
 };
 
 namespace {
+
+// A named range around the launches of one call, for timelines of tools that follow NVTX (header-only: without such a
+// tool attached a push or pop is one test of a pointer).
+struct TraceRange {
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+    TraceRange(const TraceRange&) = delete;
+    TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // finished flags after the steps taken so far
 uint8_t* done_now(const psmc_ctx* c) { return c->done2[c->t & 1]; }
@@ -255,6 +266,7 @@ extern "C" psmc_status psmc_destroy(psmc_ctx* c) {
 }
 
 extern "C" psmc_status psmc_reset(psmc_ctx* c, uint64_t seed) {
+    TraceRange trace("psmc_reset");
     if (!c) return PSMC_E_INVAL;
     if (cudaDeviceSynchronize() != cudaSuccess) return PSMC_E_CUDA;
     c->seed = seed;
@@ -309,6 +321,7 @@ WeightsArgs weights_args(psmc_ctx* c, int t, const StepExponents& x) {
 }  // namespace
 
 extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt, int64_t ld, void* stream) {
+    TraceRange trace("psmc_step");
     if (!c || !logits || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
     if (c->t >= c->T_max || c->shard_phase != 0 || c->tile_phase != 0) return PSMC_E_STATE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -345,6 +358,7 @@ extern "C" psmc_status psmc_step(psmc_ctx* c, const void* logits, psmc_dtype dt,
 // ---- the step with the vocabulary split over ranks (vocab_shard.cu) ----
 extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, psmc_dtype dt, int64_t ld, int V_local,
                                         double* triples_out, void* stream) {
+    TraceRange trace("psmc_shard_sweep");
     if (!c || !logits_local || !triples_out || V_local < 2 || V_local > c->V || ld < V_local ||
         (dt != PSMC_F32 && dt != PSMC_BF16))
         return PSMC_E_INVAL;
@@ -371,6 +385,7 @@ extern "C" psmc_status psmc_shard_sweep(psmc_ctx* c, const void* logits_local, p
 
 extern "C" psmc_status psmc_shard_locate(psmc_ctx* c, int v0, const double* all_triples, int P, int rank,
                                          psmc_shard_pick* picks_out, void* stream) {
+    TraceRange trace("psmc_shard_locate");
     if (!c || !all_triples || !picks_out || P < 1 || P > 1024 || rank < 0 || rank >= P || v0 < 0) return PSMC_E_INVAL;
     if (c->shard_phase != 1) return PSMC_E_STATE;
     if ((int64_t)v0 + c->shard_la.V > c->V) return PSMC_E_INVAL;
@@ -388,6 +403,7 @@ extern "C" psmc_status psmc_shard_locate(psmc_ctx* c, int v0, const double* all_
 
 extern "C" psmc_status psmc_shard_finish(psmc_ctx* c, const double* all_triples, const psmc_shard_pick* all_picks,
                                          int P, void* stream) {
+    TraceRange trace("psmc_shard_finish");
     if (!c || !all_triples || !all_picks) return PSMC_E_INVAL;
     if (c->shard_phase != 2) return PSMC_E_STATE;
     if (P != c->shard_P) return PSMC_E_INVAL;
@@ -404,6 +420,7 @@ extern "C" psmc_status psmc_shard_finish(psmc_ctx* c, const double* all_triples,
 // ---- the step fed one vocabulary tile at a time (the consumer side of an LM-head GEMM that never writes [R, V]) ----
 extern "C" psmc_status psmc_tiles_feed(psmc_ctx* c, const void* tile_logits, psmc_dtype dt, int64_t ld, int v0, int width,
                                        void* stream) {
+    TraceRange trace("psmc_tiles_feed");
     if (!c || !tile_logits || width < 2 || ld < width || v0 < 0 || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
     if (c->t >= c->T_max || c->shard_phase != 0 || c->tile_phase > 1) return PSMC_E_STATE;
     if (c->top_k > 0 || c->top_p > 0.0) return PSMC_E_STATE;  // ranking a row needs all of its columns
@@ -449,6 +466,7 @@ extern "C" psmc_status psmc_tiles_feed(psmc_ctx* c, const void* tile_logits, psm
 }
 
 extern "C" psmc_status psmc_tiles_need(psmc_ctx* c, int32_t* first_column_out, void* stream) {
+    TraceRange trace("psmc_tiles_need");
     if (!c || !first_column_out) return PSMC_E_INVAL;
     if (c->tile_phase != 1 || c->tile_next_v0 != c->V) return PSMC_E_STATE;  // the tiles have to cover the vocabulary
     const int t = c->t + 1;
@@ -461,6 +479,7 @@ extern "C" psmc_status psmc_tiles_need(psmc_ctx* c, int32_t* first_column_out, v
 }
 
 extern "C" psmc_status psmc_tiles_finish(psmc_ctx* c, const void* row_tiles, psmc_dtype dt, int64_t ld, void* stream) {
+    TraceRange trace("psmc_tiles_finish");
     if (!c || !row_tiles || (dt != PSMC_F32 && dt != PSMC_BF16)) return PSMC_E_INVAL;
     if (c->tile_phase != 2) return PSMC_E_STATE;
     if (ld < c->tile_width) return PSMC_E_INVAL;
@@ -492,6 +511,7 @@ extern "C" psmc_status psmc_tiles_finish(psmc_ctx* c, const void* row_tiles, psm
 
 extern "C" psmc_status psmc_step_host(psmc_ctx* c, const void* logits_host, psmc_dtype dt, int64_t ld,
                                       int32_t* tokens_out_host, void* stream) {
+    TraceRange trace("psmc_step_host");
     if (!c || !logits_host || !tokens_out_host || ld < c->V || (dt != PSMC_F32 && dt != PSMC_BF16))
         return PSMC_E_INVAL;
     if (c->t >= c->T_max) return PSMC_E_STATE;
@@ -529,6 +549,7 @@ extern "C" psmc_status psmc_step_host(psmc_ctx* c, const void* logits_host, psmc
 
 extern "C" psmc_status psmc_reindex_kv(psmc_ctx* c, const psmc_kv_desc* src, const psmc_kv_desc* dst,
                                        const int32_t* idx_override, void* stream) {
+    TraceRange trace("psmc_reindex_kv");
     if (!c || !src || !src->k || !src->v) return PSMC_E_INVAL;
     if (src->n_layers < 1 || src->n_kv_heads < 1 || src->head_dim < 1 || src->max_len < 1) return PSMC_E_INVAL;
     if (src->dt != PSMC_F32 && src->dt != PSMC_BF16) return PSMC_E_INVAL;
@@ -615,6 +636,7 @@ extern "C" psmc_status psmc_kv_paged_create(psmc_ctx* c, int n_blocks, int block
 }
 
 extern "C" psmc_status psmc_kv_paged_append(psmc_ctx* c, void* stream) {
+    TraceRange trace("psmc_kv_paged_append");
     if (!c) return PSMC_E_INVAL;
     if (!c->paged.table) return PSMC_E_STATE;
     return launch_paged_append(c->paged, c->len, done_now(c), c->status, static_cast<cudaStream_t>(stream)) == cudaSuccess
@@ -622,6 +644,7 @@ extern "C" psmc_status psmc_kv_paged_append(psmc_ctx* c, void* stream) {
 }
 
 extern "C" psmc_status psmc_reindex_kv_paged(psmc_ctx* c, const psmc_kv_pools* pools, void* stream) {
+    TraceRange trace("psmc_reindex_kv_paged");
     if (!c || !pools || !pools->k || !pools->v) return PSMC_E_INVAL;
     if (!c->paged.table) return PSMC_E_STATE;
     if (pools->n_layers < 1 || pools->n_layers > kMaxKvPtrs / 2 || pools->n_kv_heads < 1 || pools->head_dim < 1)
@@ -653,6 +676,7 @@ extern "C" const int32_t* psmc_kv_paged_free_count(psmc_ctx* c) { return c ? c->
 
 extern "C" psmc_status psmc_select(psmc_ctx* c, int32_t* out_tokens, int32_t* out_len, int32_t* out_index,
                                    void* stream) {
+    TraceRange trace("psmc_select");
     if (!c) return PSMC_E_INVAL;
     SelectArgs a{};
     a.G = c->G; a.N = c->N; a.R = c->R; a.t = c->t; a.T_max = c->T_max; a.eos = c->eos; a.seed = c->seed;
