@@ -42,6 +42,7 @@ constexpr int kGranule = 512;      // bytes: one 16-byte chunk per lane
 constexpr int kStepWarps = 23;     // streaming warps per CTA at most (with the helper: 6 warps per scheduler, 80 registers)
 constexpr int kMaxSegments = 48;   // rows one CTA's share may meet (shapes beyond that take the two-kernel step)
 constexpr int kMinGranulesPerWarp = 8;  // 4 KB, one stage: on small blocks fewer, larger pieces mean fewer triples to sum per row (measured: 4 -> 8 saves 2.5 us per step on 16 x 151936 logits, 16 loses 0.7 again)
+constexpr int kOneRowGranules = 256;  // rows up to this size (128 KB) go one to a CTA when the block has no more rows than SMs
 constexpr int kStagedTriples = 256;  // triples of a shared row that are copied to shared memory before they are summed
 static_assert(kStepWarps % 4 == 3, "the helper completes the last scheduler's set of warps");
 
@@ -569,6 +570,15 @@ bool step_geometry(int R, int V, int dt, StepGeom& g, int& grid) {
     g.gpr = (int)gpr;
     g.base = (int)(total / grid);
     g.extra = (int)(total % grid);
+    // A small block is all latency: with one whole row per CTA no row is shared between CTAs, which takes the row
+    // ticket and the trip for the other CTAs' triples out of the chain every step waits for.  Measured (launches back
+    // to back): 4 x 1024 fp32 12.4 -> 10.6 us, 8 x 32000 bf16 14.9 -> 12.2 us; rows of 300 KB lose (16 x 151936 bf16:
+    // 18.6 -> 21.0 us, one SM streams a row in 3 us), so the rule stops at 128 KB.
+    if (R <= kSMs && gpr <= kOneRowGranules) {
+        grid = R;
+        g.base = (int)gpr;
+        g.extra = 0;
+    }
     g.row_bytes16 = (int)row_bytes16;
     g.tail = V % per16;
     const int per_cta = g.base + (g.extra ? 1 : 0);
