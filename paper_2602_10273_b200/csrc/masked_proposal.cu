@@ -301,6 +301,41 @@ __device__ __forceinline__ void clear_columns(uint32_t* cnt, unsigned long long*
 }
 
 // Ascending bitonic sort of n2 (a power of two) 64-bit words in shared memory by the whole CTA.
+// 128 words, four per lane (word e sits in lane e / 4, place e % 4), sorted ascending by one warp: a bitonic network
+// whose exchanges run inside a lane for the two smallest strides and through shuffles otherwise.  No shared memory, no
+// CTA barrier.
+constexpr int kWarpList = 128;
+__device__ __forceinline__ void warp_sort_128(unsigned long long (&v)[4], int lane) {
+#pragma unroll
+    for (int size = 2; size <= kWarpList; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride >= 1; stride >>= 1) {
+            if (stride >= 4) {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int e = lane * 4 + r;
+                    const unsigned long long other = __shfl_xor_sync(kFull, v[r], stride >> 2);
+                    const bool up = (e & size) == 0, low = (e & stride) == 0;  // ascending run; this is the lower index
+                    const bool take_min = up == low;
+                    v[r] = take_min ? (v[r] < other ? v[r] : other) : (v[r] > other ? v[r] : other);
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if ((r & stride) == 0) {
+                        const int e = lane * 4 + r;
+                        const bool up = (e & size) == 0;
+                        const unsigned long long a = v[r], b = v[r | stride];
+                        const bool swap = up ? a > b : a < b;
+                        v[r] = swap ? b : a;
+                        v[r | stride] = swap ? a : b;
+                    }
+                }
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void sort_words(unsigned long long* a, int n2) {
     for (int k = 2; k <= n2; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
@@ -318,6 +353,75 @@ __device__ __forceinline__ void sort_words(unsigned long long* a, int n2) {
             __syncthreads();
         }
     }
+}
+
+// What is left of a row once a short candidate list stands behind a top-k threshold, by ONE warp (see the call).
+template <int DT, int MODE>
+__device__ __noinline__ void finish_short_list(const MaskedParams& p, const unsigned long long* list, int n_cands, int k_top,
+                                               const void* rowp, float C, double U, double S1, int row, int lane) {
+    const float neg_C = -C;
+    unsigned long long v[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int e = lane * 4 + r;
+        v[r] = ~0ull;
+        if (e < n_cands) {  // larger key first, lower id first among equal keys
+            const unsigned long long w = list[e];
+            v[r] = ((unsigned long long)(~key_of<DT>((uint32_t)w)) << 32) | (w >> 32);
+        }
+    }
+    __syncwarp();  // the list has been read: its memory takes the ranked entries' payload below
+    // (the rank order loses the logit's bits: keep them beside the id by sorting (rank word, bits) pairs would
+    // need 96 bits; instead the bits are fetched again by id from the row after the second sort)
+    warp_sort_128(v, lane);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int e = lane * 4 + r;
+        v[r] = e < k_top ? (v[r] & 0xffffffffull) : ~0ull;  // members of S by id; the rest sink to the end
+    }
+    warp_sort_128(v, lane);  // vocabulary order
+    double m[4], mine = 0.0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int e = lane * 4 + r;
+        m[r] = e < k_top ? (double)logit_mass<MODE>(load_elem<DT>(rowp, (int)v[r]), neg_C, p.bf) : 0.0;
+        mine += m[r];
+    }
+    const double incl = warp_scan_incl(mine, lane);
+    const double Sb = __shfl_sync(kFull, incl, 31), target = U * Sb;
+    const unsigned hit = __ballot_sync(kFull, mine > 0.0 && incl >= target);
+    const unsigned has = __ballot_sync(kFull, mine > 0.0);
+    if (!has) {  // no member of S has mass: cannot happen while the row's largest logit is in S
+        if (lane == 0) {
+            raise_status(p.status, PSMC_E_NUMERIC);
+            p.tok[row] = -1;
+            p.logp[row] = 0.0;
+            p.loginc[row] = 0.0;
+            p.set_size[row] = k_top;
+        }
+        return;
+    }
+    const int owner = hit ? __ffs(hit) - 1 : 31 - __clz(has);
+    if (lane != owner) return;
+    double run = incl - mine;
+    int y = -1, last = -1;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        run += m[r];
+        if (m[r] > 0.0) {
+            last = (int)v[r];
+            if (y < 0 && run >= target) y = last;
+        }
+    }
+    if (y < 0) y = last;
+    const double dl = (double)load_elem<DT>(rowp, y) - (double)C * kLn2;
+    double add_s1, add_sb;
+    ln_sum_corrections<MODE>(p.beta, add_s1, add_sb);
+    const double ln_s1 = log(S1) + add_s1, ln_sb = log(Sb) + add_sb;
+    p.tok[row] = y;
+    p.logp[row] = dl - ln_s1;
+    p.loginc[row] = (p.alpha_t - p.beta) * dl - p.alpha_t * ln_s1 + ln_sb;
+    p.set_size[row] = k_top;
 }
 
 template <int DT, int MODE>
@@ -660,6 +764,19 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
     if (listed) {
         __syncthreads();
         const int n_cands = min(n_list_sh, kListCap);
+
+        // ---- a short list behind a top-k threshold: everything that is left, by one warp and without CTA barriers ----
+        // The general way below spends a dozen CTA barriers on a hundred entries (digit search, filter, sort, two
+        // scans: 10 us of the 39 us a row took, with 15 of the 16 warps idle).  Here the candidates are ranked by
+        // (logit descending, id ascending) in one sort -- the first k of that order are S, ties at the cut included --
+        // then S is put in vocabulary order by a second sort, and the masses and the inverse CDF are warp scans.
+        const int k_top = min(p.top_k, V);
+        if (by_threshold && first_list_level == 0 && n_cands <= kWarpList && n_cands >= k_top) {
+            const double S1 = block_sum(s1, red, nw);
+            if (warp != 0) return;
+            finish_short_list<DT, MODE>(p, list, n_cands, k_top, rowp, C, U, S1, row, lane);
+            return;
+        }
 
         // ---- the levels not yet decided, over the candidates in whatever order they arrived ----
         const bool short_list = n_cands <= 2 * (int)blockDim.x;  // few entries: no columns, one counter per digit

@@ -75,6 +75,24 @@ def test_ties_at_the_cut_are_taken_in_id_order(name, rule):
     assert st.steps == 12
 
 
+@pytest.mark.parametrize("top_k", [1, 5, 50, 100, 120, 127, 128, 129, 200])
+@pytest.mark.parametrize("name", ["llama2_7b", "tiny"])
+def test_ties_straddle_the_cut_of_a_short_candidate_list(name, top_k):
+    """A few logits equal to the k-th largest, scattered over the row: the candidate list stays short (up to 128
+    entries are ranked by one warp, longer lists by the whole CTA: sizes on both sides of that limit), and which of the
+    equal logits belong to the set is decided by token id."""
+    cfg = W.CONFIGS[name]
+    gen = torch.Generator(device="cuda").manual_seed(top_k)
+
+    def plant(t, lg):
+        kth = torch.topk(lg.float(), top_k, dim=1).values[:, -1:]                  # [R, 1]
+        cols = torch.randint(0, cfg.V - 1, (lg.shape[0], 6), device="cuda", generator=gen)
+        lg.scatter_(1, cols, kth.expand(-1, 6).to(lg.dtype))
+
+    st = P.closed_loop(cfg, 13, 10, logit_bias_fn=plant, top_k=top_k)
+    assert st.steps == 10 and st.k_adopted == 0
+
+
 def test_signed_zeros_and_masked_columns():
     cfg = W.CONFIGS["tiny"]
 
