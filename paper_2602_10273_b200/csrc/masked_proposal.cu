@@ -38,6 +38,7 @@
 // for every remaining step.
 #include "internal.h"
 #include "logits_common.cuh"
+#include "logits_stream.cuh"
 #include "weights_core.cuh"
 
 namespace psmc {
@@ -606,16 +607,18 @@ __global__ void __launch_bounds__(1024, 1) masked_rows_kernel(const __grid_const
         // ---- sweep 2: the normaliser of p, and every logit at or above the threshold into the list ----
         if (DT == PSMC_BF16) {
             const uint32_t th2 = pair_threshold(theta);
+            // (the packed fp32 arithmetic of the plain logit pass: both logits of a word at once, the same operations)
+            const PackedConsts kc = packed_consts(p.bf);
+            const f32x2 nc2 = pack2(neg_C, neg_C);
             for_each_vector<DT>(
                 rowp, V,
                 [&](const uint4& v, int i0) {
                     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                    float part = 0.f;
+                    f32x2 part2 = ex2_2(rel_exponent2(widen_bf16x2(w[0]), nc2, kc));
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        part += ex2(rel_exponent(__uint_as_float(w[c] << 16), neg_C)) +
-                                ex2(rel_exponent(__uint_as_float(w[c] & 0xffff0000u), neg_C));
-                    s1 += (double)part;
+                    for (int c = 1; c < 4; ++c) part2 = add2(part2, ex2_2(rel_exponent2(widen_bf16x2(w[c]), nc2, kc)));
+                    const float2 part = unpack2(part2);
+                    s1 += (double)(part.x + part.y);
                     collect8(w, i0, th2);
                 },
                 [&](uint32_t b, int i) {
