@@ -104,15 +104,26 @@ def case_step(a):
     G = cfg.G if a.groups is None else a.groups
     wl = WC.DeviceWorkload(cfg, 1, G=G)
     n_buf = min(64, max(2, -(-2 * L2_BYTES // (wl.R * cfg.logit_bytes_per_row))))
-    T = 3 * a.iters + 8
+    T = 3 * a.iters + 12
     ps = B.Psmc(cfg.N, cfg.V, cfg.alpha, cfg.tau, cfg.kappa, 0 if a.no_ramp else cfg.ramp, 1, cfg.eos_id, G=G,
                 T_max=T, prompt_len=wl.prompt_len)
     if a.top_k or a.top_p:
         ps.set_proposal_mask(a.top_k, a.top_p)
     bufs = [wl.new_logits() for _ in range(n_buf)]
     prev = wl.first_prev.clone()
+    last = ps.device_view("psmc_last_tokens", wl.R)
+    # The blocks follow a real run for its first tokens (every row's logits depend on its own last token), so that the
+    # particles of a group see different rows, their weights differ and resampling fires as it does in a decoding
+    # loop; with the same previous token in every row of a group no step would ever resample.
+    wl.fill(bufs[0], 1, prev)
+    ps.step(bufs[0])
+    prev.copy_(last)
     for i, b in enumerate(bufs):
-        wl.fill(b, 1 + i, prev)
+        wl.fill(b, 2 + i, prev)
+        if i < 8:
+            ps.step(b)
+            prev.copy_(last)
+    ps.reset(1)
 
     def run(i):
         ps.step(bufs[i % n_buf])
