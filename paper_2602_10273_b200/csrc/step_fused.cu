@@ -99,8 +99,8 @@ struct Segment {
     int slot;    // which of the CTA's two global triple rows a shared part uses
     __device__ __forceinline__ bool local(const StepGeom& g) const { return g0 == 0 && g1 == g.gpr; }
 };
-__device__ __forceinline__ Segment segment_of_row(const StepGeom& g, int b, int row) {
-    const int first = share_first(g, b), last = first + share_count(g, b);
+// the part of row `row` inside the share [first, last) of granules
+__device__ __forceinline__ Segment segment_in_share(const StepGeom& g, int first, int last, int row) {
     const int lo = max(first, row * g.gpr), hi = min(last, (row + 1) * g.gpr);
     Segment s;
     s.row = row;
@@ -108,6 +108,10 @@ __device__ __forceinline__ Segment segment_of_row(const StepGeom& g, int b, int 
     s.g1 = hi - row * g.gpr;
     s.slot = (row == first / g.gpr) ? 0 : 1;
     return s;
+}
+__device__ __forceinline__ Segment segment_of_row(const StepGeom& g, int b, int row) {
+    const int first = share_first(g, b);
+    return segment_in_share(g, first, first + share_count(g, b), row);
 }
 // The CTA's segments in the order they are taken: the shared parts at the two ends first, then the rows in between.
 __device__ __forceinline__ int segment_in_order(int k, int S) {
@@ -162,6 +166,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Where a warp's k-th piece lies: pure geometry (a function of the launch parameters), so the first kPieceTab pieces
+// of every warp are worked out before the kernel waits for its predecessor and kept in shared memory.  The index
+// arithmetic (divisions by run-time values) would otherwise run at every piece boundary, in the producer as in the
+// consumer, with the warp's ring running dry meanwhile.
+constexpr int kPieceTab = 6;
+struct PieceRec {
+    long long off;   // first byte, relative to the start of the logit block
+    int bytes;       // bytes bulk copies fetch (a multiple of 16)
+    uint32_t meta;   // tail (bits 0-7) | segment (8-15) | local to the CTA (16) | slot of a shared part (17)
+};
+
 struct StepShared {
     uint64_t ring_bars[kStepWarps * kDepth];
     uint64_t seg_bars[kMaxSegments];       // one per segment: all streaming warps have stored their triple
@@ -170,6 +185,8 @@ struct StepShared {
     GroupScratch<32> sc;                   // the helper's; a streaming warp that closes a group uses its idle ring
     // rows this CTA finishes after the sweep, listed by the helper with their totals and the piece to re-read
     int n_pend, timed_out;
+    int own_first, own_last;               // this CTA's share of granules (worked out once)
+    PieceRec pieces[kStepWarps][kPieceTab];  // the first pieces of every streaming warp, laid out ahead of the sweep
     RowTotals pend_t[kMaxSegments];
     int pend_row[kMaxSegments], pend_a0[kMaxSegments], pend_b0[kMaxSegments];
     double end_tot[kStepWarps + 1];        // per warp: mass of its part of the selected piece
@@ -183,23 +200,40 @@ struct PieceDesc {
     int tail;          // ragged logits after them, fetched with plain loads
     int seg, place;
     bool live;
+    bool local;        // the piece's row lies wholly in this CTA's share
+    int slot;          // else: which of the CTA's two global triple rows its part uses
 };
+// the geometry of piece k of warp `warp` in the share [own_first, own_last)
+template <int DT>
+__device__ __forceinline__ PieceRec piece_layout(const StepParams& sp, int own_first, int own_last, int first_row, int S,
+                                                 int k, int warp) {
+    constexpr int kEsize = DT == PSMC_F32 ? 4 : 2;
+    const int seg = segment_in_order(k, S);
+    const Segment s = segment_in_share(sp.g, own_first, own_last, first_row + seg);
+    int p0, p1;
+    piece_granules(s, warp, sp.g.W, p0, p1);
+    PieceRec r;
+    r.off = (long long)s.row * sp.ld * kEsize + (long long)p0 * kGranule;
+    const int end = min(p1 * kGranule, sp.g.row_bytes16);
+    r.bytes = max(end - p0 * kGranule, 0);
+    const int tail = (p1 == sp.g.gpr && p1 > p0) ? sp.g.tail : 0;
+    r.meta = (uint32_t)tail | ((uint32_t)seg << 8) | (s.local(sp.g) ? 1u << 16 : 0u) | ((uint32_t)s.slot << 17);
+    return r;
+}
 template <int DT>
 __device__ __forceinline__ PieceDesc piece_at(const StepParams& sp, const StepShared& sh, int first_row, int S, int k,
                                               int warp) {
-    constexpr int kEsize = DT == PSMC_F32 ? 4 : 2;
+    const PieceRec r = k < kPieceTab ? sh.pieces[warp][k]
+                                     : piece_layout<DT>(sp, sh.own_first, sh.own_last, first_row, S, k, warp);
     PieceDesc d;
-    d.seg = segment_in_order(k, S);
-    const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + d.seg);
+    d.src = reinterpret_cast<const char*>(sp.logits) + r.off;
+    d.bytes = r.bytes;
+    d.tail = (int)(r.meta & 255u);
+    d.seg = (int)((r.meta >> 8) & 255u);
     d.place = warp;
     d.live = !sh.seg_done[d.seg];
-    int p0, p1;
-    piece_granules(s, d.place, sp.g.W, p0, p1);
-    const char* rowp = reinterpret_cast<const char*>(sp.logits) + (size_t)s.row * sp.ld * kEsize;
-    d.src = rowp + (size_t)p0 * kGranule;
-    const int end = min(p1 * kGranule, sp.g.row_bytes16);
-    d.bytes = max(end - p0 * kGranule, 0);
-    d.tail = (p1 == sp.g.gpr && p1 > p0) ? sp.g.tail : 0;
+    d.local = (r.meta >> 16) & 1u;
+    d.slot = (int)((r.meta >> 17) & 1u);
     return d;
 }
 
@@ -299,10 +333,9 @@ __device__ __forceinline__ bool stream_pieces(const StepParams& sp, StepShared& 
         const float s1 = warp_sum(pair_sum(add2(acc.s1a, acc.s1b)));
         const float sb = (MODE == kBeta1) ? 0.f : warp_sum(pair_sum(add2(acc.sba, acc.sbb)));
         if (lane == 0) {
-            const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + d.seg);
             const float4 tr = make_float4(-acc.neg_c, s1, sb, 0.f);
-            if (s.local(sp.g)) local_triples[d.seg * W + d.place] = tr;
-            else __stcg(&sp.shared_triples[((size_t)blockIdx.x * 2 + s.slot) * W + d.place], tr);
+            if (d.local) local_triples[d.seg * W + d.place] = tr;
+            else __stcg(&sp.shared_triples[((size_t)blockIdx.x * 2 + d.slot) * W + d.place], tr);
             // release: the triple is visible to whoever sees the barrier complete
             if (S > kNamedBarriers) mbar_arrive(&sh.seg_bars[d.seg]);
         }
@@ -410,7 +443,7 @@ __device__ __noinline__ void helper_warp(const StepParams& sp, StepShared& sh, c
     __syncwarp();
     for (int k = 0; k < S; ++k) {
         const int seg = segment_in_order(k, S);
-        const Segment s = segment_of_row(sp.g, (int)blockIdx.x, first_row + seg);
+        const Segment s = segment_in_share(sp.g, sh.own_first, sh.own_last, first_row + seg);
         const int row = s.row;
         if (sh.seg_done[seg]) {
             if (s.g1 == sp.g.gpr) row_arrives(sp, sh, sh.sc, row, nullptr, false, lane);
@@ -547,10 +580,17 @@ __global__ void __launch_bounds__((kStepWarps + 1) * 32, 1) psmc_step_kernel(con
     if (warp < W) stream_init_barriers(sh.ring_bars + warp * kDepth, lane);
     if ((int)threadIdx.x < S) mbar_init(&sh.seg_bars[threadIdx.x], (uint32_t)W);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (warp < W && lane < kPieceTab && lane < S)  // one lane per piece; read back only by this warp
+        sh.pieces[warp][lane] = piece_layout<DT>(sp, first, first + count, first_row, S, lane, warp);
+    __syncwarp();
     chain_begin();  // everything above is local set-up; global memory from here on
     if (sp.zero_words && blockIdx.x == 0 && threadIdx.x < 2) sp.zero_words[threadIdx.x] = 0;
     if ((int)threadIdx.x < S) sh.seg_done[threadIdx.x] = sp.a.done[first_row + threadIdx.x];
-    if (threadIdx.x == 0) sh.n_pend = sh.timed_out = 0;
+    if (threadIdx.x == 0) {
+        sh.n_pend = sh.timed_out = 0;
+        sh.own_first = first;
+        sh.own_last = first + count;
+    }
     __syncthreads();
 
     if (warp < W) {
