@@ -471,6 +471,14 @@ __device__ __noinline__ void helper_warp(const StepParams& sp, StepShared& sh, c
         int a0 = 0, b0 = 0;
         if (t.ok) selected_range<DT>(sp, s, c_first, t.jsel, a0, b0);
         if (lane == 0) {
+            // The piece that holds the target is read again when the row is finished, after the sweep.  Its lines were
+            // fetched marked evict-first and are gone from L2 by then (the block is larger than L2); asked for again
+            // now, they wait in L2 with the normal priority and the re-read costs a trip to L2 instead of one to HBM.
+            constexpr int kEs = DT == PSMC_F32 ? 4 : 2;
+            const int64_t from = (int64_t)a0 * kEs;
+            const int bytes = (int)((((int64_t)b0 * kEs) & ~(int64_t)15) - from);  // (a piece starts on a granule)
+            if (t.ok && k < S - 1 && bytes > 0)
+                bulk_prefetch_l2(reinterpret_cast<const char*>(sp.logits) + (size_t)row * sp.ld * kEs + from, (uint32_t)bytes);
             const int i = sh.n_pend++;
             sh.pend_t[i] = t;
             sh.pend_row[i] = row;
