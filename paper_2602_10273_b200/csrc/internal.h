@@ -113,6 +113,7 @@ cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa,
 
 // The step with the proposal restricted to the top_k tokens of each row, or to the nucleus of share top_p (exactly one
 // of the two > 0): one CTA per row for the logit pass, then the per-group update.  set_size: [R].
+cudaError_t launch_rows_weights(const WeightsArgs& wa, cudaStream_t stream);  // group updates from rows already in memory
 cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa, int top_k, double top_p,
                                int32_t* set_size, cudaStream_t stream);
 

@@ -1116,6 +1116,12 @@ MaskedFn pick_masked(int mode) {
 
 }  // namespace
 
+// the per-group update from row results that a kernel before it on the stream left in memory
+cudaError_t launch_rows_weights(const WeightsArgs& wa, cudaStream_t stream) {
+    const int warps = (wa.N + 31) / 32;
+    return launch_chained(rows_weights_kernel, dim3((unsigned)wa.G), dim3((unsigned)(warps * 32)), 0, stream, wa);
+}
+
 cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa, int top_k, double top_p,
                                int32_t* set_size, cudaStream_t stream) {
     MaskedParams p;
@@ -1131,8 +1137,7 @@ cudaError_t launch_step_masked(const LogitsStreamArgs& la, const WeightsArgs& wa
     const int threads = la.V < 16384 ? 256 : 512;
     e = launch_chained(fn, dim3((unsigned)la.R), dim3((unsigned)threads), smem, stream, p);
     if (e != cudaSuccess) return e;
-    const int warps = (wa.N + 31) >> 5;
-    return launch_chained(rows_weights_kernel, dim3((unsigned)wa.G), dim3((unsigned)(warps * 32)), 0, stream, wa);
+    return launch_rows_weights(wa, stream);
 }
 
 }  // namespace psmc

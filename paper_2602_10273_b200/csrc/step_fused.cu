@@ -1,4 +1,5 @@
-// The whole per-token step as ONE kernel (groups of up to 32 particles, 16-byte aligned rows): the loop body of
+// The whole per-token step as ONE kernel (16-byte aligned rows; groups of more than 32 particles get their update from
+// a second, small kernel that follows this one: everything up to the rows' tokens and weights is done here): the loop body of
 // Algorithm 1 without the cache move -- proposal sums (Corollary 1), token draw, Eq. 7, weight update, ESS (Eq. 5),
 // trigger, resampling and slot map.
 //
@@ -68,6 +69,7 @@ struct StepParams {
     int32_t* row_arrivals;    // [R] CTAs that have delivered their part of a shared row
     int32_t* group_arrivals;  // [G] rows of the group that are finished
     int32_t* zero_words;
+    int groups_here;          // 0: groups of more than 32 particles, updated by a kernel of their own after this one
 };
 
 // per_row == 0: the whole block is one run of granules dealt out evenly.  per_row = c > 0: every row is dealt to c
@@ -403,6 +405,7 @@ __device__ __forceinline__ void row_arrives(const StepParams& sp, StepShared& sh
         a.logp[row] = rr->logp;
         a.loginc[row] = rr->loginc;
     }
+    if (!sp.groups_here) return;  // the rows' results are in memory: all this kernel owes a large group
     // The group's state as the step found it (nobody writes it before the group is complete) is asked for now: should
     // this warp turn out to be the one that completes the group, the loads have overlapped the trip of the ticket.
     ParticleState st{};
@@ -666,14 +669,17 @@ bool step_geometry(int R, int V, int dt, StepGeom& g, int& grid) {
 
 size_t step_fused_scratch_bytes() { return (size_t)kSMs * 2 * kStepWarps * sizeof(float4); }
 
-// The one-kernel step needs groups that one warp can update (N <= 32), rows that bulk copies can fetch (16-byte
-// aligned starts) and a share per CTA that meets at most kMaxSegments rows.  Everything else takes the step as two
-// kernels (logits_pass.cu, weights_resample.cu).
+// This kernel needs rows that bulk copies can fetch (16-byte aligned starts) and a share per CTA that meets at most
+// kMaxSegments rows; everything else takes the step as two kernels (logits_pass.cu, weights_resample.cu).  A group
+// that one warp can update (N <= 32) is updated here by the warp that finishes its last row; larger groups by
+// rows_weights_kernel right after (measured with 151936 bf16 logits per row, launches back to back: 64 particles
+// 41.4 -> 23.6 us per step, 128 particles 73.9 -> 33.2 us against the step as two kernels).
 bool step_can_fuse(const LogitsStreamArgs& la, int N) {
     const LogitsGeometry lg = logits_geometry(la.logits, la.dt, la.R, la.V, la.ld, la.beta);
     StepGeom g;
     int grid;
-    return N <= 32 && lg.vec != 0 && step_geometry(la.R, la.V, la.dt, g, grid);
+    (void)N;  // groups of more than 32 particles take the sweep and the rows from this kernel, the update from another
+    return lg.vec != 0 && step_geometry(la.R, la.V, la.dt, g, grid);
 }
 
 cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa, void* shared_triples,
@@ -690,12 +696,15 @@ cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa,
     sp.row_arrivals = row_arrivals;
     sp.group_arrivals = group_arrivals;
     sp.zero_words = la.zero_words;
+    sp.groups_here = wa.N <= 32 ? 1 : 0;
     const size_t smem = (size_t)sp.g.W * kDepth * kStageBytes + (size_t)sp.g.seg_cap * sp.g.W * sizeof(float4);
     StepFn fn = la.dt == PSMC_F32 ? pick_step<PSMC_F32>(lg.mode) : pick_step<PSMC_BF16>(lg.mode);
     cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(fn),
                                        kStepWarps * kDepth * kStageBytes + kMaxSegments * kStepWarps * (int)sizeof(float4));
     if (e != cudaSuccess) return e;
-    return launch_chained(fn, dim3((unsigned)grid), dim3((unsigned)((sp.g.W + 1) * 32)), smem, stream, sp);
+    e = launch_chained(fn, dim3((unsigned)grid), dim3((unsigned)((sp.g.W + 1) * 32)), smem, stream, sp);
+    if (e != cudaSuccess || sp.groups_here) return e;
+    return launch_rows_weights(wa, stream);
 }
 
 }  // namespace psmc
