@@ -245,6 +245,17 @@ def test_closed_loop_many_rows_per_cta(G, N, V, dtype):
     assert st.steps == 6 and st.resample_events > 0
 
 
+@pytest.mark.parametrize("G,N,V,dtype,resampler", [(1, 64, 32000, "bf16", 0), (2, 100, 8192, "bf16", 1), (3, 33, 5000, "f32", 3),
+                                                   (1, 128, 151936, "bf16", 0), (1, 1024, 512, "f32", 2)])
+def test_closed_loop_groups_of_more_than_32_particles(G, N, V, dtype, resampler):
+    """Groups that one warp cannot update (the paper's own runs use 64 particles): the one-kernel step leaves the rows'
+    tokens and weights in memory and a second kernel updates the groups.  Sizes that are not multiples of 32, several
+    groups, every resampler."""
+    c = W.Workload("large_groups", G, N, V, dtype, 3.0, 1.5, 8, 3, 6, 4.0, 0.25, 0.6, 0, 1, 1, 8, 24)
+    st = P.closed_loop(c, seed=11, T=8, kv_shape=(1, 1, 24, 8), resampler=resampler)
+    assert st.steps == 8 and st.resample_events > 0
+
+
 def test_closed_loop_llama_shape():
     c = W.CONFIGS["llama2_7b"]
     st = P.closed_loop(c, seed=1, T=96, kv_shape=(2, 4, 512 + 96 + 8, c.head_dim))
