@@ -20,7 +20,7 @@ What is timed, in order (every pass restarts the run from its reset, so all of t
            events (rotating logit blocks: L2-cold) and on one block (L2-hot)  -> `step_without_kv`
   kv_fixed_event   the cache move of a fixed event: half the slots of every group rewritten, len = max_len / 2
   e2e      a few of the K steps through psmc_step_host
-  other_configs    the step alone on the four smaller named configurations
+  other_configs    the step alone on the four smaller named configurations, and with the paper's 64 particles
   cpu_baseline     the oracle, as it stands, on a slice of the same workload
 Supplementary runs: --paged-kv, --skip-shared-prompt, --top-k K, --top-p P (see their help lines).
 """
@@ -161,7 +161,7 @@ def step_alone(name, hbm_peak, steps=200, seed=1):
     (64 blocks at most) and are labelled L2-hot."""
     from paper_2602_10273_b200 import binding as B
     from paper_2602_10273_b200.workload import cuda as WC
-    cfg = gen.CONFIGS[name]
+    cfg = gen.CONFIGS[name] if isinstance(name, str) else name
     wl = WC.DeviceWorkload(cfg, seed)
     block_bytes = wl.R * cfg.logit_bytes_per_row
     n_buf = int(min(64, max(2, -(-2 * L2_BYTES // block_bytes))))
@@ -518,6 +518,11 @@ def run_ours(args):
     }
     if rank == 0 and world == 1 and not args.no_other_configs and not masked and not args.paged_kv:
         out["other_configs"] = {n: step_alone(n, hbm_peak) for n in ("tiny", "llama2_7b", "qwen25_7b", "resample_stress")}
+        # the particle count of the paper's own runs (Section 6: N = 64) on the largest vocabulary of the named shapes:
+        # a group one warp cannot update, so the step is the one kernel followed by the group-update kernel
+        import dataclasses
+        out["other_configs"]["qwen25_7b_64_particles"] = step_alone(
+            dataclasses.replace(gen.CONFIGS["qwen25_7b"], name="qwen25_7b_64_particles", N=64), hbm_peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, wl.seed, wl.prompt_len, [logits_to_numpy(b) for b in blocks], G)
     ps.destroy()
