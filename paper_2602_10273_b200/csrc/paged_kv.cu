@@ -190,9 +190,27 @@ __global__ void __launch_bounds__(256) paged_copy_kernel(const PagedState ps, co
         const uint4* src = reinterpret_cast<const uint4*>(pool + (int64_t)o.src_blk * blk_bytes);
         uint4* dst = reinterpret_cast<uint4*>(pool + (int64_t)o.dst_blk * blk_bytes);
         const int per_head = o.positions * pools.pos_bytes / 16, stride = (int)(head_bytes / 16);
-        for (int e = threadIdx.x; e < per_head * pools.H; e += blockDim.x) {
-            const int h = e / per_head, x = e - h * per_head;
-            dst[(int64_t)h * stride + x] = src[(int64_t)h * stride + x];
+        const int n_el = per_head * pools.H;
+        // Four loads in flight per thread, then their stores: source and destination lie in one pool, so a plain
+        // copy loop would wait for every load before it may issue the next store (one trip to memory per element;
+        // measured on 512 rows with 32 layers: the three kernels of a reindex 31.2 -> 25.7 us, eight loads 27.1 us).
+        constexpr int kBatch = 4;
+        for (int e0 = threadIdx.x; e0 < n_el; e0 += kBatch * blockDim.x) {
+            uint4 v[kBatch];
+            int64_t at[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int e = e0 + u * (int)blockDim.x;
+                at[u] = -1;
+                if (e < n_el) {
+                    const int h = e / per_head, x = e - h * per_head;
+                    at[u] = (int64_t)h * stride + x;
+                    v[u] = src[at[u]];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                if (at[u] >= 0) dst[at[u]] = v[u];
         }
     }
 }
@@ -224,7 +242,7 @@ cudaError_t launch_paged_reindex(const PagedState& ps, const PagedPools& pools, 
     e = launch_chained(paged_acquire_kernel, dim3((unsigned)((ps.R / 2 + 7) / 8 + 1)), dim3(256), 0, stream, ps, sources,
                        dst_rows, n_sources, len, done, status);
     if (e != cudaSuccess) return e;
-    return launch_chained(paged_copy_kernel, dim3(kSMs * 4), dim3(256), 0, stream, ps, pools, n_moves);
+    return launch_chained(paged_copy_kernel, dim3(kSMs * 16), dim3(256), 0, stream, ps, pools, n_moves);
 }
 
 }  // namespace psmc
