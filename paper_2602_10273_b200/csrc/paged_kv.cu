@@ -242,7 +242,10 @@ cudaError_t launch_paged_reindex(const PagedState& ps, const PagedPools& pools, 
     e = launch_chained(paged_acquire_kernel, dim3((unsigned)((ps.R / 2 + 7) / 8 + 1)), dim3(256), 0, stream, ps, sources,
                        dst_rows, n_sources, len, done, status);
     if (e != cudaSuccess) return e;
-    return launch_chained(paged_copy_kernel, dim3(kSMs * 16), dim3(256), 0, stream, ps, pools, n_moves);
+    // items = rewritten slots x pools; about an eighth of the rows are rewritten in a step with resampling
+    int64_t ctas = (int64_t)(ps.R / 8 + 1) * (2 * pools.n_layers);
+    ctas = ctas < kSMs ? kSMs : (ctas > kSMs * 16 ? kSMs * 16 : ctas);
+    return launch_chained(paged_copy_kernel, dim3((unsigned)ctas), dim3(256), 0, stream, ps, pools, n_moves);
 }
 
 }  // namespace psmc
