@@ -180,9 +180,24 @@ __global__ void __launch_bounds__(256) reindex_plain_kernel(const __grid_constan
         it.seg_ptr = c.seg_ptr; it.seg_head = c.seg_head; it.dst_begin = c.dst_begin; it.n_dst = c.n_dst; it.dst_off = 0;
         const int64_t n_units_u = c.seg_bytes / (int64_t)sizeof(U);
         const U* s = reinterpret_cast<const U*>(c.src);
-        for (int64_t e = c.off / (int64_t)sizeof(U) + threadIdx.x; e < n_units_u; e += blockDim.x) {
-            const U v = s[e];
-            for (int d = 0; d < it.n_dst; ++d) reinterpret_cast<U*>(dst_addr(k, it, d))[e] = v;
+        // four loads in flight per thread, then their stores (source and destination may lie in one tensor, so a plain
+        // loop would wait for every load before the next store may go out)
+        constexpr int kBatch = 4;
+        for (int64_t e0 = c.off / (int64_t)sizeof(U) + threadIdx.x; e0 < n_units_u; e0 += (int64_t)kBatch * blockDim.x) {
+            U v[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int64_t e = e0 + (int64_t)u * blockDim.x;
+                if (e < n_units_u) v[u] = s[e];
+            }
+            for (int d = 0; d < it.n_dst; ++d) {
+                U* out = reinterpret_cast<U*>(dst_addr(k, it, d));
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int64_t e = e0 + (int64_t)u * blockDim.x;
+                    if (e < n_units_u) out[e] = v[u];
+                }
+            }
         }
     }
     if (threadIdx.x == 0) leave_queue(k.work);
