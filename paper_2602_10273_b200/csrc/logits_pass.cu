@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) logits_stream_kernel(const 
                            per_warp > 0 ? per_warp : 1, 0, [](int) {});
 }
 
-// Rows of any alignment: plain loads, one logit per lane per load.
+// Rows of any alignment: plain loads, 16 bytes per lane between a span's first and last 16-byte boundary.
 template <int DT, int MODE>
 __global__ void __launch_bounds__(256) logits_stream_scalar_kernel(const __grid_constant__ StreamParams p) {
     const int lane = threadIdx.x & 31;
@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256) logits_stream_scalar_kernel(const __grid_
         const int a0 = sp * p.span, b0 = min(p.V, a0 + p.span);
         const void* rowp = reinterpret_cast<const char*>(p.logits) + (size_t)row * p.ld * (DT == PSMC_F32 ? 4 : 2);
         LaneSums acc = lane_sums_init();
-        span_scalar<DT, MODE>(rowp, a0, b0, kc, lane, acc);
+        span_any_alignment<DT, MODE>(rowp, a0, b0, kc, lane, acc);
         store_triple<MODE>(p, row, sp, acc, lane);
     }
 }

@@ -245,6 +245,40 @@ __device__ __forceinline__ void span_scalar(const void* rowp, int a0, int b0, co
     }
 }
 
+// A span of a row that starts anywhere (rows whose pitch or base is not a multiple of 16 bytes: a vocabulary of odd
+// size in a dense tensor).  The logits up to the first 16-byte boundary and after the last one go one per lane; the
+// stretch between them is read 16 bytes per lane at a time and summed exactly as the staged sweep sums its stages.
+template <int DT, int MODE>
+__device__ __forceinline__ void span_any_alignment(const void* rowp, int a0, int b0, const PackedConsts& k, int lane,
+                                                   LaneSums& acc) {
+    constexpr int kEs = DT == PSMC_F32 ? 4 : 2, kPer = 16 / kEs;
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(rowp) + (size_t)a0 * kEs;
+    int head = (addr % kEs) ? b0 - a0 : (int)(((16 - (addr & 15)) & 15) / kEs);  // (a base off its element size: all scalar)
+    head = head < b0 - a0 ? head : b0 - a0;
+    const int mid0 = a0 + head, chunks = (b0 - mid0) / kPer, tail0 = mid0 + chunks * kPer;
+    if (head > 0) span_scalar<DT, MODE>(rowp, a0, mid0, k, lane, acc);
+    if (chunks > 0) {
+        __nv_bfloat162 thr2 = __float2bfloat162_rn(acc.thr);
+        const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(rowp) + (size_t)mid0 * kEs);
+        int c0 = 0;
+        for (; c0 + 128 <= chunks; c0 += 128) {  // four 16-byte loads per lane in flight
+            const uint4 v0 = __ldg(&q[c0 + lane]), v1 = __ldg(&q[c0 + 32 + lane]), v2 = __ldg(&q[c0 + 64 + lane]),
+                        v3 = __ldg(&q[c0 + 96 + lane]);
+            const uint32_t w[16] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w,
+                                    v2.x, v2.y, v2.z, v2.w, v3.x, v3.y, v3.z, v3.w};
+            consume<DT, MODE, 16>(w, k, acc, thr2);
+        }
+        constexpr uint32_t kNoLogit = DT == PSMC_BF16 ? 0xff80ff80u : 0xff800000u;  // -inf: no mass, never a maximum
+        for (; c0 < chunks; c0 += 32) {  // the same trip count in every lane
+            const bool in = c0 + lane < chunks;
+            const uint4 v0 = in ? __ldg(&q[c0 + lane]) : make_uint4(kNoLogit, kNoLogit, kNoLogit, kNoLogit);
+            const uint32_t w[4] = {v0.x, v0.y, v0.z, v0.w};
+            consume<DT, MODE, 4>(w, k, acc, thr2);
+        }
+    }
+    if (tail0 < b0) span_scalar<DT, MODE>(rowp, tail0, b0, k, lane, acc);
+}
+
 struct StreamParams {
     const void* logits;
     int R, V;
