@@ -647,10 +647,13 @@ bool step_geometry(int R, int V, int dt, StepGeom& g, int& grid) {
         g.base = (int)gpr;
         g.extra = 0;
     }
-    // Larger rows of a block with at most half as many rows as SMs: c = SMs / R CTAs per row, so that every CTA
-    // streams one part of one row (one ticket, no tiny pieces at a boundary between two rows).  Measured along a run with resampling:
-    // 16 x 151936 bf16 20.7 -> 20.3 us per step, 32 x 151936 24.0 -> 23.0 us.
-    else if (R <= kSMs / 2 && gpr >= 2 * (kSMs / R)) {
+    // Larger rows of a block with no more rows than SMs: c = SMs / R CTAs per row (one whole row per CTA from 75 rows
+    // on), so that every CTA streams one part of one row (one ticket, no tiny pieces at a boundary between two rows;
+    // with c = 1 no ticket at all).  Measured along a run with resampling, rows of 151936 bf16 logits: 16 rows
+    // 20.7 -> 20.3 us per step, 32 rows 24.0 -> 23.0 us, 64 rows 28.2 -> 23.6 us, 100 rows 31.2 -> 23.3 us, 128 rows
+    // 33.4 -> 23.7 us.  (Whole rows for larger blocks, three or four to a CTA, lose more to the uneven shares than
+    // they gain: 512 x 128256 37.9 -> 39.7 us.)
+    else if (R <= kSMs && gpr >= 2 * (kSMs / R)) {
         g.per_row = kSMs / R;
         grid = R * g.per_row;
         g.base = (int)(gpr / g.per_row);
