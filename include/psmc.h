@@ -409,6 +409,18 @@ psmc_status psmc_state_load(psmc_ctx*, const void* host_buf, size_t bytes);
 psmc_status psmc_timing_enable(psmc_ctx*, int on);
 psmc_status psmc_timing_read(psmc_ctx*, double* ms_out, int64_t* launches_out);
 
+/* Diagnostic, host only (no GPU, no context): how the one-kernel form of psmc_step (Algorithm 1's loop body without the
+ * cache move) deals a block of R rows x V logits to its CTAs.  Rows are cut into granules of 512 bytes; CTA b streams
+ * the granules [shares_out[b], shares_out[b + 1]) of the block in row-major order.  layout_out: HOST array of 8:
+ * [0] 1 if the shape fits the one-kernel form (16-byte aligned rows assumed), else 0; [1] CTAs; [2] streaming warps per
+ * CTA; [3] granules per row; [4] bound on the rows one CTA's share meets; [5] CTAs per row when every row is dealt to
+ * CTAs of its own, else 0; [6] bytes of a row that bulk copies fetch; [7] logits of a row after them.  shares_out: HOST
+ * array of at least CTAs + 1 entries (shares_cap says how many there are), or NULL.  PSMC_E_INVAL: bad arguments or an
+ * array too short.  psmc_step_share_of: the CTA whose share holds a granule, -1 for a granule outside the block or a
+ * shape that does not fit.  (The paper has no counterpart: this is the kernel's own work division, exposed for tests.) */
+psmc_status psmc_step_layout(int R, int V, psmc_dtype dt, int32_t* layout_out, int32_t* shares_out, int shares_cap);
+int psmc_step_share_of(int R, int V, psmc_dtype dt, int granule);
+
 /* Synchronises `stream` and returns the sticky device status word (PSMC_OK if
  * nothing went wrong since the last reset). */
 psmc_status psmc_sync_status(psmc_ctx*, void* stream);

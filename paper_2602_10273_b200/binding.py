@@ -70,6 +70,10 @@ def lib():
         L.psmc_step_host.argtypes = [vp, vp, C.c_int, C.c_int64, vp, vp]
         L.psmc_logits_pass_scratch_bytes.restype = C.c_size_t
         L.psmc_logits_pass_scratch_bytes.argtypes = [C.c_int, C.c_int]
+        L.psmc_step_layout.restype = C.c_int
+        L.psmc_step_layout.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_int]
+        L.psmc_step_share_of.restype = C.c_int
+        L.psmc_step_share_of.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
         L.psmc_logits_pass.restype = C.c_int
         L.psmc_logits_pass.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_double, C.c_double, f64p, u8p,
                                        vp, C.c_size_t, i32p, f64p, f64p, i32p, vp]
@@ -421,6 +425,19 @@ def init_batched(G, N, V, alpha, tau, ess_thresh, ramp, seed, eos_id, T_max, pro
 
 def logits_pass_scratch_bytes(R: int, V: int) -> int:
     return lib().psmc_logits_pass_scratch_bytes(R, V)
+
+
+def step_layout(R: int, V: int, dtype_code: int):
+    """psmc_step_layout: (the eight layout words, the CTAs' first granules followed by the total); host only."""
+    words = (C.c_int32 * 8)()
+    _check(lib().psmc_step_layout(R, V, dtype_code, words, None, 0), "psmc_step_layout")
+    shares = (C.c_int32 * (words[1] + 1))()
+    _check(lib().psmc_step_layout(R, V, dtype_code, words, shares, len(shares)), "psmc_step_layout")
+    return list(words), list(shares)
+
+
+def step_share_of(R: int, V: int, dtype_code: int, granule: int) -> int:
+    return lib().psmc_step_share_of(R, V, dtype_code, granule)
 
 
 def logits_pass(logits: torch.Tensor, beta: float, alpha_t: float, u: torch.Tensor, done, scratch: torch.Tensor,

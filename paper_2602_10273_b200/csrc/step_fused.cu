@@ -711,3 +711,34 @@ cudaError_t launch_step_fused(const LogitsStreamArgs& la, const WeightsArgs& wa,
 }
 
 }  // namespace psmc
+
+// ---- host-only queries of the dealing (tests of the geometry need no GPU) ----
+extern "C" psmc_status psmc_step_layout(int R, int V, psmc_dtype dt, int32_t* layout_out, int32_t* shares_out,
+                                        int shares_cap) {
+    if (R <= 0 || V <= 0 || (dt != PSMC_F32 && dt != PSMC_BF16) || !layout_out) return PSMC_E_INVAL;
+    psmc::StepGeom g;
+    int grid = 0;
+    const bool ok = psmc::step_geometry(R, V, dt, g, grid);
+    layout_out[0] = ok ? 1 : 0;
+    layout_out[1] = grid;
+    layout_out[2] = g.W;
+    layout_out[3] = g.gpr;
+    layout_out[4] = g.seg_cap;
+    layout_out[5] = g.per_row;
+    layout_out[6] = g.row_bytes16;
+    layout_out[7] = g.tail;
+    if (shares_out) {
+        if (shares_cap < grid + 1) return PSMC_E_INVAL;
+        for (int b = 0; b < grid; ++b) shares_out[b] = psmc::share_first(g, b);
+        shares_out[grid] = psmc::share_first(g, grid - 1) + psmc::share_count(g, grid - 1);
+    }
+    return PSMC_OK;
+}
+extern "C" int psmc_step_share_of(int R, int V, psmc_dtype dt, int granule) {
+    psmc::StepGeom g;
+    int grid = 0;
+    if (R <= 0 || V <= 0 || (dt != PSMC_F32 && dt != PSMC_BF16) || !psmc::step_geometry(R, V, dt, g, grid)) return -1;
+    if (granule < 0 || (int64_t)granule >= (int64_t)R * g.gpr) return -1;
+    return psmc::share_of(g, granule);
+}
+
